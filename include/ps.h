@@ -1,0 +1,214 @@
+/*
+ * ps.h -- C interface of the HBM-resident parameter store.
+ *
+ * One NVIDIA B200 holds every parameter row, a location table
+ * key -> (owner, slot) and one free-slot stack per logical worker.  The calls
+ * are the primitives of a parameter server with dynamic parameter allocation
+ * (Renz-Wieland et al., VLDB 2020): pull and push (Section 2.1, Table 2),
+ * localize (Sections 2.3, 3.1, 3.2), plus three fused minibatch steps
+ * (pull -> per-example gradient -> push) for the tasks of Section 4.1.
+ *
+ * Conventions that hold for every call
+ * ------------------------------------
+ * Memory.   The library never allocates device memory.  Every `d_*` pointer is
+ *           DEVICE memory owned by the caller and must stay valid until the
+ *           stream has executed the call.  Every `h_*` pointer is HOST memory
+ *           owned by the caller.  The library owns only the host handle.
+ * Streams.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *           Every call except ps_create/ps_destroy/ps_sync/ps_export*, the
+ *           counters and the `*_host` variants only enqueues work and returns;
+ *           stream order is program order, which gives each key a single
+ *           serial history (the per-key sequential consistency of Section 3.4).
+ * Keys.     Dense in [0, num_keys) (the dense store of Section 3.7); duplicates
+ *           are allowed in every key list: pull returns one row per
+ *           occurrence, push sums, localize collapses.
+ * Batch semantics.  Inside one call every read sees the state before the call;
+ *           all additive terms of the call are summed per key (fp64) and added
+ *           once, row = (float)((double)row + sum).  Results do not depend on
+ *           thread scheduling: there are no floating-point atomics.
+ * Errors.   Host-detectable errors (null pointer, size beyond the workspace,
+ *           worker out of range) return at once and enqueue nothing.  Errors
+ *           only the device can see (key out of range, partition full) make the
+ *           offending CALL a no-op for store, table and free lists, latch the
+ *           first such code on the device, and surface at the next ps_sync.
+ *           Nothing ever traps, asserts or aborts.
+ */
+#ifndef PS_B200_PS_H
+#define PS_B200_PS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ps_store ps_store_t;     /* opaque host handle */
+typedef int ps_status_t;
+
+enum {
+    PS_OK = 0,
+    PS_ERR_INVALID_ARG = 1,     /* null pointer, zero size where one is needed, bad config */
+    PS_ERR_KEY_RANGE = 2,       /* a key (or an index that forms one) is >= num_keys */
+    PS_ERR_WORKER_RANGE = 3,    /* worker >= num_workers */
+    PS_ERR_CAPACITY = 4,        /* localize: the requester's partition has too few free slots */
+    PS_ERR_WORKSPACE = 5,       /* the call needs more key occurrences than the workspace was sized for */
+    PS_ERR_CUDA = 6,            /* a CUDA runtime call failed */
+    PS_ERR_UNSUPPORTED = 7      /* configuration outside what the kernels implement */
+};
+
+typedef struct {
+    uint64_t num_keys;          /* K; must be < 2^32 - 1 */
+    uint32_t row_len;           /* fp32 values per key, optimizer state included; multiple of 4 */
+    uint32_t num_workers;       /* N logical workers = partitions of the store; <= 65536 */
+    uint64_t slots_per_part;    /* S, capacity of each partition; >= ceil(K/N), < 2^32 */
+    int32_t device;             /* CUDA device ordinal */
+} ps_config_t;
+
+typedef struct {
+    size_t store_bytes;         /* N * S * row_len * 4 */
+    size_t table_bytes;         /* K * 8: (uint32 owner, uint32 slot) per key */
+    size_t freelist_bytes;      /* N stack heights, then N stacks of S uint32 */
+    size_t workspace_bytes;     /* scratch for calls of up to max_batch_keys key occurrences */
+} ps_sizes_t;
+
+/* Sizes of the four device buffers the caller must allocate (256-byte aligned).
+ * `max_batch_keys` bounds the key occurrences of any later call: n for
+ * pull/push/localize, 2n for ps_step_mf, (3 + n_neg) * n for ps_step_kge,
+ * n_centers * (1 + 2 * window * (1 + n_neg)) for ps_step_sgns. */
+ps_status_t ps_query_sizes(const ps_config_t* cfg, uint64_t max_batch_keys, ps_sizes_t* out);
+
+/* Creates the host handle around caller-allocated device buffers of at least
+ * the queried sizes.  Synchronous.  The store's contents are left as they are;
+ * call ps_init_range_partition before anything else. */
+ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void* d_freelists,
+                      void* d_workspace, size_t workspace_bytes, uint64_t max_batch_keys,
+                      ps_store_t** out);
+
+/* Frees the host handle only (after synchronising the device work it issued). */
+ps_status_t ps_destroy(ps_store_t* ps);
+
+/* Static initial allocation by range partitioning (Section 3.5; classic PSs,
+ * Section 2.1): with B = ceil(K/N), key k goes to owner k / B, slot k % B.
+ * Partition p's free stack then holds S-1, ..., cnt_p bottom to top, so its
+ * lowest free slot is taken first.  Row values are not touched. */
+ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream);
+
+/* Overwrites the rows of `d_keys` (n keys, distinct) with `d_vals` (n x row_len). */
+ps_status_t ps_set_rows(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_vals,
+                        void* stream);
+
+/* pull (Table 2): d_out[t, :] = current row of d_keys[t], t < n; location-transparent. */
+ps_status_t ps_pull(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, float* d_out, void* stream);
+
+/* push (Table 2; cumulative, Section 2.1): row(k) += sum over {t : d_keys[t] = k} of
+ * d_updates[t, :].  Occurrences are sorted by key and reduced segment by segment. */
+ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_updates,
+                    void* stream);
+
+/* localize (Sections 3.1, 3.2): every distinct key of the call that `worker` does
+ * not own moves, with its whole row, into worker's partition, and the location
+ * table is rewritten -- the end state of the relocation protocol of Figure 4.
+ * Calls apply in stream order, so a key localized by several workers ends at
+ * the last requester (localization conflicts, Section 3.2).
+ * Slot policy: moved keys in ascending order; the m-th takes the m-th slot from
+ * the top of worker's free stack; afterwards each vacated slot is pushed onto
+ * its old owner's stack, ascending by key.  If worker has fewer free slots
+ * than keys to move: PS_ERR_CAPACITY is latched and nothing changes. */
+ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n,
+                        void* stream);
+
+/* One SGD minibatch of low-rank matrix factorization (task of Section 4.1).
+ * Key i is row factor w_i (i < col_key_base); key col_key_base + j is column
+ * factor h_j.  For each of n cells (d_i[t], d_j[t], d_v[t]), at the pre-batch
+ * state: e = v - <w, h>; loss e^2/2 + lambda/2 (|w|^2 + |h|^2);
+ * w += lr (e h - lambda w), h += lr (e w - lambda h), summed per key.
+ * *d_loss_accum (device, may be NULL) += the batch's loss. */
+ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
+                       uint64_t n, uint64_t col_key_base, float lr, float lambda,
+                       double* d_loss_accum, void* stream);
+
+/* One minibatch of ComplEx with AdaGrad and negative sampling (Section 4.1,
+ * Appendix A).  Key e is an entity (e < rel_key_base), key rel_key_base + r a
+ * relation.  A row is [Re | Im | G_Re | G_Im], dim_complex fp32 each
+ * (row_len = 4 * dim_complex); G are the AdaGrad accumulators.
+ * Data point t = triple (d_s[t], d_r[t], d_o[t]) plus n_neg negatives
+ * (n_neg <= 29): negative q replaces the subject (d_neg_side[t*n_neg+q] = 0)
+ * or the object (1) by entity d_neg_ent[t*n_neg+q].  Score
+ * phi = Re sum e_s w_r conj(e_o); loss softplus(-y phi).  For each distinct
+ * key of a data point, g = its gradient of the data point's loss at the
+ * pre-batch state; the call pushes dG = g*g and
+ * dtheta = -lr g / (sqrt(G + g*g) + eps), summed per key. */
+ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                        const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n,
+                        uint32_t n_neg, uint64_t rel_key_base, uint32_t dim_complex, float lr,
+                        float eps, double* d_loss_accum, void* stream);
+
+/* One minibatch of skip-gram with negative sampling (Section 4.1, Appendix A).
+ * Key w is the input vector of word w (w < out_key_base), key out_key_base + w
+ * its output vector.  d_tokens is the whole stream (corpus_len tokens); the
+ * centers are positions [first_pos, first_pos + n_centers); contexts of p are
+ * the positions q != p, |q - p| <= window, inside the stream.  Pairs (p, q) are
+ * numbered from 0 in (p, q) ascending order; pair z uses
+ * d_negs[z*n_neg .. z*n_neg + n_neg).  Per pair and target (u, y) in
+ * {(context, 1), (negative, 0)...}: x = <v, u>, g = sigmoid(x) - y,
+ * u += -lr g v, v += -lr g u, summed per key.  row_len <= 512. */
+ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t first_pos,
+                         uint64_t n_centers, uint64_t corpus_len, uint32_t window,
+                         const uint32_t* d_negs, uint32_t n_neg, uint64_t out_key_base, float lr,
+                         double* d_loss_accum, void* stream);
+
+/* The same steps for callers whose batch lives in HOST memory (pinned memory
+ * makes the copies asynchronous).  Each copies the batch into the workspace,
+ * runs the step, copies the accumulated loss back to *h_loss and waits for the
+ * stream.  ps_step_sgns_host takes the tokens [tok_first, tok_first + tok_count)
+ * that cover the batch's window; first_pos and corpus_len stay absolute. */
+ps_status_t ps_step_mf_host(ps_store_t* ps, const uint32_t* h_i, const uint32_t* h_j, const float* h_v,
+                            uint64_t n, uint64_t col_key_base, float lr, float lambda,
+                            double* d_loss_accum, double* h_loss, void* stream);
+ps_status_t ps_step_kge_host(ps_store_t* ps, const uint32_t* h_s, const uint32_t* h_r, const uint32_t* h_o,
+                             const uint32_t* h_neg_ent, const uint8_t* h_neg_side, uint64_t n,
+                             uint32_t n_neg, uint64_t rel_key_base, uint32_t dim_complex, float lr,
+                             float eps, double* d_loss_accum, double* h_loss, void* stream);
+ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t tok_first,
+                              uint64_t tok_count, uint64_t first_pos, uint64_t n_centers,
+                              uint64_t corpus_len, uint32_t window, const uint32_t* h_negs,
+                              uint64_t n_negs, uint32_t n_neg, uint64_t out_key_base, float lr,
+                              double* d_loss_accum, double* h_loss, void* stream);
+
+/* d_owner[t], d_slot[t] = current location of d_keys[t]. */
+ps_status_t ps_get_location(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner,
+                            uint32_t* d_slot, void* stream);
+
+/* Synchronous copies for tests.  ps_export: rows by key (K x row_len), owner
+ * and slot of every key (any pointer may be NULL to skip it).
+ * ps_export_freelists: the N stacks (N x S, entries above a stack's height are
+ * unspecified) and the N heights. */
+ps_status_t ps_export(ps_store_t* ps, float* h_rows_by_key, uint32_t* h_owner, uint32_t* h_slot);
+ps_status_t ps_export_freelists(ps_store_t* ps, uint32_t* h_stacks, uint64_t* h_tops);
+
+/* Waits for `stream`; returns and clears the first error latched on the device. */
+ps_status_t ps_sync(ps_store_t* ps, void* stream);
+
+/* Number of kernels this handle has launched so far. */
+uint64_t ps_launch_count(const ps_store_t* ps);
+
+/* Synchronous: *h_out = rows relocated by all successful ps_localize calls of this handle. */
+ps_status_t ps_rows_moved(ps_store_t* ps, uint64_t* h_out);
+
+/* Per-kernel timing for measurement runs.  After ps_profile_start the next
+ * `max_launches` kernel launches of this handle are bracketed by CUDA events on
+ * their stream.  ps_profile_stop waits for the device, writes one line per
+ * kernel, "name launches total_microseconds\n", in first-launch order, into
+ * h_report (NUL-terminated, truncated to `capacity` bytes) and turns timing off.
+ * The events add a little time between kernels: do not time a run end to end
+ * while profiling is on. */
+ps_status_t ps_profile_start(ps_store_t* ps, uint32_t max_launches);
+ps_status_t ps_profile_stop(ps_store_t* ps, char* h_report, size_t capacity);
+
+const char* ps_status_string(ps_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PS_B200_PS_H */

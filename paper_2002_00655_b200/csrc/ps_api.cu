@@ -1,0 +1,501 @@
+// The exported C interface (include/ps.h): argument checks, workspace layout,
+// and the order in which the kernels of a call are enqueued.
+#include <map>
+#include <new>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string>
+#include <string.h>
+#include <vector>
+
+#include "ps_internal.cuh"
+
+namespace psb {
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
+    WsLayout l;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        const size_t at = off;
+        off = align_up(off + bytes, 256);
+        return at;
+    };
+    const uint64_t mk = max_keys ? max_keys : 1;
+    const size_t sort_tiles = (mk + kSortTile - 1) / kSortTile;
+    const size_t reduce_tiles = (mk + kReduceTile - 1) / kReduceTile;
+    const size_t row_bytes = (size_t)cfg.row_len * 4;
+    l.status = take(sizeof(DevStatus));
+    l.keysA = take(mk * 4);
+    l.keysB = take(mk * 4);
+    l.valsA = take(mk * 4);
+    l.valsB = take(mk * 4);
+    l.hist = take(sort_tiles * kRadix * 4);
+    l.totals = take(kRadix * 4);
+    l.scan_sums = take(((mk + 255) / 256) * 4);
+    l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
+    l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
+    l.loss_partial = take(kMaxLossBlocks * 8);
+    l.staging = take(mk * 8 + 256);
+    l.total = off;
+    return l;
+}
+
+struct ProfRec {
+    const char* name;
+    cudaEvent_t a, b;
+};
+struct Profile {
+    std::vector<ProfRec> recs;
+    size_t cap;
+    bool open;          // an event pair has been started and not yet closed
+};
+
+void prof_before(ps_store* ps, const char* name, cudaStream_t s) {
+    Profile* p = ps->prof;
+    p->open = false;
+    if (p->recs.size() >= p->cap) return;
+    ProfRec r;
+    r.name = name;
+    if (cudaEventCreate(&r.a) != cudaSuccess) return;
+    if (cudaEventCreate(&r.b) != cudaSuccess) {
+        cudaEventDestroy(r.a);
+        return;
+    }
+    cudaEventRecord(r.a, s);
+    p->recs.push_back(r);
+    p->open = true;
+}
+
+void prof_after(ps_store* ps, cudaStream_t s) {
+    Profile* p = ps->prof;
+    if (p->open) cudaEventRecord(p->recs.back().b, s);
+    p->open = false;
+}
+
+static int bits_for(uint64_t max_value) {
+    int b = 0;
+    while (b < 32 && (max_value >> b) != 0) ++b;
+    return b < 1 ? 1 : b;
+}
+
+static ps_status_t check_cfg(const ps_config_t* cfg) {
+    if (!cfg) return PS_ERR_INVALID_ARG;
+    if (cfg->num_keys == 0 || cfg->row_len == 0 || cfg->num_workers == 0) return PS_ERR_INVALID_ARG;
+    if (cfg->num_keys >= 0xFFFFFFFFull) return PS_ERR_UNSUPPORTED;
+    if (cfg->row_len % 4 != 0) return PS_ERR_UNSUPPORTED;
+    if (cfg->num_workers > 65536) return PS_ERR_UNSUPPORTED;
+    const uint64_t B = (cfg->num_keys + cfg->num_workers - 1) / cfg->num_workers;
+    if (cfg->slots_per_part < B) return PS_ERR_INVALID_ARG;
+    if (cfg->slots_per_part >= 0xFFFFFFFFull) return PS_ERR_UNSUPPORTED;
+    return PS_OK;
+}
+
+static ps_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? PS_OK : PS_ERR_CUDA; }
+
+// Errors raised by a launch itself (bad configuration) show up here; errors inside kernels
+// are reported through the device status word.
+static ps_status_t after_launch() { return cuda_ok(cudaGetLastError()); }
+
+static void next_epoch(ps_store* ps) {
+    ps->epoch++;
+    if (ps->epoch == 0) ps->epoch = 1;
+}
+
+}  // namespace psb
+
+using namespace psb;
+
+extern "C" {
+
+ps_status_t ps_query_sizes(const ps_config_t* cfg, uint64_t max_batch_keys, ps_sizes_t* out) {
+    if (!out) return PS_ERR_INVALID_ARG;
+    const ps_status_t c = check_cfg(cfg);
+    if (c != PS_OK) return c;
+    if (max_batch_keys == 0 || max_batch_keys >= 0x7FFFFFFFull) return PS_ERR_INVALID_ARG;
+    const uint64_t N = cfg->num_workers, S = cfg->slots_per_part;
+    out->store_bytes = (size_t)(N * S) * cfg->row_len * 4;
+    out->table_bytes = (size_t)cfg->num_keys * 8;
+    out->freelist_bytes = align_up((size_t)N * 8, 256) + (size_t)(N * S) * 4;
+    out->workspace_bytes = ws_layout(*cfg, max_batch_keys).total;
+    return PS_OK;
+}
+
+ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void* d_freelists, void* d_workspace,
+                      size_t workspace_bytes, uint64_t max_batch_keys, ps_store_t** out) {
+    if (!out || !d_store || !d_table || !d_freelists || !d_workspace) return PS_ERR_INVALID_ARG;
+    ps_sizes_t sz;
+    const ps_status_t c = ps_query_sizes(cfg, max_batch_keys, &sz);
+    if (c != PS_OK) return c;
+    if (workspace_bytes < sz.workspace_bytes) return PS_ERR_WORKSPACE;
+    if (((uintptr_t)d_store | (uintptr_t)d_table | (uintptr_t)d_freelists | (uintptr_t)d_workspace) & 15)
+        return PS_ERR_INVALID_ARG;
+    if (cudaSetDevice(cfg->device) != cudaSuccess) return PS_ERR_CUDA;
+    ps_store* ps = new (std::nothrow) ps_store();
+    if (!ps) return PS_ERR_INVALID_ARG;
+    memset(ps, 0, sizeof(*ps));
+    ps->cfg = *cfg;
+    ps->max_keys = max_batch_keys;
+    ps->key_bits = bits_for(cfg->num_keys);                 // keys 0..K, K marks "no key"
+    ps->owner_bits = bits_for(cfg->num_workers - 1);
+    ps->store = (float*)d_store;
+    ps->table = (uint2*)d_table;
+    ps->tops = (unsigned long long*)d_freelists;
+    ps->stacks = (uint32_t*)((char*)d_freelists + align_up((size_t)cfg->num_workers * 8, 256));
+    ps->ws = (char*)d_workspace;
+    ps->ws_bytes = workspace_bytes;
+    const WsLayout l = ws_layout(*cfg, max_batch_keys);
+    ps->status = (DevStatus*)(ps->ws + l.status);
+    ps->keysA = (uint32_t*)(ps->ws + l.keysA);
+    ps->keysB = (uint32_t*)(ps->ws + l.keysB);
+    ps->valsA = (uint32_t*)(ps->ws + l.valsA);
+    ps->valsB = (uint32_t*)(ps->ws + l.valsB);
+    ps->hist = (uint32_t*)(ps->ws + l.hist);
+    ps->totals = (uint32_t*)(ps->ws + l.totals);
+    ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
+    ps->upd = (float*)(ps->ws + l.upd);
+    ps->carry = (double*)(ps->ws + l.carry);
+    ps->loss_partial = (double*)(ps->ws + l.loss_partial);
+    ps->staging = ps->ws + l.staging;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0) {
+        delete ps;
+        return PS_ERR_CUDA;
+    }
+    ps->sm_count = sms;
+    if (cudaMemset(ps->status, 0, sizeof(DevStatus)) != cudaSuccess) {
+        delete ps;
+        return PS_ERR_CUDA;
+    }
+    *out = ps;
+    return PS_OK;
+}
+
+ps_status_t ps_destroy(ps_store_t* ps) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    cudaSetDevice(ps->cfg.device);
+    cudaDeviceSynchronize();
+    if (ps->prof) ps_profile_stop(ps, nullptr, 0);
+    delete ps;
+    return PS_OK;
+}
+
+#define PS_BEGIN_CALL(ps)                                            \
+    if (!(ps)) return PS_ERR_INVALID_ARG;                           \
+    cudaStream_t s = (cudaStream_t)stream;                          \
+    next_epoch(ps);
+
+ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
+    PS_BEGIN_CALL(ps);
+    launch_init_range_partition(ps, s);
+    return after_launch();
+}
+
+ps_status_t ps_set_rows(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_vals, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_keys || !d_vals) return PS_ERR_INVALID_ARG;
+    launch_set_rows(ps, d_keys, n, d_vals, s);
+    return after_launch();
+}
+
+ps_status_t ps_pull(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, float* d_out, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_keys || !d_out) return PS_ERR_INVALID_ARG;
+    launch_pull(ps, d_keys, n, d_out, s);
+    return after_launch();
+}
+
+ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_updates, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_keys || !d_updates) return PS_ERR_INVALID_ARG;
+    if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    launch_prepare_keys(ps, d_keys, n, s);
+    run_push_pipeline(ps, (uint32_t)n, d_updates, nullptr, 0, s);
+    return after_launch();
+}
+
+ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (worker >= ps->cfg.num_workers) return PS_ERR_WORKER_RANGE;
+    if (n == 0) return PS_OK;
+    if (!d_keys) return PS_ERR_INVALID_ARG;
+    if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    launch_prepare_keys(ps, d_keys, n, s);
+    run_localize(ps, worker, (uint32_t)n, s);
+    return after_launch();
+}
+
+ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
+                       uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_i || !d_j || !d_v) return PS_ERR_INVALID_ARG;
+    if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
+    if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
+    run_push_pipeline(ps, (uint32_t)(2 * n), ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    return after_launch();
+}
+
+ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                        const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
+                        uint64_t rel_key_base, uint32_t dim_complex, float lr, float eps, double* d_loss_accum,
+                        void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_s || !d_r || !d_o || (n_neg && (!d_neg_ent || !d_neg_side))) return PS_ERR_INVALID_ARG;
+    if (n_neg > 29) return PS_ERR_UNSUPPORTED;
+    if (dim_complex == 0 || ps->cfg.row_len != 4 * (uint64_t)dim_complex) return PS_ERR_INVALID_ARG;
+    if ((3 + (uint64_t)n_neg) * n > ps->max_keys) return PS_ERR_WORKSPACE;
+    if (rel_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    const uint32_t lb =
+        launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex, lr, eps, s);
+    run_push_pipeline(ps, (uint32_t)((3 + (uint64_t)n_neg) * n), ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    return after_launch();
+}
+
+static ps_status_t sgns_checks(ps_store_t* ps, uint64_t first_pos, uint64_t n_centers, uint64_t corpus_len,
+                               uint32_t window, uint32_t n_neg, uint64_t out_key_base, uint64_t* occ) {
+    if (first_pos + n_centers > corpus_len) return PS_ERR_INVALID_ARG;
+    if (ps->cfg.row_len > 512) return PS_ERR_UNSUPPORTED;
+    if (out_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    *occ = n_centers * (1 + (uint64_t)2 * window * (1 + (uint64_t)n_neg));
+    if (*occ > ps->max_keys) return PS_ERR_WORKSPACE;
+    return PS_OK;
+}
+
+ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t first_pos, uint64_t n_centers,
+                         uint64_t corpus_len, uint32_t window, const uint32_t* d_negs, uint32_t n_neg,
+                         uint64_t out_key_base, float lr, double* d_loss_accum, void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n_centers == 0) return PS_OK;
+    if (!d_tokens || (n_neg && window && !d_negs)) return PS_ERR_INVALID_ARG;
+    uint64_t occ;
+    const ps_status_t c = sgns_checks(ps, first_pos, n_centers, corpus_len, window, n_neg, out_key_base, &occ);
+    if (c != PS_OK) return c;
+    const uint32_t lb = launch_step_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
+                                         out_key_base, lr, s);
+    run_push_pipeline(ps, (uint32_t)occ, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    return after_launch();
+}
+
+// ---- host-batch variants ----
+static ps_status_t finish_host_step(double* d_loss_accum, double* h_loss, cudaStream_t s) {
+    if (d_loss_accum && h_loss &&
+        cudaMemcpyAsync(h_loss, d_loss_accum, sizeof(double), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return PS_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return PS_ERR_CUDA;
+    return PS_OK;
+}
+
+ps_status_t ps_step_mf_host(ps_store_t* ps, const uint32_t* h_i, const uint32_t* h_j, const float* h_v, uint64_t n,
+                            uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, double* h_loss,
+                            void* stream) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (n == 0) return PS_OK;
+    if (!h_i || !h_j || !h_v) return PS_ERR_INVALID_ARG;
+    if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t* d_i = (uint32_t*)ps->staging;
+    uint32_t* d_j = d_i + n;
+    float* d_v = (float*)(d_j + n);
+    if (cudaMemcpyAsync(d_i, h_i, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(d_j, h_j, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(d_v, h_v, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PS_ERR_CUDA;
+    const ps_status_t c = ps_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, d_loss_accum, stream);
+    if (c != PS_OK) return c;
+    return finish_host_step(d_loss_accum, h_loss, s);
+}
+
+ps_status_t ps_step_kge_host(ps_store_t* ps, const uint32_t* h_s, const uint32_t* h_r, const uint32_t* h_o,
+                             const uint32_t* h_neg_ent, const uint8_t* h_neg_side, uint64_t n, uint32_t n_neg,
+                             uint64_t rel_key_base, uint32_t dim_complex, float lr, float eps, double* d_loss_accum,
+                             double* h_loss, void* stream) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (n == 0) return PS_OK;
+    if (!h_s || !h_r || !h_o || (n_neg && (!h_neg_ent || !h_neg_side))) return PS_ERR_INVALID_ARG;
+    if ((3 + (uint64_t)n_neg) * n > ps->max_keys) return PS_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t* d_s = (uint32_t*)ps->staging;
+    uint32_t* d_r = d_s + n;
+    uint32_t* d_o = d_r + n;
+    uint32_t* d_ne = d_o + n;
+    uint8_t* d_ns = (uint8_t*)(d_ne + n * n_neg);
+    if (cudaMemcpyAsync(d_s, h_s, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(d_r, h_r, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(d_o, h_o, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PS_ERR_CUDA;
+    if (n_neg && (cudaMemcpyAsync(d_ne, h_neg_ent, n * n_neg * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+                  cudaMemcpyAsync(d_ns, h_neg_side, n * n_neg, cudaMemcpyHostToDevice, s) != cudaSuccess))
+        return PS_ERR_CUDA;
+    const ps_status_t c = ps_step_kge(ps, d_s, d_r, d_o, d_ne, d_ns, n, n_neg, rel_key_base, dim_complex, lr, eps,
+                                      d_loss_accum, stream);
+    if (c != PS_OK) return c;
+    return finish_host_step(d_loss_accum, h_loss, s);
+}
+
+ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t tok_first, uint64_t tok_count,
+                              uint64_t first_pos, uint64_t n_centers, uint64_t corpus_len, uint32_t window,
+                              const uint32_t* h_negs, uint64_t n_negs, uint32_t n_neg, uint64_t out_key_base,
+                              float lr, double* d_loss_accum, double* h_loss, void* stream) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (n_centers == 0) return PS_OK;
+    if (!h_tokens || (n_negs && !h_negs)) return PS_ERR_INVALID_ARG;
+    uint64_t occ;
+    ps_status_t c = sgns_checks(ps, first_pos, n_centers, corpus_len, window, n_neg, out_key_base, &occ);
+    if (c != PS_OK) return c;
+    // the tokens handed over must cover the batch's window
+    const uint64_t need_lo = first_pos >= window ? first_pos - window : 0;
+    uint64_t need_hi = first_pos + n_centers - 1 + window;
+    if (need_hi > corpus_len - 1) need_hi = corpus_len - 1;
+    if (tok_first > need_lo || tok_first + tok_count <= need_hi) return PS_ERR_INVALID_ARG;
+    if ((tok_count + n_negs) * 4 > ps->max_keys * 8) return PS_ERR_WORKSPACE;
+    cudaStream_t s = (cudaStream_t)stream;
+    next_epoch(ps);
+    uint32_t* d_tok = (uint32_t*)ps->staging;
+    uint32_t* d_negs = d_tok + tok_count;
+    if (cudaMemcpyAsync(d_tok, h_tokens, tok_count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return PS_ERR_CUDA;
+    if (n_negs && cudaMemcpyAsync(d_negs, h_negs, n_negs * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return PS_ERR_CUDA;
+    const uint32_t lb = launch_step_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
+                                         out_key_base, lr, s);
+    run_push_pipeline(ps, (uint32_t)occ, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    c = after_launch();
+    if (c != PS_OK) return c;
+    return finish_host_step(d_loss_accum, h_loss, s);
+}
+
+ps_status_t ps_get_location(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner, uint32_t* d_slot,
+                            void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_keys || !d_owner || !d_slot) return PS_ERR_INVALID_ARG;
+    launch_get_location(ps, d_keys, n, d_owner, d_slot, s);
+    return after_launch();
+}
+
+ps_status_t ps_export(ps_store_t* ps, float* h_rows_by_key, uint32_t* h_owner, uint32_t* h_slot) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;
+    const uint64_t K = ps->cfg.num_keys;
+    const uint32_t L = ps->cfg.row_len;
+    if (h_rows_by_key) {
+        const uint64_t chunk = ps->max_keys;                // rows that fit in the update-row scratch
+        for (uint64_t k0 = 0; k0 < K; k0 += chunk) {
+            const uint64_t c = K - k0 < chunk ? K - k0 : chunk;
+            launch_gather_rows_by_key(ps, k0, c, ps->upd, 0);
+            if (cudaMemcpy(h_rows_by_key + k0 * L, ps->upd, c * L * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+                return PS_ERR_CUDA;
+        }
+    }
+    if (h_owner || h_slot) {
+        uint2* tmp = (uint2*)malloc(K * sizeof(uint2));
+        if (!tmp) return PS_ERR_INVALID_ARG;
+        if (cudaMemcpy(tmp, ps->table, K * sizeof(uint2), cudaMemcpyDeviceToHost) != cudaSuccess) {
+            free(tmp);
+            return PS_ERR_CUDA;
+        }
+        for (uint64_t k = 0; k < K; ++k) {
+            if (h_owner) h_owner[k] = tmp[k].x;
+            if (h_slot) h_slot[k] = tmp[k].y;
+        }
+        free(tmp);
+    }
+    return after_launch();
+}
+
+ps_status_t ps_export_freelists(ps_store_t* ps, uint32_t* h_stacks, uint64_t* h_tops) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;
+    const uint64_t N = ps->cfg.num_workers, S = ps->cfg.slots_per_part;
+    if (h_stacks && cudaMemcpy(h_stacks, ps->stacks, N * S * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PS_ERR_CUDA;
+    if (h_tops && cudaMemcpy(h_tops, ps->tops, N * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
+    return PS_OK;
+}
+
+ps_status_t ps_sync(ps_store_t* ps, void* stream) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return PS_ERR_CUDA;
+    unsigned int code = 0;
+    if (cudaMemcpy(&code, &ps->status->sticky, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
+    if (code != 0 && cudaMemset(&ps->status->sticky, 0, 4) != cudaSuccess) return PS_ERR_CUDA;
+    return (ps_status_t)code;
+}
+
+uint64_t ps_launch_count(const ps_store_t* ps) { return ps ? ps->launches : 0; }
+
+ps_status_t ps_rows_moved(ps_store_t* ps, uint64_t* h_out) {
+    if (!ps || !h_out) return PS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;
+    unsigned long long v = 0;
+    if (cudaMemcpy(&v, &ps->status->rows_moved, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
+    *h_out = v;
+    return PS_OK;
+}
+
+ps_status_t ps_profile_start(ps_store_t* ps, uint32_t max_launches) {
+    if (!ps || ps->prof || max_launches == 0) return PS_ERR_INVALID_ARG;
+    Profile* p = new (std::nothrow) Profile();
+    if (!p) return PS_ERR_INVALID_ARG;
+    p->cap = max_launches;
+    p->open = false;
+    p->recs.reserve(max_launches);
+    ps->prof = p;
+    return PS_OK;
+}
+
+ps_status_t ps_profile_stop(ps_store_t* ps, char* h_report, size_t capacity) {
+    if (!ps || !ps->prof) return PS_ERR_INVALID_ARG;
+    Profile* p = ps->prof;
+    ps->prof = nullptr;
+    const ps_status_t rc = cudaDeviceSynchronize() == cudaSuccess ? PS_OK : PS_ERR_CUDA;
+    std::map<std::string, std::pair<uint64_t, double>> agg;
+    std::vector<std::string> order;
+    for (const ProfRec& r : p->recs) {
+        float ms = 0.f;
+        if (rc == PS_OK && cudaEventElapsedTime(&ms, r.a, r.b) == cudaSuccess) {
+            if (!agg.count(r.name)) order.push_back(r.name);
+            agg[r.name].first += 1;
+            agg[r.name].second += (double)ms * 1000.0;
+        }
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    delete p;
+    if (h_report && capacity) {
+        size_t used = 0;
+        h_report[0] = 0;
+        for (const std::string& name : order) {
+            char line[256];
+            const int len = snprintf(line, sizeof line, "%s %llu %.3f\n", name.c_str(),
+                                     (unsigned long long)agg[name].first, agg[name].second);
+            if (len < 0 || used + (size_t)len + 1 > capacity) break;
+            memcpy(h_report + used, line, (size_t)len + 1);
+            used += (size_t)len;
+        }
+    }
+    return rc;
+}
+
+const char* ps_status_string(ps_status_t status) {
+    switch (status) {
+        case PS_OK: return "ok";
+        case PS_ERR_INVALID_ARG: return "invalid argument";
+        case PS_ERR_KEY_RANGE: return "key out of range";
+        case PS_ERR_WORKER_RANGE: return "worker out of range";
+        case PS_ERR_CAPACITY: return "partition full";
+        case PS_ERR_WORKSPACE: return "workspace too small for this call";
+        case PS_ERR_CUDA: return "CUDA runtime error";
+        case PS_ERR_UNSUPPORTED: return "unsupported configuration";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,172 @@
+// Internal declarations shared by the translation units of the library.
+// Nothing here is part of the public interface (see include/ps.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ps.h"
+
+namespace psb {
+
+constexpr uint32_t kSentinelPad = 0xFFFFFFFFu;   // never a key: num_keys < 2^32 - 1
+constexpr int kSortThreads = 256;
+constexpr int kSortItems = 8;
+constexpr int kSortTile = kSortThreads * kSortItems;   // keys per sort block
+constexpr int kRadixBits = 8;
+constexpr int kRadix = 1 << kRadixBits;
+constexpr int kReduceTile = 32;                  // sorted occurrences per warp in the segmented reduction
+constexpr int kMaxLossBlocks = 4096;
+
+// Device-resident status words.  An error is latched per call with the call's
+// epoch, so no kernel has to clear anything before a call starts.
+struct DevStatus {
+    unsigned int sticky;            // first error code since the last ps_sync
+    unsigned int call_err_epoch;    // epoch of the last call that failed on the device
+    unsigned int moved_total;       // localize: number of keys that move in the current call
+    unsigned int pad;
+    unsigned long long rows_moved;  // rows relocated by all successful localize calls so far
+};
+
+struct Profile;
+
+}  // namespace psb
+
+struct ps_store {
+    ps_config_t cfg;
+    uint64_t max_keys;
+    int key_bits;                   // bits needed for keys 0..K inclusive (K is the "no key" mark)
+    int owner_bits;
+    // caller-owned device buffers
+    float* store;
+    uint2* table;                   // (owner, slot) per key
+    unsigned long long* tops;       // N stack heights
+    uint32_t* stacks;               // N x S
+    char* ws;
+    size_t ws_bytes;
+    // carved out of the workspace
+    psb::DevStatus* status;
+    uint32_t *keysA, *keysB, *valsA, *valsB;
+    uint32_t* hist;                 // kRadix x nSortTiles
+    uint32_t* totals;               // kRadix
+    uint32_t* scan_sums;            // block sums of the device-wide scan
+    float* upd;                     // max_keys x row_len update rows (also localize scratch)
+    double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
+    double* loss_partial;           // kMaxLossBlocks
+    char* staging;                  // host-batch staging, max_keys x 8 bytes
+    // host state
+    uint32_t epoch;
+    uint64_t launches;
+    int sm_count;
+    psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
+};
+
+namespace psb {
+
+struct WsLayout {
+    size_t status, keysA, keysB, valsA, valsB, hist, totals, scan_sums, upd, carry, loss_partial,
+        staging, total;
+};
+WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
+
+inline uint32_t div_up_u32(uint64_t a, uint64_t b) { return (uint32_t)((a + b - 1) / b); }
+template <class T> __host__ __device__ inline T tmin(T a, T b) { return a < b ? a : b; }
+template <class T> __host__ __device__ inline T tmax(T a, T b) { return a > b ? a : b; }
+
+// ---- ps_api.cu: optional per-kernel timing ----
+void prof_before(ps_store* ps, const char* name, cudaStream_t s);
+void prof_after(ps_store* ps, cudaStream_t s);
+
+#define PS_LAUNCH(ps, kernel, grid, block, stream, ...)                       \
+    do {                                                                     \
+        if ((ps)->prof) psb::prof_before((ps), #kernel, (stream));           \
+        kernel<<<(grid), (block), 0, (stream)>>>(__VA_ARGS__);               \
+        if ((ps)->prof) psb::prof_after((ps), (stream));                     \
+        (ps)->launches++;                                                    \
+    } while (0)
+
+// ---- sort.cu ----
+// Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key.
+// Input in the A buffers (start = 0) or the B buffers (start = 1); values are
+// implied as 0..n-1 when iota_vals.  If n_dev is not null the element count is
+// read from device memory (n is then an upper bound used for the launch
+// shapes).  Returns 0 if the result is in the A buffers, 1 if in the B buffers.
+int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
+                     cudaStream_t stream, int start);
+
+// ---- pull_push.cu ----
+void launch_init_range_partition(ps_store* ps, cudaStream_t s);
+void launch_set_rows(ps_store* ps, const uint64_t* d_keys, uint64_t n, const float* d_vals, cudaStream_t s);
+void launch_pull(ps_store* ps, const uint64_t* d_keys, uint64_t n, float* d_out, cudaStream_t s);
+void launch_get_location(ps_store* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner, uint32_t* d_slot,
+                         cudaStream_t s);
+void launch_gather_rows_by_key(ps_store* ps, uint64_t first_key, uint64_t n, float* d_out, cudaStream_t s);
+// keys64 -> keysA (range-checked)
+void launch_prepare_keys(ps_store* ps, const uint64_t* d_keys, uint64_t n, cudaStream_t s);
+// sort keysA (values = occurrence index), reduce `upd` rows per key, apply to the store, and add the
+// first `loss_blocks` loss partials to *d_loss_accum (if not null)
+void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
+                       cudaStream_t s);
+
+// ---- localize.cu ----
+void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s);
+
+// ---- steps.cu ----
+// Each writes the occurrences' keys to keysA and their update rows to `upd`, and
+// returns the number of per-block loss partials it wrote.
+uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
+                        uint64_t col_key_base, float lr, float lambda, cudaStream_t s);
+uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                         const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
+                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s);
+uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
+                          uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
+                          uint32_t n_neg, uint64_t out_key_base, float lr, cudaStream_t s);
+
+// ---- device helpers ----
+#ifdef __CUDACC__
+__device__ __forceinline__ void latch_error(DevStatus* st, unsigned int epoch, unsigned int code) {
+    atomicCAS(&st->sticky, 0u, code);
+    atomicExch(&st->call_err_epoch, epoch);
+}
+__device__ __forceinline__ bool call_failed(const DevStatus* st, unsigned int epoch) {
+    return *((const volatile unsigned int*)&st->call_err_epoch) == epoch;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ uint64_t phys_row(uint2 e, uint64_t S) { return (uint64_t)e.x * S + e.y; }
+
+// Exclusive scan of one value per thread over a block of 256 threads.
+// `smem` must hold 8 uint32.  Returns the exclusive prefix; *total = block sum.
+__device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_t* smem, uint32_t* total) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) smem[w] = incl;
+    __syncthreads();
+    uint32_t wbase = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t t = smem[i];
+        if (i < w) wbase += t;
+        tot += t;
+    }
+    __syncthreads();
+    *total = tot;
+    return wbase + incl - v;
+}
+#endif
+
+}  // namespace psb

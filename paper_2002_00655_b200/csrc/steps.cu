@@ -1,0 +1,436 @@
+// Fused pull -> per-example gradient kernels of the three training tasks of
+// Section 4.1 / Appendix A of the paper.  One warp handles one example (a
+// matrix cell, a knowledge-graph data point with its negatives, a skip-gram
+// center word with its window): it looks the example's keys up in the location
+// table, gathers their rows with coalesced loads, forms dot products with warp
+// shuffles, and writes one additive update row per key occurrence plus that
+// occurrence's key.  The push stage (pull_push.cu) then sorts the occurrences
+// by key, sums them per key and applies them, so every read in here sees the
+// state from before the step.
+#include "ps_internal.cuh"
+
+namespace psb {
+
+__device__ __forceinline__ float softplusf(float z) { return fmaxf(z, 0.f) + log1pf(expf(-fabsf(z))); }
+__device__ __forceinline__ float sigmoidf(float z) {
+    if (z >= 0.f) return 1.f / (1.f + expf(-z));
+    const float e = expf(z);
+    return e / (1.f + e);
+}
+__device__ __forceinline__ double softplus_d(double z) { return fmax(z, 0.0) + log1p(exp(-fabs(z))); }
+__device__ __forceinline__ double sigmoid_d(double z) {
+    if (z >= 0.0) return 1.0 / (1.0 + exp(-z));
+    const double e = exp(z);
+    return e / (1.0 + e);
+}
+
+// Sum of the warps' loss terms -> loss_partial[blockIdx.x]; fixed order.
+__device__ __forceinline__ void block_loss_out(double loss, double* __restrict__ loss_partial) {
+    __shared__ double wl[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) wl[w] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += wl[i];
+        loss_partial[blockIdx.x] = t;
+    }
+}
+
+static uint32_t step_grid(ps_store* ps, uint64_t n_examples) {
+    uint64_t g = (n_examples + 7) / 8;
+    const uint64_t cap = (uint64_t)ps->sm_count * 8;
+    if (g > cap) g = cap;
+    if (g > kMaxLossBlocks) g = kMaxLossBlocks;
+    return g ? (uint32_t)g : 1u;
+}
+
+// ------------------------------------------------------------------ MF ----
+// kCh = number of float4 a lane holds per row (row_len <= 128 * kCh); 0 = any
+// row length, rows re-read from cache for the second pass.
+template <int kCh>
+__global__ void __launch_bounds__(256)
+mf_step_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, const float* __restrict__ cv,
+               uint64_t n, uint64_t col_base, float lr, float lam, const float4* __restrict__ store,
+               const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t L4,
+               uint32_t* __restrict__ keys_out, float4* __restrict__ upd, double* __restrict__ loss_partial,
+               DevStatus* st, unsigned int epoch) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    constexpr int kRegs = kCh > 0 ? kCh : 1;
+    double loss = 0;
+    for (uint64_t t = warp; t < n; t += n_warps) {
+        const uint32_t i = ci[t], j = cj[t];
+        const float v = cv[t];
+        const uint64_t kw = i, kh = col_base + j;
+        if (kw >= col_base || kh >= K) {
+            if (lane == 0) {
+                latch_error(st, epoch, PS_ERR_KEY_RANGE);
+                keys_out[2 * t] = (uint32_t)K;
+                keys_out[2 * t + 1] = (uint32_t)K;
+            }
+            continue;
+        }
+        const float4* W = store + phys_row(table[kw], S) * L4;
+        const float4* H = store + phys_row(table[kh], S) * L4;
+        float4 w[kRegs], h[kRegs];
+        float dot = 0.f, nw = 0.f, nh = 0.f;
+        if constexpr (kCh > 0) {
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                const uint32_t f = lane + 32 * c;
+                w[c] = f < L4 ? W[f] : make_float4(0.f, 0.f, 0.f, 0.f);
+                h[c] = f < L4 ? H[f] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                dot += w[c].x * h[c].x + w[c].y * h[c].y + w[c].z * h[c].z + w[c].w * h[c].w;
+                nw += w[c].x * w[c].x + w[c].y * w[c].y + w[c].z * w[c].z + w[c].w * w[c].w;
+                nh += h[c].x * h[c].x + h[c].y * h[c].y + h[c].z * h[c].z + h[c].w * h[c].w;
+            }
+        } else {
+            for (uint32_t f = lane; f < L4; f += 32) {
+                const float4 a = W[f], b = H[f];
+                dot += a.x * b.x + a.y * b.y + a.z * b.z + a.w * b.w;
+                nw += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+                nh += b.x * b.x + b.y * b.y + b.z * b.z + b.w * b.w;
+            }
+        }
+        dot = warp_sum(dot);
+        nw = warp_sum(nw);
+        nh = warp_sum(nh);
+        const float e = v - dot;
+        loss += (double)(0.5f * e * e + 0.5f * lam * (nw + nh));
+        float4* UW = upd + (2 * t) * L4;
+        float4* UH = upd + (2 * t + 1) * L4;
+        auto emit = [&](uint32_t f, const float4& a, const float4& b) {
+            float4 dw, dh;
+            dw.x = lr * (e * b.x - lam * a.x); dw.y = lr * (e * b.y - lam * a.y);
+            dw.z = lr * (e * b.z - lam * a.z); dw.w = lr * (e * b.w - lam * a.w);
+            dh.x = lr * (e * a.x - lam * b.x); dh.y = lr * (e * a.y - lam * b.y);
+            dh.z = lr * (e * a.z - lam * b.z); dh.w = lr * (e * a.w - lam * b.w);
+            UW[f] = dw;
+            UH[f] = dh;
+        };
+        if constexpr (kCh > 0) {
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                const uint32_t f = lane + 32 * c;
+                if (f < L4) emit(f, w[c], h[c]);
+            }
+        } else {
+            for (uint32_t f = lane; f < L4; f += 32) emit(f, W[f], H[f]);
+        }
+        if (lane == 0) {
+            keys_out[2 * t] = (uint32_t)kw;
+            keys_out[2 * t + 1] = (uint32_t)kh;
+        }
+    }
+    block_loss_out(loss, loss_partial);
+}
+
+uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
+                        uint64_t col_key_base, float lr, float lambda, cudaStream_t s) {
+    const uint32_t L4 = ps->cfg.row_len / 4;
+    const uint32_t grid = step_grid(ps, n);
+#define MF_ARGS d_i, d_j, d_v, n, col_key_base, lr, lambda, (const float4*)ps->store, ps->table,                 \
+                ps->cfg.slots_per_part, ps->cfg.num_keys, L4, ps->keysA, (float4*)ps->upd, ps->loss_partial,   \
+                ps->status, ps->epoch
+    if (L4 <= 32) PS_LAUNCH(ps, mf_step_kernel<1>, grid, 256, s, MF_ARGS);
+    else if (L4 <= 64) PS_LAUNCH(ps, mf_step_kernel<2>, grid, 256, s, MF_ARGS);
+    else if (L4 <= 128) PS_LAUNCH(ps, mf_step_kernel<4>, grid, 256, s, MF_ARGS);
+    else PS_LAUNCH(ps, mf_step_kernel<0>, grid, 256, s, MF_ARGS);
+#undef MF_ARGS
+    return grid;
+}
+
+// ------------------------------------------------------------- ComplEx ----
+// Slots of a data point: 0 = subject, 1 = relation, 2 = object, 3 + q = the
+// q-th negative entity.  Lane u holds slot u's key and row offset.  Slots that
+// repeat an earlier slot's key emit no update (key mark K): their gradient is
+// folded into the first slot with that key, so that AdaGrad sees the gradient
+// of the data point's loss with respect to each DISTINCT key.
+//
+// Scores and gradient sums are formed in fp64 from the fp32 rows.  With a zero
+// accumulator AdaGrad's step is -lr * g / (|g| + eps), which near g = 0 turns
+// rounding noise of g into a visible change of the parameter; fp64 sums keep
+// that noise far below the fp32 resolution of the result.  The final AdaGrad
+// expression is evaluated in fp32 on the rounded gradient.
+__global__ void __launch_bounds__(256)
+kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
+                const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
+                uint32_t n_neg, uint64_t rel_base, uint32_t d, float lr, float eps, const float* __restrict__ store,
+                const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t* __restrict__ keys_out,
+                float* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const int n_slots = 3 + (int)n_neg;
+    const uint32_t L = 4 * d;
+    const unsigned full = 0xffffffffu;
+    double loss = 0;
+    for (uint64_t t = warp; t < n; t += n_warps) {
+        // ---- keys, validity, row offsets, first-slot-with-same-key ----
+        uint64_t key = K;
+        int side = 0;
+        bool bad = false;
+        if (lane < n_slots) {
+            if (lane == 1) {
+                key = rel_base + tr[t];
+                bad = key >= K;
+            } else {
+                const uint32_t e = lane == 0 ? ts[t] : (lane == 2 ? to[t] : neg_ent[t * n_neg + (lane - 3)]);
+                key = e;
+                bad = e >= rel_base;
+                if (lane >= 3) side = neg_side[t * n_neg + (lane - 3)] != 0;
+            }
+        }
+        uint32_t* kout = keys_out + t * n_slots;
+        if (__any_sync(full, bad)) {
+            if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+            if (lane < n_slots) kout[lane] = (uint32_t)K;
+            continue;
+        }
+        uint64_t off = 0;
+        if (lane < n_slots) off = phys_row(table[key], S) * L;
+        int rep = lane;
+        for (int z = n_slots - 1; z >= 0; --z) {
+            const uint64_t kz = __shfl_sync(full, key, z);
+            if (z < lane && kz == key) rep = z;
+        }
+        const float* Srow = store + __shfl_sync(full, off, 0);
+        const float* Rrow = store + __shfl_sync(full, off, 1);
+        const float* Orow = store + __shfl_sync(full, off, 2);
+
+        // ---- pass A: the 1 + n_neg scores; lane q keeps triple q's score ----
+        double phi_mine = 0;
+        for (int q = 0; q <= (int)n_neg; ++q) {
+            const float* Sq = Srow;
+            const float* Oq = Orow;
+            if (q > 0) {
+                const int sd = __shfl_sync(full, side, 2 + q);
+                const float* Nq = store + __shfl_sync(full, off, 2 + q);
+                if (sd == 0) Sq = Nq; else Oq = Nq;
+            }
+            double part = 0;
+            for (uint32_t c = lane; c < d; c += 32) {
+                const double a = Sq[c], b = Sq[d + c], cr = Rrow[c], ci = Rrow[d + c], e = Oq[c], f = Oq[d + c];
+                part += cr * (a * e + b * f) + ci * (a * f - b * e);
+            }
+            const double phi = warp_sum_d(part);
+            if (lane == q) phi_mine = phi;
+        }
+        // lane q: loss term and d loss / d phi of triple q (label +1 for the positive, -1 for negatives)
+        double coef = 0, loss_q = 0;
+        if (lane <= (int)n_neg) {
+            const double y = lane == 0 ? 1.0 : -1.0;
+            loss_q = softplus_d(-y * phi_mine);
+            coef = -y * sigmoid_d(-y * phi_mine);
+        }
+        loss += warp_sum_d(loss_q);
+
+        // ---- weights with which each entity slot receives the two "negative role" directions ----
+        // A negative with side 0 stands in the subject's place: its gradient is coef * dphi/dS(r, o).
+        // With side 1 it stands in the object's place: coef * dphi/dO(s, r).  Summed over the
+        // negatives whose key's first slot is this lane.
+        double wS = 0, wO = 0;
+        for (int q = 1; q <= (int)n_neg; ++q) {
+            const int rq = __shfl_sync(full, rep, 2 + q);
+            const int sd = __shfl_sync(full, side, 2 + q);
+            const double cf = __shfl_sync(full, coef, q);
+            if (rq == lane) {
+                if (sd == 0) wS += cf; else wO += cf;
+            }
+        }
+        const double cf0 = __shfl_sync(full, coef, 0);
+        const int rep_o = __shfl_sync(full, rep, 2);            // 0 if object == subject
+        const double wS0 = __shfl_sync(full, wS, 0), wO0 = __shfl_sync(full, wO, 0);
+        const double wS2 = __shfl_sync(full, wS, 2), wO2 = __shfl_sync(full, wO, 2);
+
+        // ---- pass B: gradients per block of 32 complex dimensions, AdaGrad, update rows ----
+        float* U = upd + (t * n_slots) * L;
+        for (uint32_t c0 = 0; c0 < d; c0 += 32) {
+            const uint32_t c = c0 + lane;
+            const bool act = c < d;
+            double a = 0, b = 0, cr = 0, ci = 0, e = 0, f = 0;
+            if (act) {
+                a = Srow[c]; b = Srow[d + c]; cr = Rrow[c]; ci = Rrow[d + c]; e = Orow[c]; f = Orow[d + c];
+            }
+            // directions that do not depend on the negative
+            const double dS_re = cr * e + ci * f, dS_im = cr * f - ci * e;      // d phi / d subject, object = o
+            const double dO_re = cr * a - ci * b, dO_im = cr * b + ci * a;      // d phi / d object, subject = s
+            double gs_re = cf0 * dS_re, gs_im = cf0 * dS_im;
+            double go_re = cf0 * dO_re, go_im = cf0 * dO_im;
+            double gr_re = cf0 * (a * e + b * f), gr_im = cf0 * (a * f - b * e);
+            for (int q = 1; q <= (int)n_neg; ++q) {
+                const double cf = __shfl_sync(full, coef, q);
+                const int sd = __shfl_sync(full, side, 2 + q);
+                const float* Nq = store + __shfl_sync(full, off, 2 + q);
+                double na = 0, nb = 0;
+                if (act) { na = Nq[c]; nb = Nq[d + c]; }
+                if (sd == 0) {          // triple (n, r, o)
+                    gr_re += cf * (na * e + nb * f); gr_im += cf * (na * f - nb * e);
+                    go_re += cf * (cr * na - ci * nb); go_im += cf * (cr * nb + ci * na);
+                } else {                // triple (s, r, n)
+                    gr_re += cf * (a * na + b * nb); gr_im += cf * (a * nb - b * na);
+                    gs_re += cf * (cr * na + ci * nb); gs_im += cf * (cr * nb - ci * na);
+                }
+            }
+            // negatives that coincide with the subject or the object
+            gs_re += wS0 * dS_re + wO0 * dO_re; gs_im += wS0 * dS_im + wO0 * dO_im;
+            go_re += wS2 * dS_re + wO2 * dO_re; go_im += wS2 * dS_im + wO2 * dO_im;
+            if (rep_o == 0) { gs_re += go_re; gs_im += go_im; }
+            for (int u = 0; u < n_slots; ++u) {
+                const int ru = __shfl_sync(full, rep, u);
+                const double wSu = __shfl_sync(full, wS, u), wOu = __shfl_sync(full, wO, u);
+                const uint64_t offu = __shfl_sync(full, off, u);
+                if (ru != u || !act) continue;
+                double gd_re, gd_im;
+                if (u == 0) { gd_re = gs_re; gd_im = gs_im; }
+                else if (u == 1) { gd_re = gr_re; gd_im = gr_im; }
+                else if (u == 2) { gd_re = go_re; gd_im = go_im; }
+                else { gd_re = wSu * dS_re + wOu * dO_re; gd_im = wSu * dS_im + wOu * dO_im; }
+                const float g_re = (float)gd_re, g_im = (float)gd_im;
+                const float G_re = store[offu + 2 * d + c], G_im = store[offu + 3 * d + c];
+                const float g2_re = g_re * g_re, g2_im = g_im * g_im;
+                float* Uu = U + (uint64_t)u * L;
+                Uu[c] = -lr * g_re / (sqrtf(G_re + g2_re) + eps);
+                Uu[d + c] = -lr * g_im / (sqrtf(G_im + g2_im) + eps);
+                Uu[2 * d + c] = g2_re;
+                Uu[3 * d + c] = g2_im;
+            }
+        }
+        if (lane < n_slots) kout[lane] = rep == lane ? (uint32_t)key : (uint32_t)K;
+    }
+    block_loss_out(loss, loss_partial);
+}
+
+uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                         const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
+                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s) {
+    const uint32_t grid = step_grid(ps, n);
+    PS_LAUNCH(ps, kge_step_kernel, grid, 256, s, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim,
+              lr, eps, (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->keysA,
+              ps->upd, ps->loss_partial, ps->status, ps->epoch);
+    return grid;
+}
+
+// ---------------------------------------------------------------- SGNS ----
+// number of (center, context) pairs of all centers before position p
+__device__ __forceinline__ uint64_t sgns_pairs_before(uint64_t p, uint64_t T, uint64_t W) {
+    // left contexts: sum over q < p of min(q, W)
+    const uint64_t m = p < W ? p : W;
+    const uint64_t left = m * (m - (m > 0)) / 2 + (p - m) * W;
+    // right contexts: sum over q < p of min(T - 1 - q, W)
+    const uint64_t full = T > W ? (p < T - W ? p : T - W) : 0;
+    const uint64_t rest = p - full;
+    const uint64_t first = T - 1 - full;                    // value at q = full (only used if rest > 0)
+    const uint64_t right = full * W + (rest ? rest * first - rest * (rest - 1) / 2 : 0);
+    return left + right;
+}
+
+// Occurrence slots of center number c of the batch: slot_base = c * (1 + 2W(1 + n_neg));
+// slot_base = the center's input vector; then per context j (ascending position) 1 + n_neg output vectors.
+template <int kCh>
+__global__ void __launch_bounds__(256)
+sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64_t first_pos, uint64_t n_centers,
+                 uint64_t T, uint32_t window, const uint32_t* __restrict__ negs, uint32_t n_neg, uint64_t out_base,
+                 float lr, const float4* __restrict__ store, const uint2* __restrict__ table, uint64_t S, uint64_t K,
+                 uint32_t L4, uint32_t* __restrict__ keys_out, float4* __restrict__ upd,
+                 double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t per_ctx = 1 + n_neg;
+    const uint64_t slots = 1 + (uint64_t)2 * window * per_ctx;
+    const uint64_t pairs0 = sgns_pairs_before(first_pos, T, window);
+    double loss = 0;
+    for (uint64_t cidx = warp; cidx < n_centers; cidx += n_warps) {
+        const uint64_t p = first_pos + cidx;
+        const uint64_t lo = p >= window ? p - window : 0;
+        const uint64_t hi = p + window < T ? p + window : T - 1;
+        const uint64_t z0 = sgns_pairs_before(p, T, window) - pairs0;
+        uint32_t* kout = keys_out + cidx * slots;
+        float4* U = upd + cidx * slots * L4;
+        const uint32_t wtok = tokens[p - tok_first];
+        // mark every slot unused first; used ones are overwritten below
+        for (uint64_t x = lane; x < slots; x += 32) kout[x] = (uint32_t)K;
+        __syncwarp();
+        if (wtok >= out_base) {
+            if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+            continue;
+        }
+        const float4* V = store + phys_row(table[wtok], S) * L4;
+        float4 v[kCh], dv[kCh];
+#pragma unroll
+        for (int c = 0; c < kCh; ++c) {
+            const uint32_t f = lane + 32 * c;
+            v[c] = f < L4 ? V[f] : make_float4(0.f, 0.f, 0.f, 0.f);
+            dv[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float loss_c = 0.f;
+        bool bad = false;
+        uint32_t j = 0;
+        for (uint64_t q = lo; q <= hi; ++q) {
+            if (q == p) continue;
+            const uint64_t z = z0 + j;
+            for (uint32_t i = 0; i <= n_neg; ++i) {
+                const uint32_t word = i == 0 ? tokens[q - tok_first] : negs[z * n_neg + (i - 1)];
+                const uint64_t ku = out_base + word;
+                const uint64_t slot = 1 + (uint64_t)j * per_ctx + i;
+                if (ku >= K) { bad = true; continue; }
+                const float4* Urow = store + phys_row(table[ku], S) * L4;
+                float4 u[kCh];
+                float x = 0.f;
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    const uint32_t f = lane + 32 * c;
+                    u[c] = f < L4 ? Urow[f] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    x += v[c].x * u[c].x + v[c].y * u[c].y + v[c].z * u[c].z + v[c].w * u[c].w;
+                }
+                x = warp_sum(x);
+                const float y = i == 0 ? 1.f : 0.f;
+                const float g = sigmoidf(x) - y;
+                loss_c += i == 0 ? softplusf(-x) : softplusf(x);
+                const float sc = -lr * g;
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    const uint32_t f = lane + 32 * c;
+                    dv[c].x += sc * u[c].x; dv[c].y += sc * u[c].y; dv[c].z += sc * u[c].z; dv[c].w += sc * u[c].w;
+                    if (f < L4)
+                        U[slot * L4 + f] = make_float4(sc * v[c].x, sc * v[c].y, sc * v[c].z, sc * v[c].w);
+                }
+                if (lane == 0) kout[slot] = (uint32_t)ku;
+            }
+            ++j;
+        }
+        if (bad && lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+#pragma unroll
+        for (int c = 0; c < kCh; ++c) {
+            const uint32_t f = lane + 32 * c;
+            if (f < L4) U[f] = dv[c];
+        }
+        if (lane == 0) kout[0] = wtok;
+        loss += (double)loss_c;
+    }
+    block_loss_out(loss, loss_partial);
+}
+
+uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
+                          uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
+                          uint32_t n_neg, uint64_t out_key_base, float lr, cudaStream_t s) {
+    const uint32_t L4 = ps->cfg.row_len / 4;
+    const uint32_t grid = step_grid(ps, n_centers);
+#define SG_ARGS d_tokens, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, lr,   \
+                (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4, ps->keysA,   \
+                (float4*)ps->upd, ps->loss_partial, ps->status, ps->epoch
+    if (L4 <= 32) PS_LAUNCH(ps, sgns_step_kernel<1>, grid, 256, s, SG_ARGS);
+    else if (L4 <= 64) PS_LAUNCH(ps, sgns_step_kernel<2>, grid, 256, s, SG_ARGS);
+    else if (L4 <= 96) PS_LAUNCH(ps, sgns_step_kernel<3>, grid, 256, s, SG_ARGS);
+    else PS_LAUNCH(ps, sgns_step_kernel<4>, grid, 256, s, SG_ARGS);
+#undef SG_ARGS
+    return grid;
+}
+
+}  // namespace psb
