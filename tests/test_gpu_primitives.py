@@ -1,0 +1,158 @@
+"""GPU parity: pull, push, localize through the C-ABI against the CPU oracle (Table 2, Sections 3.1-3.2)."""
+import numpy as np
+import pytest
+import torch
+
+from tests.util import assert_close, compare_state, dev, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def f_row(keys, L):
+    keys = np.asarray(keys, dtype=np.int64)
+    return ((keys[:, None] * 31 + np.arange(L)[None, :] * 7) % 1021).astype(np.float32)
+
+
+@pytest.mark.parametrize("K,L,N,n", [(5000, 100, 1, 4099), (3001, 128, 7, 10007), (640, 8, 3, 33), (900, 300, 2, 1),
+                                      (2000, 400, 5, 2500), (700, 516, 1, 777)])
+def test_pull_is_bit_exact(K, L, N, n):
+    g, o = make_pair(K, L, N, rows=f_row(np.arange(K), L))
+    keys = np.random.default_rng(n).integers(0, K, size=n)
+    keys[: min(n, 5)] = K - 1                                   # duplicates and the last key
+    got = g.pull(dev(keys)).cpu().numpy()
+    g.sync()
+    assert (got == o.pull(keys)).all()
+    assert (got == f_row(keys, L)).all()                        # recomputable without any store
+    assert g.pull(dev(np.zeros(0, np.int64))).shape == (0, L)
+
+
+@pytest.mark.parametrize("L", [4, 100, 128, 300])
+def test_push_integer_updates_are_exact_and_order_free(L):
+    K, n = 3000, 20011
+    g, o = make_pair(K, L, 4, rows=f_row(np.arange(K), L), max_batch_keys=n)
+    rng = np.random.default_rng(L)
+    keys = rng.integers(0, K, size=n)
+    keys[rng.random(n) < 0.3] = 17                              # one segment spanning hundreds of tiles
+    keys[rng.random(n) < 0.05] = 2999
+    upd = rng.integers(-4, 5, size=(n, L)).astype(np.float32)
+    g.push(dev(keys), dev(upd))
+    g.sync()
+    o.push(keys, upd)
+    compare_state(g, o, exact_rows=True, what="push")
+    perm = rng.permutation(n)                                   # same multiset, another order: same sums
+    g.push(dev(keys[perm]), dev(upd[perm]))
+    g.sync()
+    o.push(keys, upd)
+    compare_state(g, o, exact_rows=True, what="push permuted")
+
+
+@pytest.mark.parametrize("K,L,n,hot", [(4000, 100, 9001, 0.2), (1000, 128, 65, 0.0), (50000, 128, 60000, 0.1),
+                                         (300, 400, 4000, 0.5), (64, 8, 31, 0.9), (64, 8, 32, 1.0)])
+def test_push_matches_oracle(K, L, n, hot):
+    g, o = make_pair(K, L, 3, max_batch_keys=n)
+    rng = np.random.default_rng(n)
+    keys = rng.integers(0, K, size=n)
+    keys[rng.random(n) < hot] = K // 2
+    upd = rng.normal(size=(n, L)).astype(np.float32)
+    for _ in range(2):
+        g.push(dev(keys), dev(upd))
+        o.push(keys, upd)
+    g.sync()
+    compare_state(g, o, what="push")
+
+
+def test_push_and_pull_reject_bad_keys_without_touching_the_store():
+    import paper_2002_00655_b200 as ps
+    K, L = 500, 12
+    g, o = make_pair(K, L, 2)
+    keys = np.array([1, 2, K, 3])
+    g.push(dev(keys), dev(np.ones((4, L), np.float32)))
+    assert g.sync(check=False) == ps.PS_ERR_KEY_RANGE
+    assert g.sync(check=False) == ps.PS_OK                      # reading the error clears it
+    compare_state(g, o, exact_rows=True, what="rejected push")
+    out = g.pull(dev(keys)).cpu().numpy()
+    assert g.sync(check=False) == ps.PS_ERR_KEY_RANGE
+    assert (out[2] == 0).all() and (out[[0, 1, 3]] == o.pull([1, 2, 3])).all()
+    with pytest.raises(ps.PSError) as e:                        # more occurrences than the workspace was sized for
+        g.push(dev(np.zeros(g.max_batch_keys + 1, np.int64)), dev(np.zeros((g.max_batch_keys + 1, L), np.float32)))
+    assert e.value.code == ps.PS_ERR_WORKSPACE
+    with pytest.raises(ps.PSError) as e:
+        g.localize(2, dev(keys[:2]))
+    assert e.value.code == ps.PS_ERR_WORKER_RANGE
+
+
+@pytest.mark.parametrize("K,L,N,slack,n,seed", [(5000, 16, 4, 1.5, 700, 0), (20000, 128, 8, 1.25, 6000, 1),
+                                                 (1000, 4, 64, 2.0, 300, 2), (3000, 100, 3, 1.3, 2048, 3)])
+def test_localize_sequences_are_bit_exact(K, L, N, slack, n, seed):
+    S = int(np.ceil(slack * -(-K // N)))
+    g, o = make_pair(K, L, N, S, max_batch_keys=n)
+    rng = np.random.default_rng(seed)
+    from oracle.ps_oracle import OracleError
+    import paper_2002_00655_b200 as ps
+    moved = 0
+    for it in range(14):
+        w = int(rng.integers(0, N))
+        m = int(rng.integers(1, n + 1))
+        keys = (rng.zipf(1.3, size=m) - 1) % K if it % 2 else rng.integers(0, K, size=m)
+        before = o.owner.copy()
+        g.localize(w, dev(keys))
+        code = g.sync(check=False)
+        try:
+            o.localize(w, keys)
+            assert code == ps.PS_OK
+            moved += int((before != o.owner).sum())
+        except OracleError as e:
+            assert e.code == 4 and code == ps.PS_ERR_CAPACITY
+        compare_state(g, o, exact_rows=True, what=f"localize call {it}")
+        if it == 5:                                             # an identical second call changes nothing
+            g.localize(w, dev(keys))
+            assert g.sync(check=False) == code
+            compare_state(g, o, exact_rows=True, what="repeated localize")
+        upd = rng.integers(-2, 3, size=(m, L)).astype(np.float32)
+        g.push(dev(keys), dev(upd))                             # push through the new locations
+        o.push(keys, upd)
+    g.sync()
+    compare_state(g, o, exact_rows=True, what="after pushes")
+    assert ps.ps_rows_moved(g.h) == moved
+    owner, slot = o.get_location(np.arange(K))
+    d_owner = torch.empty(K, dtype=torch.int32, device="cuda")
+    d_slot = torch.empty(K, dtype=torch.int32, device="cuda")
+    ps.ps_get_location(g.h, dev(np.arange(K)), d_owner, d_slot)
+    g.sync()
+    assert (d_owner.cpu().numpy().view(np.uint32) == owner).all() and (d_slot.cpu().numpy().view(np.uint32) == slot).all()
+
+
+def test_localize_capacity_failure_and_bad_key_leave_everything_unchanged():
+    import paper_2002_00655_b200 as ps
+    K, L, N = 64, 4, 4
+    g, o = make_pair(K, L, N, 18)                               # 16 keys per partition, 2 spare slots
+    g.localize(0, dev(np.array([20, 21, 22, 40])))
+    assert g.sync(check=False) == ps.PS_ERR_CAPACITY
+    compare_state(g, o, exact_rows=True, what="over capacity")
+    g.localize(0, dev(np.array([20, 20, 40, 40, 5])))           # duplicates collapse, key 5 is already local: fits
+    g.sync()
+    o.localize(0, [20, 20, 40, 40, 5])
+    compare_state(g, o, exact_rows=True, what="at capacity")
+    g.localize(1, dev(np.array([3, K + 7])))
+    assert g.sync(check=False) == ps.PS_ERR_KEY_RANGE
+    compare_state(g, o, exact_rows=True, what="bad key")
+
+
+def test_stress_twin_pull_push_localize_loop():
+    """The pull / push / localize stress loop on a scaled-down twin, every batch checked against the oracle."""
+    from synth import workloads as W
+    cfg = W.STRESS_TINY
+    rows = W.stress_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    g, o = make_pair(cfg.num_keys, cfg.row_len, cfg.workers, cfg.slots_per_part, rows=rows, max_batch_keys=cfg.batch)
+    for b in range(cfg.n_batches):
+        keys = W.stress_keys(cfg, b, "cpu")
+        upd = W.stress_updates(cfg, b, "cpu")
+        got = g.pull(keys.cuda())
+        g.sync()
+        assert (got.cpu().numpy() == g.export(table=False)[0].numpy()[keys.numpy()]).all()   # pulled = stored, bit for bit
+        g.push(keys.cuda(), upd.cuda())
+        o.push(keys, upd)
+        g.localize(cfg.requester(b), keys[:cfg.localize_count].cuda())
+        o.localize(cfg.requester(b), keys[:cfg.localize_count])
+        g.sync()
+        compare_state(g, o, what=f"stress batch {b}")

@@ -1,0 +1,207 @@
+"""GPU parity: the three fused training steps through the C-ABI against the CPU oracle.
+
+Two modes: single-step (the oracle's pre-step state is loaded into the GPU store,
+one step runs on both, every row is compared) and free-running (both sides train
+side by side; rows, tables and the epoch loss are compared at the end).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2002_00655_b200 as ps
+from synth import workloads as W
+from tests.util import assert_close, close, compare_state, dev, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def loss_of(g):
+    return float(g.loss.cpu()[0])
+
+
+# ------------------------------------------------------------------ MF ----
+def mf_data(cfg):
+    planted = W.mf_planted(cfg, "cpu")
+    return W.mf_cells(cfg, planted, 0, cfg.n_cells, "cpu")
+
+
+def test_mf_tiny_epoch_free_running_and_localize_transparency():
+    cfg = W.MF_TINY
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    g, o = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
+    g2, _ = make_pair(cfg.num_keys, cfg.rank, 8, cfg.num_keys, rows=rows,
+                      max_batch_keys=2 * cfg.batch)           # same run with relocations in between
+    di, dj, dv = i.cuda(), j.cuda(), v.cuda()
+    rng = np.random.default_rng(0)
+    for b in range(cfg.n_batches):
+        s, c = cfg.batch_range(b)
+        ps.ps_step_mf(g.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+        ps.ps_step_mf(g2.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g2.loss)
+        g2.localize(int(rng.integers(0, 8)), dev(rng.integers(0, cfg.num_keys, size=150)))
+        o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+    g.sync()
+    g2.sync()
+    compare_state(g, o, what="mf_tiny epoch")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    r1, r2 = g.export(table=False)[0], g2.export(table=False)[0]
+    assert (r1 == r2).all(), "relocations changed the parameters (location transparency, Section 2.3)"
+    assert loss_of(g) == loss_of(g2)
+    assert ps.ps_rows_moved(g2.h) > 1000
+
+
+@pytest.mark.parametrize("R,Cc,L,n,zipf", [(3000, 500, 100, 5000, 1.1), (400, 300, 8, 1024, None), (1000, 50, 128, 2047, 1.1),
+                                           (200, 200, 260, 999, None), (90, 70, 640, 300, 1.1)])
+def test_mf_single_steps(R, Cc, L, n, zipf):
+    cfg = W.MFConfig("t", R, Cc, L, 4 * n, n, 0.002, 0.05, 0.1, 0.5, zipf)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    g, o = make_pair(cfg.num_keys, L, rows=rows, max_batch_keys=2 * n)
+    for b in range(cfg.n_batches):
+        s, c = cfg.batch_range(b)
+        if b == cfg.n_batches - 1:
+            c = c - 37                                           # ragged last batch
+        g.set_all_rows(torch.from_numpy(o.rows.copy()))         # oracle's pre-step state
+        g.loss.zero_(); o.loss[0] = 0
+        ps.ps_step_mf(g.h, i[s:s + c].cuda(), j[s:s + c].cuda(), v[s:s + c].cuda(), cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+        o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+        g.sync()
+        compare_state(g, o, what=f"mf step {b}")
+        assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
+def test_mf_bad_index_makes_the_step_a_no_op():
+    g, o = make_pair(100, 8)
+    i = dev(np.array([1, 2, 60, 3]), torch.int32)               # 60 >= col_key_base
+    j = dev(np.array([1, 2, 3, 4]), torch.int32)
+    ps.ps_step_mf(g.h, i, j, dev(np.ones(4, np.float32)), 50, 0.1, 0.0, g.loss)
+    assert g.sync(check=False) == ps.PS_ERR_KEY_RANGE
+    compare_state(g, o, exact_rows=True, what="bad mf step")
+    assert loss_of(g) == 0.0
+
+
+# ------------------------------------------------------------- ComplEx ----
+def kge_run(cfg, steps, single_step, first=0):
+    rows = W.kge_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    g, o = make_pair(cfg.num_keys, cfg.row_len, rows=rows, max_batch_keys=(3 + cfg.n_neg) * cfg.batch)
+    for b in range(first, first + steps):
+        s0, c = cfg.batch_range(b)
+        s, r, t, neg, side = W.kge_triples(cfg, s0, c, "cpu")
+        if single_step:
+            g.set_all_rows(torch.from_numpy(o.rows.copy()))
+            g.loss.zero_(); o.loss[0] = 0
+        ps.ps_step_kge(g.h, s.cuda(), r.cuda(), t.cuda(), neg.cuda(), side.cuda(), cfg.n_neg, cfg.rel_key_base,
+                       cfg.dim, cfg.lr, cfg.eps, g.loss)
+        o.step_kge(s, r, t, neg, side, cfg.rel_key_base, cfg.dim, cfg.lr, cfg.eps)
+        g.sync()
+        if single_step:
+            compare_state(g, o, what=f"kge step {b}")
+            assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    return g, o
+
+
+def test_kge_tiny_epoch_single_steps():
+    cfg = W.KGE_TINY                                            # 2,000 Zipf entities: s = o and negative = s/o do occur
+    s, r, t, neg, side = W.kge_triples(cfg, 0, cfg.n_triples, "cpu")
+    assert (s == t).any() and ((neg == s[:, None]) | (neg == t[:, None])).any()
+    kge_run(cfg, cfg.n_batches, single_step=True)
+
+
+def test_kge_free_running():
+    cfg = W.KGE_TINY
+    g, o = kge_run(cfg, 8, single_step=False)
+    compare_state(g, o, what="kge free-running")
+    assert close(loss_of(g), o.loss[0])
+
+
+@pytest.mark.parametrize("dim,n_neg,batch,ents", [(100, 10, 700, 5000), (32, 1, 333, 40), (36, 29, 64, 9), (4, 0, 100, 30)])
+def test_kge_shapes_and_heavy_key_collisions(dim, n_neg, batch, ents):
+    cfg = W.scaled(W.KGE_TINY, entities=ents, relations=5, dim=dim, n_neg=n_neg, batch=batch, n_triples=3 * batch - 11)
+    kge_run(cfg, cfg.n_batches, single_step=True)
+
+
+# ---------------------------------------------------------------- SGNS ----
+def sgns_run(cfg, batches, single_step, random_init):
+    if random_init:
+        rows = torch.from_numpy(np.random.default_rng(3).normal(0, 0.3, size=(cfg.num_keys, cfg.dim)).astype(np.float32))
+    else:
+        rows = W.sgns_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    tokens = W.sgns_tokens(cfg, 0, cfg.n_tokens, "cpu")
+    occ = cfg.batch * (1 + 2 * cfg.window * (1 + cfg.n_neg))
+    g, o = make_pair(cfg.num_keys, cfg.dim, rows=rows, max_batch_keys=occ)
+    d_tok = tokens.cuda()
+    for b in batches:
+        first, n = cfg.batch_range(b)
+        negs = W.sgns_negatives(cfg, first, n, "cpu")
+        if single_step:
+            g.set_all_rows(torch.from_numpy(o.rows.copy()))
+            g.loss.zero_(); o.loss[0] = 0
+        ps.ps_step_sgns(g.h, d_tok, first, n, cfg.window, negs.cuda(), cfg.n_neg, cfg.out_key_base, cfg.lr, g.loss)
+        o.step_sgns(tokens, first, n, cfg.window, negs, cfg.n_neg, cfg.out_key_base, cfg.lr)
+        g.sync()
+        if single_step:
+            compare_state(g, o, what=f"sgns step {b}")
+            assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    return g, o
+
+
+def test_sgns_tiny_single_steps_cover_both_stream_ends():
+    cfg = W.SGNS_TINY
+    sgns_run(cfg, [0, 1, 17, cfg.n_batches - 1], single_step=True, random_init=True)
+
+
+def test_sgns_tiny_free_running_from_the_standard_init():
+    cfg = W.SGNS_TINY
+    g, o = sgns_run(cfg, range(10), single_step=False, random_init=False)
+    compare_state(g, o, what="sgns free-running")
+    assert close(loss_of(g), o.loss[0])
+
+
+@pytest.mark.parametrize("dim,window,n_neg,batch,T", [(300, 5, 3, 200, 650), (8, 2, 0, 64, 130), (128, 1, 5, 100, 100),
+                                                      (512, 3, 2, 40, 41)])
+def test_sgns_shapes(dim, window, n_neg, batch, T):
+    cfg = W.scaled(W.SGNS_TINY, vocab=500, n_tokens=T, dim=dim, window=window, n_neg=n_neg, batch=batch)
+    sgns_run(cfg, range(cfg.n_batches), single_step=True, random_init=True)
+
+
+# ------------------------------------------------------- host variants ----
+def test_host_batch_variants_match_the_device_calls():
+    cfg = W.MF_TINY
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    a, _ = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
+    b, _ = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
+    h_loss = torch.zeros(1, dtype=torch.float64).pin_memory()
+    for s in range(0, 5 * cfg.batch, cfg.batch):
+        sl = slice(s, s + cfg.batch)
+        ps.ps_step_mf(a.h, i[sl].cuda(), j[sl].cuda(), v[sl].cuda(), cfg.col_key_base, cfg.lr, cfg.lam, a.loss)
+        ps.ps_step_mf_host(b.h, i[sl].pin_memory(), j[sl].pin_memory(), v[sl].pin_memory(), cfg.col_key_base, cfg.lr,
+                           cfg.lam, b.loss, h_loss)
+        a.sync()
+        assert h_loss[0] == loss_of(a)
+    assert (a.export(table=False)[0] == b.export(table=False)[0]).all()
+
+    kc = W.KGE_TINY
+    rows = W.kge_init_rows(kc, 0, kc.num_keys, "cpu")
+    a, _ = make_pair(kc.num_keys, kc.row_len, rows=rows, max_batch_keys=13 * kc.batch)
+    b, _ = make_pair(kc.num_keys, kc.row_len, rows=rows, max_batch_keys=13 * kc.batch)
+    s, r, t, neg, side = W.kge_triples(kc, 0, kc.batch, "cpu")
+    ps.ps_step_kge(a.h, s.cuda(), r.cuda(), t.cuda(), neg.cuda(), side.cuda(), kc.n_neg, kc.rel_key_base, kc.dim, kc.lr, kc.eps, a.loss)
+    ps.ps_step_kge_host(b.h, s, r, t, neg.contiguous(), side.contiguous(), kc.n_neg, kc.rel_key_base, kc.dim, kc.lr, kc.eps, b.loss, h_loss)
+    a.sync()
+    assert h_loss[0] == loss_of(a) and (a.export(table=False)[0] == b.export(table=False)[0]).all()
+
+    sc = W.SGNS_TINY
+    rows = torch.from_numpy(np.random.default_rng(1).normal(0, 0.3, size=(sc.num_keys, sc.dim)).astype(np.float32))
+    occ = sc.batch * (1 + 2 * sc.window * (1 + sc.n_neg))
+    a, _ = make_pair(sc.num_keys, sc.dim, rows=rows, max_batch_keys=occ)
+    b, _ = make_pair(sc.num_keys, sc.dim, rows=rows, max_batch_keys=occ)
+    tokens = W.sgns_tokens(sc, 0, sc.n_tokens, "cpu")
+    first, n = sc.batch_range(3)
+    negs = W.sgns_negatives(sc, first, n, "cpu")
+    ps.ps_step_sgns(a.h, tokens.cuda(), first, n, sc.window, negs.cuda(), sc.n_neg, sc.out_key_base, sc.lr, a.loss)
+    lo, hi = first - sc.window, first + n + sc.window
+    ps.ps_step_sgns_host(b.h, tokens[lo:hi].contiguous(), lo, first, n, sc.n_tokens, sc.window, negs, sc.n_neg,
+                         sc.out_key_base, sc.lr, b.loss, h_loss)
+    a.sync()
+    assert h_loss[0] == loss_of(a) and (a.export(table=False)[0] == b.export(table=False)[0]).all()
