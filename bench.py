@@ -1,0 +1,673 @@
+"""Benchmark of the parameter-store hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mf_large] [--impl ours|reference]
+
+A step is one pass of the whole hot path over one batch of seeded synthetic
+input: for the training workloads one fused pull -> gradient -> push call
+(ps_step_mf / ps_step_kge / ps_step_sgns), for the stress workload one ps_pull,
+one ps_push and one ps_localize.  Default workload: matrix factorization,
+10M x 1M, rank 100, minibatches of 65,536 cells.  The path does not shard
+(one GPU holds the whole store), so with N > 1 every rank runs an independent
+replica and the value is the sum over replicas.
+
+Prints ONE JSON line: throughput with the batch resident in HBM (`value`),
+the same through the host-buffer entry point (`e2e`), the fraction of the
+measured HBM copy bandwidth that the algorithmic bytes of a step reach
+(`roofline`), a per-kernel time table (`kernels`), and the CPU oracle timed on
+a bounded sample of the same workload (`cpu_baseline`).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from synth import workloads as W
+
+METRIC = "sgd_examples_per_sec"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ----------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons of one GPU through NVML while the timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._halt = threading.Event()
+        self.h = None
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = torch.cuda.get_device_properties(device_index).uuid
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.h = None
+
+    def run(self):
+        if self.h is None:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            except Exception:
+                break
+            time.sleep(0.002)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        if self.h is None or not self.samples:
+            return smi_clocks()
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in self.REASONS.items() if self.reason_bits & b], "samples": len(self.samples),
+                "source": "nvml"}
+
+
+def smi_clocks():
+    try:
+        out = subprocess.run(["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm,clocks_event_reasons.active",
+                              "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=10).stdout
+        sm, mx, reasons = [x.strip() for x in out.splitlines()[0].split(",")]
+        return {"sm_mhz": float(sm), "sm_max_mhz": float(mx), "reasons": [reasons], "samples": 1,
+                "source": "nvidia-smi after the timed region"}
+    except Exception as e:                                     # noqa: BLE001
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": f"unavailable: {e}"}
+
+
+# ----------------------------------------------------------------------------------------
+# workloads
+# ----------------------------------------------------------------------------------------
+def n_unique(*tensors) -> int:
+    return int(torch.unique(torch.cat([t.reshape(-1).to(torch.int64) for t in tensors])).numel())
+
+
+class MFWorkload:
+    """Matrix factorization (Section 4.1 task): cells/s through ps_step_mf."""
+
+    def __init__(self, cfg):
+        self.cfg, self.example = cfg, "cells"
+        self.row_bytes = cfg.rank * 4
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": c.name, "rows": c.rows, "cols": c.cols, "rank": c.rank, "minibatch": c.batch,
+                "store_gb": round(c.num_keys * c.rank * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def max_steps(self):
+        return self.cfg.n_batches - 1                           # full batches only
+
+    def gen_init(self, device, chunk=1 << 20):
+        for s in range(0, self.cfg.num_keys, chunk):
+            c = min(chunk, self.cfg.num_keys - s)
+            yield s, W.mf_init_rows(self.cfg, s, c, device)
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        self.store = ps.Store(c.num_keys, c.rank, 1, max_batch_keys=2 * c.batch, device=device.index)
+        self.host_init = torch.empty((c.num_keys, c.rank), dtype=torch.float32) if keep_host_init else None
+        for s, rows in self.gen_init(device):
+            self.store.set_rows(torch.arange(s, s + rows.shape[0], dtype=torch.int64, device=device), rows)
+            if keep_host_init:
+                self.host_init[s:s + rows.shape[0]] = rows.cpu()
+        planted = W.mf_planted(c, device)
+        self.i, self.j, self.v = W.mf_cells(c, planted, 0, n_steps * c.batch, device)
+        del planted
+        torch.cuda.synchronize(device)
+
+    def units(self, k):
+        return self.cfg.batch
+
+    def step(self, k):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice(k * b, (k + 1) * b)
+        self.ps.ps_step_mf(self.store.h, self.i[sl], self.j[sl], self.v[sl], c.col_key_base, c.lr, c.lam,
+                           self.store.loss)
+
+    def host_setup(self, steps):
+        b = self.cfg.batch
+        n = len(steps) * b
+        lo = steps[0] * b
+        self.hi_, self.hj_, self.hv_ = (t[lo:lo + n].cpu().pin_memory() for t in (self.i, self.j, self.v))
+        self.h_lo = steps[0]
+        self.h_loss = torch.zeros(1, dtype=torch.float64).pin_memory()
+        return b * 12, 8
+
+    def step_host(self, k):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice((k - self.h_lo) * b, (k - self.h_lo + 1) * b)
+        self.ps.ps_step_mf_host(self.store.h, self.hi_[sl], self.hj_[sl], self.hv_[sl], c.col_key_base, c.lr, c.lam,
+                                self.store.loss, self.h_loss)
+
+    def alg_bytes(self, k):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice(k * b, (k + 1) * b)
+        u = n_unique(self.i[sl]) + n_unique(self.j[sl])
+        return b * 12 + 2 * b * (8 + self.row_bytes) + u * 2 * self.row_bytes
+
+    # --- oracle leg ---
+    def oracle_setup(self, device):
+        from oracle import OracleStore
+        c = self.cfg
+        o = OracleStore(c.num_keys, c.rank, 1)
+        if getattr(self, "host_init", None) is not None:
+            for s in range(0, c.num_keys, 1 << 20):
+                e = min(s + (1 << 20), c.num_keys)
+                o.set_rows(np.arange(s, e), self.host_init[s:e].numpy())
+        else:
+            for s, rows in self.gen_init(device):
+                o.set_rows(np.arange(s, s + rows.shape[0]), rows.cpu().numpy())
+        self.oracle = o
+        return o
+
+    def oracle_data(self, device, n_steps):
+        if not hasattr(self, "i"):
+            planted = W.mf_planted(self.cfg, device)
+            self.i, self.j, self.v = W.mf_cells(self.cfg, planted, 0, n_steps * self.cfg.batch, device)
+        n = n_steps * self.cfg.batch
+        self.oi, self.oj, self.ov = (t[:n].cpu().numpy() for t in (self.i, self.j, self.v))
+
+    def oracle_step(self, k, cells):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice(k * b, k * b + cells)
+        self.oracle.step_mf(self.oi[sl], self.oj[sl], self.ov[sl], c.col_key_base, c.lr, c.lam)
+        return cells
+
+
+class KGEWorkload:
+    """ComplEx + AdaGrad (Section 4.1 / Appendix A task): triples/s through ps_step_kge."""
+
+    def __init__(self, cfg):
+        self.cfg, self.example = cfg, "triples"
+        self.row_bytes = cfg.row_len * 4
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": c.name, "entities": c.entities, "relations": c.relations, "dim_complex": c.dim,
+                "negatives": c.n_neg, "minibatch": c.batch, "store_gb": round(c.num_keys * c.row_len * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def max_steps(self):
+        return self.cfg.n_batches - 1
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        self.store = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(3 + c.n_neg) * c.batch, device=device.index)
+        rows = W.kge_init_rows(c, 0, c.num_keys, device)
+        self.store.set_all_rows(rows)
+        self.host_init = rows.cpu() if keep_host_init else None
+        del rows
+        self.s, self.r, self.o, self.neg, self.side = W.kge_triples(c, 0, n_steps * c.batch, device)
+        torch.cuda.synchronize(device)
+
+    def units(self, k):
+        return self.cfg.batch
+
+    def _sl(self, k):
+        b = self.cfg.batch
+        return slice(k * b, (k + 1) * b)
+
+    def step(self, k):
+        c, sl = self.cfg, self._sl(k)
+        self.ps.ps_step_kge(self.store.h, self.s[sl], self.r[sl], self.o[sl], self.neg[sl], self.side[sl], c.n_neg,
+                            c.rel_key_base, c.dim, c.lr, c.eps, self.store.loss)
+
+    def host_setup(self, steps):
+        b = self.cfg.batch
+        lo, n = steps[0] * b, len(steps) * b
+        self.h = [t[lo:lo + n].cpu().contiguous().pin_memory() for t in (self.s, self.r, self.o, self.neg, self.side)]
+        self.h_lo = steps[0]
+        self.h_loss = torch.zeros(1, dtype=torch.float64).pin_memory()
+        return b * (12 + self.cfg.n_neg * 5), 8
+
+    def step_host(self, k):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice((k - self.h_lo) * b, (k - self.h_lo + 1) * b)
+        s, r, o, neg, side = (t[sl] for t in self.h)
+        self.ps.ps_step_kge_host(self.store.h, s, r, o, neg, side, c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps,
+                                 self.store.loss, self.h_loss)
+
+    def alg_bytes(self, k):
+        c, sl, b = self.cfg, self._sl(k), self.cfg.batch
+        occ = (3 + c.n_neg) * b
+        u = n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl])
+        return b * (12 + c.n_neg * 5) + occ * (8 + self.row_bytes) + u * 2 * self.row_bytes
+
+    def oracle_setup(self, device):
+        from oracle import OracleStore
+        c = self.cfg
+        o = OracleStore(c.num_keys, c.row_len, 1)
+        rows = self.host_init if getattr(self, "host_init", None) is not None else W.kge_init_rows(c, 0, c.num_keys, device).cpu()
+        o.set_rows(np.arange(c.num_keys), rows.numpy())
+        self.oracle = o
+        return o
+
+    def oracle_data(self, device, n_steps):
+        if not hasattr(self, "s"):
+            self.s, self.r, self.o, self.neg, self.side = W.kge_triples(self.cfg, 0, n_steps * self.cfg.batch, device)
+        n = n_steps * self.cfg.batch
+        self.od = [t[:n].cpu().numpy() for t in (self.s, self.r, self.o, self.neg, self.side)]
+
+    def oracle_step(self, k, n):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice(k * b, k * b + n)
+        s, r, o, neg, side = (t[sl] for t in self.od)
+        self.oracle.step_kge(s, r, o, neg, side, c.rel_key_base, c.dim, c.lr, c.eps)
+        return n
+
+
+class SGNSWorkload:
+    """Skip-gram with negative sampling (Section 4.1 / Appendix A task): center words/s through ps_step_sgns."""
+
+    def __init__(self, cfg):
+        self.cfg, self.example = cfg, "centers"
+        self.row_bytes = cfg.dim * 4
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": c.name, "vocab": c.vocab, "dim": c.dim, "window": c.window, "negatives": c.n_neg,
+                "minibatch_centers": c.batch, "store_gb": round(c.num_keys * c.dim * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def max_steps(self):
+        return min(self.cfg.n_batches - 2, 400)
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        occ = c.batch * (1 + 2 * c.window * (1 + c.n_neg))
+        self.store = ps.Store(c.num_keys, c.dim, 1, max_batch_keys=occ, device=device.index)
+        rows = W.sgns_init_rows(c, 0, c.num_keys, device)
+        # a trained-looking state instead of all-zero output vectors, so that the arithmetic is not degenerate
+        rows[c.vocab:] = W.sgns_init_rows(W.scaled(c, seed=c.seed + 1), 0, c.vocab, device)
+        self.store.set_all_rows(rows)
+        self.host_init = rows.cpu() if keep_host_init else None
+        del rows
+        self.prefix = n_steps * c.batch + c.window + 1
+        self.tokens = W.sgns_tokens(c, 0, self.prefix, device)
+        self.negs = [W.sgns_negatives(c, k * c.batch, c.batch, device) for k in range(n_steps)]
+        torch.cuda.synchronize(device)
+
+    def units(self, k):
+        return self.cfg.batch
+
+    def step(self, k):
+        c = self.cfg
+        self.ps.ps_step_sgns(self.store.h, self.tokens, k * c.batch, c.batch, c.window, self.negs[k], c.n_neg,
+                             c.out_key_base, c.lr, self.store.loss)
+
+    def host_setup(self, steps):
+        c = self.cfg
+        self.h_tokens = self.tokens.cpu().pin_memory()
+        self.h_negs = {k: self.negs[k].cpu().pin_memory() for k in steps}
+        self.h_loss = torch.zeros(1, dtype=torch.float64).pin_memory()
+        return (c.batch + 2 * c.window) * 4 + int(np.mean([v.numel() for v in self.h_negs.values()])) * 4, 8
+
+    def step_host(self, k):
+        c = self.cfg
+        first = k * c.batch
+        lo, hi = max(0, first - c.window), min(self.prefix, first + c.batch + c.window)
+        self.ps.ps_step_sgns_host(self.store.h, self.h_tokens[lo:hi], lo, first, c.batch, self.prefix, c.window,
+                                  self.h_negs[k], c.n_neg, c.out_key_base, c.lr, self.store.loss, self.h_loss)
+
+    def alg_bytes(self, k):
+        c = self.cfg
+        first = k * c.batch
+        pairs = c.pairs_before(first + c.batch) - c.pairs_before(first)
+        centers = self.tokens[first:first + c.batch]
+        lo = max(0, first - c.window)
+        ctx = self.tokens[lo:first + c.batch + c.window]
+        u = n_unique(centers) + n_unique(ctx, self.negs[k])    # contexts: every token of the window span, to rounding
+        occ = c.batch + pairs * (1 + c.n_neg)
+        return c.batch * 4 + pairs * (1 + c.n_neg) * 4 + occ * (8 + self.row_bytes) + u * 2 * self.row_bytes
+
+    def oracle_setup(self, device):
+        from oracle import OracleStore
+        c = self.cfg
+        o = OracleStore(c.num_keys, c.dim, 1)
+        if getattr(self, "host_init", None) is not None:
+            rows = self.host_init
+        else:
+            rows = W.sgns_init_rows(c, 0, c.num_keys, device)
+            rows[c.vocab:] = W.sgns_init_rows(W.scaled(c, seed=c.seed + 1), 0, c.vocab, device)
+            rows = rows.cpu()
+        o.set_rows(np.arange(c.num_keys), rows.numpy())
+        self.oracle = o
+        return o
+
+    def oracle_data(self, device, n_steps):
+        c = self.cfg
+        if not hasattr(self, "tokens"):
+            self.prefix = n_steps * c.batch + c.window + 1
+            self.tokens = W.sgns_tokens(c, 0, self.prefix, device)
+            self.negs = [W.sgns_negatives(c, k * c.batch, c.batch, device) for k in range(n_steps)]
+        self.o_tokens = self.tokens.cpu().numpy()
+        self.o_negs = [t.cpu().numpy() for t in self.negs[:n_steps]]
+
+    def oracle_step(self, k, n):
+        c = self.cfg
+        first = k * c.batch
+        pairs = c.pairs_before(first + n) - c.pairs_before(first)
+        self.oracle.step_sgns(self.o_tokens, first, n, c.window, self.o_negs[k][:pairs * c.n_neg], c.n_neg,
+                              c.out_key_base, c.lr)
+        return n
+
+
+class StressWorkload:
+    """pull + push + localize of one key batch: keys/s through ps_pull, ps_push, ps_localize."""
+
+    POOL = 8        # distinct pre-generated batches; step k uses batch k % POOL's updates and batch k's keys
+
+    def __init__(self, cfg):
+        self.cfg, self.example = cfg, "keys"
+        self.row_bytes = cfg.row_len * 4
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": c.name, "keys": c.num_keys, "row_len": c.row_len, "workers": c.workers,
+                "batch_keys": c.batch, "localize_keys": c.localize_count,
+                "store_gb": round(c.workers * c.slots_per_part * c.row_len * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def max_steps(self):
+        return min(self.cfg.n_batches, 200)
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        self.store = ps.Store(c.num_keys, c.row_len, c.workers, c.slots_per_part, max_batch_keys=c.batch,
+                              device=device.index)
+        chunk = 1 << 21
+        for s in range(0, c.num_keys, chunk):
+            n = min(chunk, c.num_keys - s)
+            self.store.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=device),
+                                W.stress_init_rows(c, s, n, device))
+        self.keys = [W.stress_keys(c, k, device) for k in range(n_steps)]
+        self.upd = [W.stress_updates(c, k, device) for k in range(min(self.POOL, n_steps))]
+        self.out = torch.empty((c.batch, c.row_len), dtype=torch.float32, device=device)
+        self.moved_before = 0
+        torch.cuda.synchronize(device)
+
+    def units(self, k):
+        return self.cfg.batch
+
+    def step(self, k):
+        c, h = self.cfg, self.store.h
+        self.ps.ps_pull(h, self.keys[k], self.out)
+        self.ps.ps_push(h, self.keys[k], self.upd[k % len(self.upd)])
+        self.ps.ps_localize(h, c.requester(k), self.keys[k][:c.localize_count])
+
+    def host_setup(self, steps):
+        return None
+
+    def alg_bytes(self, k):
+        c, n, rb = self.cfg, self.cfg.batch, self.row_bytes
+        u = n_unique(self.keys[k])
+        pull = n * (16 + 2 * rb)
+        push = n * (16 + rb) + u * 2 * rb
+        loc = c.localize_count * 16                              # rows moved are added from the device counter
+        return pull + push + loc
+
+    def oracle_setup(self, device):
+        return None
+
+
+def make_workload(name):
+    table = {"mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
+             "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
+             "sgns": lambda: SGNSWorkload(W.SGNS), "sgns_tiny": lambda: SGNSWorkload(W.SGNS_TINY),
+             "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY)}
+    return table[name]()
+
+
+# ----------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------
+def dist_setup(n_gpus):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl" if torch.cuda.is_available() else "gloo")
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x, world, device):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def timed_loop(fn, steps, device, world):
+    """CUDA-event time (ms) of fn(k) for k in steps, bracketed by barrier + synchronize."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    torch.cuda.synchronize(device)
+    a.record()
+    for k in steps:
+        fn(k)
+    b.record()
+    torch.cuda.synchronize(device)
+    barrier(world)
+    return max_over_ranks(a.elapsed_time(b), world, device)
+
+
+def cpu_baseline(wl, device, max_steps, budget_s=15.0):
+    """The oracle, as it stands, on this machine's host cores (one thread), on a bounded sample of the workload."""
+    if wl.oracle_setup(device) is None:
+        return None
+    wl.oracle_data(device, max_steps)
+    full = wl.units(0)
+    t0 = time.perf_counter()
+    done, k = 0, 0
+    probe = max(1, full // 16)
+    done += wl.oracle_step(0, probe)                            # a short probe sizes the rest
+    rate = done / max(time.perf_counter() - t0, 1e-9)
+    k = 1
+    while k < max_steps and (time.perf_counter() - t0) + full / rate < budget_s:
+        done += wl.oracle_step(k, full)
+        k += 1
+    dt = time.perf_counter() - t0
+    return {"value": done / dt, "unit": f"{wl.example}/s", "cores": 1, "kind": "oracle", "host_cores": os.cpu_count(),
+            "sample": f"{done} {wl.example} ({k} batches: one of {probe}, then full ones) of {wl.cfg.name}, "
+                      f"{dt:.1f} s of CPU time, sequential C oracle, fp64 accumulation"}
+
+
+def run_ours(args):
+    import paper_2002_00655_b200 as ps
+    rank, world, local = dist_setup(args.gpus)
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device: the library has no CPU path"
+    device = torch.device("cuda", local if world > 1 else 0)
+    torch.cuda.set_device(device)
+    wl = make_workload(args.workload)
+    steps = min(args.steps, wl.max_steps() - args.warmup)
+    e2e_steps = min(steps, 200)
+    prof_steps = min(steps, 50)
+    total = args.warmup + steps
+    want_cpu = world == 1 and not args.no_cpu_baseline
+    wl.setup(ps, device, total, keep_host_init=want_cpu)
+    h = wl.store.h
+    code = wl.store.sync(check=False)
+    assert code == 0, f"device error during setup: {code}"
+
+    for k in range(args.warmup):
+        wl.step(k)
+    torch.cuda.synchronize(device)
+    launches0 = ps.ps_launch_count(h)
+    moved0 = ps.ps_rows_moved(h)
+    sampler = ClockSampler(device.index)
+    sampler.start()
+    timed = list(range(args.warmup, total))
+    ms = timed_loop(wl.step, timed, device, world)
+    clocks = sampler.stop()
+    launches = ps.ps_launch_count(h) - launches0
+    moved = ps.ps_rows_moved(h) - moved0
+    code = wl.store.sync(check=False)
+    assert code == 0, f"device error in the timed region: {ps.ps_status_string(code)}"
+    loss = float(wl.store.loss.cpu()[0])
+    assert np.isfinite(loss), "non-finite loss"
+
+    units = sum(wl.units(k) for k in timed)
+    value = units * world / (ms / 1e3)
+    sample_ks = timed[:: max(1, len(timed) // 16)]
+    alg = float(np.mean([wl.alg_bytes(k) for k in sample_ks]))
+    if moved:
+        alg += moved / len(timed) * (2 * wl.row_bytes + 8)
+    peak, peak_src = measured_hbm_peak()
+    achieved = alg / (ms / 1e3 / len(timed)) / 1e9
+
+    # end to end: batch in pinned host memory, copies and the loss read-back inside the timed region
+    e2e = None
+    e2e_ks = timed[:e2e_steps]
+    hb = wl.host_setup(e2e_ks)
+    if hb is not None:
+        h2d, d2h = hb
+        for k in e2e_ks[:3]:
+            wl.step_host(k)
+        ms_e = timed_loop(wl.step_host, e2e_ks, device, world)
+        e2e = {"value": sum(wl.units(k) for k in e2e_ks) * world / (ms_e / 1e3), "unit": f"{wl.example}/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": len(e2e_ks),
+               "ms_per_step": ms_e / len(e2e_ks)}
+
+    # per-kernel times from event pairs around every launch (a separate, untimed pass)
+    ps.ps_profile_start(h, 64 * prof_steps + 64)
+    for k in timed[:prof_steps]:
+        wl.step(k)
+    prof = ps.ps_profile_stop(h)
+    tot_us = sum(us for _, us in prof.values()) or 1.0
+    kernels = [{"name": name, "launches_per_step": n / prof_steps, "us_per_step": us / prof_steps,
+                "share": us / tot_us} for name, (n, us) in prof.items()]
+
+    out = {
+        "metric": METRIC, "value": value, "unit": f"{wl.example}/s", "n_gpus": world, "steps": len(timed),
+        "warmup": args.warmup, "ms_per_step": ms / len(timed), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "impl": "ours",
+        "config": dict(wl.describe(), parallelism="replicas only" if world > 1 else "single GPU",
+                       accumulation="per-key sums in f64, state f32"),
+        "gpu_launches": int(launches), "launches_per_step": launches / len(timed),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_step": alg,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "scope": "one step = all kernels of one C-ABI call sequence; algorithmic bytes = batch arrays "
+                              "+ occurrences x (8 B table entry + row read) + distinct keys x (row read + row write)"},
+        "kernels": kernels, "e2e": e2e, "clocks": clocks, "loss_sum": loss,
+    }
+    if want_cpu:
+        try:
+            out["cpu_baseline"] = cpu_baseline(wl, device, min(64, total))
+        except MemoryError as e:
+            out["cpu_baseline"] = {"unavailable": f"host memory: {e}"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on the same workload
+# ----------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    device = torch.device("cuda", 0) if torch.cuda.is_available() else torch.device("cpu")
+    wl = make_workload(args.workload)
+    if wl.oracle_setup(device) is None:
+        print(json.dumps({"impl": "reference", "unavailable": "no oracle leg for this workload at full size"}))
+        return
+    total = args.warmup + args.steps
+    n_batches = min(total, 64)
+    wl.oracle_data(device, n_batches)
+    full = wl.units(0)
+    # size one step so that the whole run stays within about two minutes
+    t0 = time.perf_counter()
+    probe = max(1, full // 16)
+    wl.oracle_step(0, probe)
+    rate = probe / max(time.perf_counter() - t0, 1e-9)
+    per_step = int(max(1, min(full, rate * 120.0 / max(total, 1))))
+    for k in range(args.warmup):
+        wl.oracle_step(k % n_batches, per_step)
+    t0 = time.perf_counter()
+    done = 0
+    for k in range(args.steps):
+        done += wl.oracle_step((args.warmup + k) % n_batches, per_step)
+    dt = time.perf_counter() - t0
+    value = done / dt
+    sample = (f"each step = the first {per_step} {wl.example} of a batch of {full} ({wl.cfg.name}); sequential C oracle, "
+              f"1 thread of {os.cpu_count()} host cores")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": f"{wl.example}/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": wl.describe(),
+        "cpu_baseline": {"value": value, "unit": f"{wl.example}/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": f"{wl.example}/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--workload", default="mf_large",
+                    choices=["mf_large", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
