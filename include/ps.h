@@ -176,6 +176,35 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
                               uint64_t n_negs, uint32_t n_neg, uint64_t out_key_base, float lr,
                               double* d_loss_accum, double* h_loss, void* stream);
 
+/* The push for callers that cannot allocate device memory (the paper has no
+ * counterpart to this entry point).  It is meant for code that runs where
+ * cudaMalloc is off limits: a plug-in inside an application whose own pool holds
+ * all GPU memory, a process with a fixed memory budget, a latency-critical loop
+ * that cannot afford the device-wide synchronisation an allocation implies.
+ * Such a caller cannot provide the workspace of ps_create, so this call needs
+ * no handle: all scratch memory (sort buffers, partial sums) lives in a static
+ * device array inside the library, about 2.3 MB, present on every GPU that
+ * loads the library until the process exits.  The call itself calls neither
+ * cudaMalloc nor cudaFree nor anything else that allocates.
+ *   d_store, d_table: a store and its location table as laid out by ps_create /
+ *   ps_init_range_partition (N * S rows of row_len fp32; (uint32 owner, uint32
+ *   slot) per key), on the CURRENT device; num_keys, row_len, slots_per_part as
+ *   in ps_config_t.  Result: exactly that of ps_push on the same arguments.
+ * Limits: n <= PS_PUSH_STATIC_MAX_KEYS and row_len <= PS_PUSH_STATIC_MAX_ROW_LEN
+ * (a multiple of 4); larger n returns PS_ERR_WORKSPACE, larger row_len
+ * PS_ERR_UNSUPPORTED, and nothing is enqueued.
+ * The call enqueues on `stream`, WAITS for it, and returns PS_ERR_KEY_RANGE
+ * (store untouched) if a key is >= num_keys.
+ * The first call on each device looks up the array's device address; make that
+ * first call outside any stream capture.  Every call on a GPU uses the same
+ * array: two calls that overlap in time on one GPU (different streams or
+ * threads) race on it, so serialise them. */
+#define PS_PUSH_STATIC_MAX_KEYS 16384
+#define PS_PUSH_STATIC_MAX_ROW_LEN 256
+ps_status_t ps_push_static(void* d_store, const void* d_table, uint64_t num_keys, uint32_t row_len,
+                           uint64_t slots_per_part, const uint64_t* d_keys, uint64_t n,
+                           const float* d_updates, void* stream);
+
 /* d_owner[t], d_slot[t] = current location of d_keys[t]. */
 ps_status_t ps_get_location(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner,
                             uint32_t* d_slot, void* stream);

@@ -26,6 +26,8 @@ PS_ERR_CAPACITY = 4
 PS_ERR_WORKSPACE = 5
 PS_ERR_CUDA = 6
 PS_ERR_UNSUPPORTED = 7
+PS_PUSH_STATIC_MAX_KEYS = 16384
+PS_PUSH_STATIC_MAX_ROW_LEN = 256
 
 
 class ps_config_t(C.Structure):
@@ -57,6 +59,7 @@ SIGNATURES = {
     "ps_step_kge_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _u32, _f32, _f32, _vp, _vp, _vp]),
     "ps_step_sgns_host": (C.c_int, [_vp, _vp, _u64, _u64, _u64, _u64, _u64, _u32, _vp, _u64, _u32, _u64, _f32, _vp,
                                     _vp, _vp]),
+    "ps_push_static": (C.c_int, [_vp, _vp, _u64, _u32, _u64, _vp, _u64, _vp, _vp]),
     "ps_get_location": (C.c_int, [_vp, _vp, _u64, _vp, _vp, _vp]),
     "ps_export": (C.c_int, [_vp, _vp, _vp, _vp]),
     "ps_export_freelists": (C.c_int, [_vp, _vp, _vp]),
@@ -208,6 +211,12 @@ def ps_step_sgns_host(ps, h_tokens, tok_first, first_pos, n_centers, corpus_len,
                                             n_centers, corpus_len, window, _hptr(h_negs, _U32), h_negs.numel(),
                                             n_neg, out_key_base, lr, _dptr(d_loss_accum, _F64),
                                             _hptr(h_loss, _F64), _stream()), "ps_step_sgns_host")
+
+
+def ps_push_static(d_store, d_table, num_keys, row_len, slots_per_part, d_keys, d_updates) -> int:
+    """Handle-free push that allocates nothing (static scratch inside the library); returns the status code."""
+    return load_library().ps_push_static(_dptr(d_store, _F32), _dptr(d_table), num_keys, row_len, slots_per_part,
+                                         _dptr(d_keys, _U64), d_keys.numel(), _dptr(d_updates, _F32), _stream())
 
 
 def ps_get_location(ps, d_keys, d_owner, d_slot):
