@@ -36,6 +36,8 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     l.scan_sums = take(((mk + 255) / 256) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
+    l.starters = take(reduce_tiles * 4);
+    l.starter_count = take(4);
     l.loss_partial = take(kMaxLossBlocks * 8);
     l.staging = take(mk * 8 + 256);
     l.total = off;
@@ -156,6 +158,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
+    ps->starters = (uint32_t*)(ps->ws + l.starters);
+    ps->starter_count = (unsigned int*)(ps->ws + l.starter_count);
     ps->loss_partial = (double*)(ps->ws + l.loss_partial);
     ps->staging = ps->ws + l.staging;
     int sms = 0;

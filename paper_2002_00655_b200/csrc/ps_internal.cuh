@@ -52,6 +52,8 @@ struct ps_store {
     uint32_t* scan_sums;            // block sums of the device-wide scan
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
+    uint32_t* starters;             // tiles that start a border-crossing segment (nReduceTiles)
+    unsigned int* starter_count;
     double* loss_partial;           // kMaxLossBlocks
     char* staging;                  // host-batch staging, max_keys x 8 bytes
     // host state
@@ -64,8 +66,8 @@ struct ps_store {
 namespace psb {
 
 struct WsLayout {
-    size_t status, keysA, keysB, valsA, valsB, hist, totals, scan_sums, upd, carry, loss_partial,
-        staging, total;
+    size_t status, keysA, keysB, valsA, valsB, hist, totals, scan_sums, upd, carry, starters, starter_count,
+        loss_partial, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
 
@@ -91,8 +93,9 @@ void prof_after(ps_store* ps, cudaStream_t s);
 // implied as 0..n-1 when iota_vals.  If n_dev is not null the element count is
 // read from device memory (n is then an upper bound used for the launch
 // shapes).  Returns 0 if the result is in the A buffers, 1 if in the B buffers.
+// If zero_me is not null the first kernel also sets *zero_me = 0.
 int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
-                     cudaStream_t stream, int start);
+                     cudaStream_t stream, int start, unsigned int* zero_me);
 
 // ---- pull_push.cu ----
 void launch_init_range_partition(ps_store* ps, cudaStream_t s);

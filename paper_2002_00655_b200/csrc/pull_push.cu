@@ -174,16 +174,26 @@ struct d4 {
     double x, y, z, w;
 };
 
+constexpr int kReduceGroup = 4;     // sorted occurrences whose loads are issued together
+constexpr int kFixupWarps = 8;
+
 // A warp owns sorted positions [tile*32, tile*32+32).  A segment (run of equal
-// keys) that starts and ends inside the tile is summed and applied here; a
-// segment that continues from the previous tile parks its partial sum in carry
-// slot 0 of the tile, one that continues into the next tile in slot 1.
+// keys) that starts and ends inside the tile is summed in fp64 and applied with
+// one read-modify-write of its row; a segment that continues from the previous
+// tile parks its partial sum in carry slot 0 of the tile, one that continues
+// into the next tile in slot 1, and the tile that starts such a segment is
+// appended to the list the fix-up kernel works through.
+// Every lane looks up the row of its own position's key, so the 32 table reads
+// go out together; then the positions are walked in groups whose update rows
+// and target rows are all requested before the first is used.
 __global__ void __launch_bounds__(256)
 push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
                    const float4* __restrict__ upd, float4* __restrict__ store, const uint2* __restrict__ table,
-                   uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry, const DevStatus* st,
-                   unsigned int epoch) {
+                   uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry,
+                   uint32_t* __restrict__ starters, unsigned int* __restrict__ starter_count,
+                   const DevStatus* st, unsigned int epoch) {
     if (call_failed(st, epoch)) return;
+    const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t base = (uint64_t)tile * kReduceTile;
@@ -191,120 +201,167 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
     const uint32_t n_valid = (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base);
     const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
     const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
-    uint32_t prev = __shfl_up_sync(0xffffffffu, key, 1);
+    const bool usable = key < K;                    // "no key" marks and padding sort last
+    uint64_t row = 0;
+    if (usable) row = phys_row(table[key], S);
+    uint32_t prev = __shfl_up_sync(full, key, 1);
     if (lane == 0) prev = base > 0 ? sk[base - 1] : kSentinelPad;
-    const bool head = key != prev;
     const uint32_t next_after = (base + kReduceTile < n) ? sk[base + kReduceTile] : kSentinelPad;
-    const bool head0 = __shfl_sync(0xffffffffu, (int)head, 0) != 0;
-    unsigned heads = __ballot_sync(0xffffffffu, head) | 1u;
+    uint32_t next = __shfl_down_sync(full, key, 1);
+    if (lane == 31) next = next_after;
+    const unsigned head_mask = __ballot_sync(full, key != prev);
+    const unsigned usable_mask = __ballot_sync(full, usable);
+    // positions at which a segment's part in this tile ends: its true end, or the tile's last position
+    const unsigned end_mask = __ballot_sync(full, usable && (key != next || lane == 31));
+    // positions before the first head belong to a segment that came in from the previous tile
+    const int first_head = head_mask ? (__ffs(head_mask) - 1) : 32;
+    // the last segment runs on iff the position after the tile holds the same usable key
+    const uint32_t key31 = __shfl_sync(full, key, 31);
+    const bool runs_on = key31 < K && next_after == key31;
+    // a border-crossing segment starts in this tile iff it runs on and has its head here
+    if (runs_on && head_mask != 0u && lane == 0) starters[atomicAdd(starter_count, 1u)] = tile;
     const uint32_t L = L4 * 4;
-    while (heads) {
-        const int start = __ffs(heads) - 1;
-        heads &= heads - 1;
-        int end = heads ? (__ffs(heads) - 1) : kReduceTile;
-        const uint32_t rkey = __shfl_sync(0xffffffffu, key, start);
-        if (rkey >= K) break;                       // "no key" marks sort last
-        const bool to_tile_end = end >= (int)n_valid;
-        if (to_tile_end) end = (int)n_valid;
-        const bool cont_start = (start == 0) && !head0;
-        const bool cont_end = to_tile_end && n_valid == kReduceTile && next_after == rkey;
-        const uint64_t row = phys_row(table[rkey], S);
-        for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
-            const uint32_t f = f0 + lane;
-            const bool act = f < L4;
-            d4 acc = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll 4
-            for (int p = start; p < end; ++p) {
-                const uint32_t o = __shfl_sync(0xffffffffu, occ, p);
-                if (act) {
-                    const float4 u = __ldcs(upd + (uint64_t)o * L4 + f);
-                    acc.x += (double)u.x; acc.y += (double)u.y; acc.z += (double)u.z; acc.w += (double)u.w;
-                }
+    for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
+        const uint32_t f = f0 + lane;
+        const bool act = f < L4;
+        d4 acc = {0.0, 0.0, 0.0, 0.0};
+        for (int p0 = 0; p0 < (int)n_valid; p0 += kReduceGroup) {
+            float4 u[kReduceGroup], r[kReduceGroup];
+            uint64_t rows[kReduceGroup];
+#pragma unroll
+            for (int k = 0; k < kReduceGroup; ++k) {
+                const int p = p0 + k;                       // p <= 31 because p0 < n_valid <= 32 and p0 % 4 == 0
+                const uint32_t o = __shfl_sync(full, occ, p);
+                rows[k] = __shfl_sync(full, row, p);
+                const bool ok = (usable_mask >> p) & 1u;
+                const bool ends = ok && ((end_mask >> p) & 1u);
+                const bool parked = ends && (p < first_head || (p == 31 && runs_on));
+                u[k] = (ok && act) ? __ldcs(upd + (uint64_t)o * L4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+                r[k] = (ends && !parked && act) ? store[rows[k] * L4 + f] : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            if (!act) continue;
-            if (!cont_start && !cont_end) {
-                float4 r = store[row * L4 + f];
-                r.x = (float)((double)r.x + acc.x); r.y = (float)((double)r.y + acc.y);
-                r.z = (float)((double)r.z + acc.z); r.w = (float)((double)r.w + acc.w);
-                store[row * L4 + f] = r;
-            } else {
-                double* c = carry + ((uint64_t)tile * 2 + (cont_start ? 0 : 1)) * L + (uint64_t)f * 4;
-                *(double2*)c = make_double2(acc.x, acc.y);
-                *(double2*)(c + 2) = make_double2(acc.z, acc.w);
+#pragma unroll
+            for (int k = 0; k < kReduceGroup; ++k) {
+                const int p = p0 + k;
+                if (!((usable_mask >> p) & 1u)) continue;
+                acc.x += (double)u[k].x; acc.y += (double)u[k].y; acc.z += (double)u[k].z; acc.w += (double)u[k].w;
+                if ((end_mask >> p) & 1u) {
+                    const bool from_prev = p < first_head;
+                    const bool parked = from_prev || (p == 31 && runs_on);
+                    if (act) {
+                        if (!parked) {
+                            float4 v = r[k];
+                            v.x = (float)((double)v.x + acc.x); v.y = (float)((double)v.y + acc.y);
+                            v.z = (float)((double)v.z + acc.z); v.w = (float)((double)v.w + acc.w);
+                            store[rows[k] * L4 + f] = v;
+                        } else {
+                            double* c = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
+                            *(double2*)c = make_double2(acc.x, acc.y);
+                            *(double2*)(c + 2) = make_double2(acc.z, acc.w);
+                        }
+                    }
+                    acc.x = acc.y = acc.z = acc.w = 0.0;
+                }
             }
         }
     }
 }
 
-// first index in [lo, n) whose key is greater than `key`
-__device__ __forceinline__ uint64_t upper_bound_u32(const uint32_t* __restrict__ a, uint64_t lo, uint64_t n,
-                                                    uint32_t key) {
-    uint64_t hi = n;
-    while (lo < hi) {
-        const uint64_t mid = (lo + hi) >> 1;
-        if (a[mid] <= key) lo = mid + 1; else hi = mid;
-    }
-    return lo;
-}
-
-// One warp per tile whose last segment starts in the tile and runs on into the
-// next: it adds the parked partials tile by tile and applies the sum.  The
-// block after the last tile block adds the call's loss partials, in index order.
-__global__ void __launch_bounds__(256)
+// Blocks work through the list of tiles that start a border-crossing segment.
+// For one such segment the block's warps add the parked partials of the tiles
+// it runs through (warp w takes every 8th tile), the eight warp sums are added
+// in warp order to the starting tile's own partial, and the row is updated.
+// The shape of this sum depends only on the sorted positions.  The last block
+// adds the call's loss partials, in index order.
+__global__ void __launch_bounds__(32 * kFixupWarps)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
-                  const double* __restrict__ carry, const double* __restrict__ loss_partial,
-                  uint32_t loss_blocks, double* __restrict__ loss_accum, uint32_t tile_blocks,
-                  const DevStatus* st, unsigned int epoch) {
+                  const double* __restrict__ carry, const uint32_t* __restrict__ starters,
+                  const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
+                  uint32_t loss_blocks, double* __restrict__ loss_accum, const DevStatus* st, unsigned int epoch) {
+    __shared__ d4 part[kFixupWarps][32];
     if (call_failed(st, epoch)) return;
-    if (blockIdx.x >= tile_blocks) {
-        if (loss_accum && threadIdx.x == 0) {
-            double tot = 0;
-            for (uint32_t b = 0; b < loss_blocks; ++b) tot += loss_partial[b];
-            *loss_accum += tot;
+    if (blockIdx.x == gridDim.x - 1) {
+        if (loss_accum) {                           // fixed-shape sum: strided per thread, then a tree
+            __shared__ double ws[kFixupWarps];
+            double t = 0;
+            for (uint32_t b = threadIdx.x; b < loss_blocks; b += blockDim.x) t += loss_partial[b];
+            t = warp_sum_d(t);
+            if ((threadIdx.x & 31) == 0) ws[threadIdx.x >> 5] = t;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                double tot = 0;
+                for (int i = 0; i < kFixupWarps; ++i) tot += ws[i];
+                *loss_accum += tot;
+            }
         }
         return;
     }
-    const int lane = threadIdx.x & 31;
-    const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t base = (uint64_t)tile * kReduceTile;
-    if (base + kReduceTile >= n) return;             // the last tile cannot run on
-    const uint32_t kl = sk[base + kReduceTile - 1];
-    if (kl >= K || sk[base + kReduceTile] != kl) return;
-    if (sk[base] == kl && base > 0 && sk[base - 1] == kl) return;   // continues a segment from before
-    const uint64_t end_pos = upper_bound_u32(sk, base + kReduceTile, n, kl);
-    const uint32_t last_tile = (uint32_t)((end_pos - 1) / kReduceTile);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t count = *starter_count;
     const uint32_t L = L4 * 4;
-    const uint64_t row = phys_row(table[kl], S);
-    for (uint32_t f = lane; f < L4; f += 32) {
-        const double* c = carry + ((uint64_t)tile * 2 + 1) * L + (uint64_t)f * 4;
-        double2 a = *(const double2*)c, b = *(const double2*)(c + 2);
-#pragma unroll 4
-        for (uint32_t t2 = tile + 1; t2 <= last_tile; ++t2) {
-            const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
-            const double2 a2 = *(const double2*)c2, b2 = *(const double2*)(c2 + 2);
-            a.x += a2.x; a.y += a2.y; b.x += b2.x; b.y += b2.y;
+    for (uint32_t si = blockIdx.x; si < count; si += gridDim.x - 1) {
+        const uint32_t tile = starters[si];
+        const uint64_t base = (uint64_t)tile * kReduceTile;
+        const uint32_t kl = sk[base + kReduceTile - 1];
+        const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
+        const uint64_t row = phys_row(table[kl], S);
+        // last tile of the segment: every later tile whose first key is the segment's key belongs to it
+        // (keys are sorted); the block's threads probe 256 tiles at a time
+        uint32_t last_tile = tile;
+        for (;;) {
+            const uint32_t t2 = last_tile + 1 + threadIdx.x;
+            const int hit = t2 < n_tiles && sk[(uint64_t)t2 * kReduceTile] == kl;
+            const int cnt = __syncthreads_count(hit);         // hits are a prefix of the probed range
+            last_tile += (uint32_t)cnt;
+            if (cnt < (int)blockDim.x) break;
         }
-        float4 r = store[row * L4 + f];
-        r.x = (float)((double)r.x + a.x); r.y = (float)((double)r.y + a.y);
-        r.z = (float)((double)r.z + b.x); r.w = (float)((double)r.w + b.y);
-        store[row * L4 + f] = r;
+        for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
+            const uint32_t f = f0 + lane;
+            const bool act = f < L4;
+            d4 a = {0.0, 0.0, 0.0, 0.0};
+            if (act) {
+#pragma unroll 4
+                for (uint32_t t2 = tile + 1 + w; t2 <= last_tile; t2 += kFixupWarps) {
+                    const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
+                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
+                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
+                }
+            }
+            part[w][lane] = a;
+            __syncthreads();
+            if (w == 0 && act) {
+                const double* c = carry + ((uint64_t)tile * 2 + 1) * L + (uint64_t)f * 4;
+                const double2 x = *(const double2*)c, y = *(const double2*)(c + 2);
+                d4 t = {x.x, x.y, y.x, y.y};
+#pragma unroll
+                for (int i = 0; i < kFixupWarps; ++i) {
+                    t.x += part[i][lane].x; t.y += part[i][lane].y; t.z += part[i][lane].z; t.w += part[i][lane].w;
+                }
+                float4 r = store[row * L4 + f];
+                r.x = (float)((double)r.x + t.x); r.y = (float)((double)r.y + t.y);
+                r.z = (float)((double)r.z + t.z); r.w = (float)((double)r.w + t.w);
+                store[row * L4 + f] = r;
+            }
+            __syncthreads();
+        }
     }
 }
 
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
                        cudaStream_t s) {
-    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0);
+    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count);
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     const uint32_t* sv = which ? ps->valsB : ps->valsA;
     const uint32_t tiles = div_up_u32(n, kReduceTile);
     const uint32_t blocks = div_up_u32(tiles, 8);
     const uint32_t L4 = ps->cfg.row_len / 4;
     PS_LAUNCH(ps, push_reduce_kernel, blocks, 256, s, sk, sv, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->status, ps->epoch);
-    PS_LAUNCH(ps, push_fixup_kernel, blocks + 1, 256, s, sk, n, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->loss_partial, loss_blocks,
-              loss_blocks ? d_loss_accum : nullptr, blocks, ps->status, ps->epoch);
+              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
+              ps->status, ps->epoch);
+    uint32_t fix_blocks = tiles < (uint32_t)ps->sm_count * 8 ? tiles : (uint32_t)ps->sm_count * 8;
+    PS_LAUNCH(ps, push_fixup_kernel, fix_blocks + 1, 32 * kFixupWarps, s, sk, n, (float4*)ps->store, ps->table,
+              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
+              ps->loss_partial, loss_blocks, loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch);
 }
 
 }  // namespace psb

@@ -29,8 +29,10 @@ constexpr size_t kOffValsB = kOffValsA + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffHist = kOffValsB + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffTotals = kOffHist + pad256(((kStaticMaxKeys + kSortTile - 1) / kSortTile) * kRadix * 4);
 constexpr size_t kOffCarry = kOffTotals + pad256(kRadix * 4);
-constexpr size_t kStaticBytes =
+constexpr size_t kOffStarters =
     kOffCarry + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 2 * (size_t)kStaticMaxRowLen * 8);
+constexpr size_t kOffStarterCount = kOffStarters + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 4);
+constexpr size_t kStaticBytes = kOffStarterCount + 256;
 
 // About 2.3 MB per GPU.  In host code this name is only a handle for the
 // runtime; the address a kernel can use comes from cudaGetSymbolAddress.
@@ -104,6 +106,8 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     tmp.hist = (uint32_t*)(dev.scratch + kOffHist);
     tmp.totals = (uint32_t*)(dev.scratch + kOffTotals);
     tmp.carry = (double*)(dev.scratch + kOffCarry);
+    tmp.starters = (uint32_t*)(dev.scratch + kOffStarters);
+    tmp.starter_count = (unsigned int*)(dev.scratch + kOffStarterCount);
     tmp.epoch = 1;
     tmp.sm_count = dev.sm_count;
 

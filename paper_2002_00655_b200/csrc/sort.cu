@@ -12,8 +12,9 @@ namespace psb {
 
 __global__ void __launch_bounds__(kSortThreads)
 sort_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n_host, const unsigned int* __restrict__ n_dev,
-                 int shift, uint32_t* __restrict__ counts, uint32_t n_tiles) {
+                 int shift, uint32_t* __restrict__ counts, uint32_t n_tiles, unsigned int* __restrict__ zero_me) {
     __shared__ uint32_t h[kRadix];
+    if (zero_me && blockIdx.x == 0 && threadIdx.x == 0) *zero_me = 0u;      // a counter a later kernel of the call uses
     const uint32_t n = n_dev ? tmin<uint32_t>(*n_dev, n_host) : n_host;
     h[threadIdx.x] = 0;
     __syncthreads();
@@ -108,7 +109,7 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
 }
 
 int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
-                     cudaStream_t stream, int start) {
+                     cudaStream_t stream, int start, unsigned int* zero_me) {
     if (n == 0) return start;
     const uint32_t n_tiles = div_up_u32(n, kSortTile);
     uint32_t *kin = ps->keysA, *vin = ps->valsA, *kout = ps->keysB, *vout = ps->valsB;
@@ -118,7 +119,8 @@ int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bi
     int which = start;
     if (bits < 1) bits = 1;
     for (int shift = 0; shift < bits; shift += kRadixBits) {
-        PS_LAUNCH(ps, sort_hist_kernel, n_tiles, kSortThreads, stream, kin, n, n_dev, shift, ps->hist, n_tiles);
+        PS_LAUNCH(ps, sort_hist_kernel, n_tiles, kSortThreads, stream, kin, n, n_dev, shift, ps->hist, n_tiles,
+                  shift == 0 ? zero_me : nullptr);
         PS_LAUNCH(ps, sort_scan_kernel, kRadix, 256, stream, ps->hist, n_tiles, ps->totals);
         if (iota_vals && shift == 0)
             PS_LAUNCH(ps, sort_scatter_kernel<true>, n_tiles, kSortThreads, stream, kin, vin, kout, vout, n, n_dev,
