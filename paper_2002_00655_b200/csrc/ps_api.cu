@@ -31,8 +31,8 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     l.keysB = take(mk * 4);
     l.valsA = take(mk * 4);
     l.valsB = take(mk * 4);
-    l.hist = take(sort_tiles * kRadix * 4);
-    l.totals = take(kRadix * 4);
+    l.tile_state = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
+    l.sort_ctl = take((size_t)kSortCtlWords * 4);
     l.scan_sums = take(((mk + 255) / 256) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
@@ -100,6 +100,15 @@ static ps_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? PS_OK : PS
 // are reported through the device status word.
 static ps_status_t after_launch() { return cuda_ok(cudaGetLastError()); }
 
+// The keys of a step's occurrences depend on the batch alone, so their extraction and sort run on the
+// handle's side stream while the gradient kernel runs on the caller's; both meet before the reduction.
+static bool fork_side(ps_store* ps, cudaStream_t s) {
+    return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
+}
+static bool join_side(ps_store* ps, cudaStream_t s) {
+    return cudaEventRecord(ps->ev_join, ps->side) == cudaSuccess && cudaStreamWaitEvent(s, ps->ev_join, 0) == cudaSuccess;
+}
+
 static void next_epoch(ps_store* ps) {
     ps->epoch++;
     if (ps->epoch == 0) ps->epoch = 1;
@@ -115,7 +124,7 @@ ps_status_t ps_query_sizes(const ps_config_t* cfg, uint64_t max_batch_keys, ps_s
     if (!out) return PS_ERR_INVALID_ARG;
     const ps_status_t c = check_cfg(cfg);
     if (c != PS_OK) return c;
-    if (max_batch_keys == 0 || max_batch_keys >= 0x7FFFFFFFull) return PS_ERR_INVALID_ARG;
+    if (max_batch_keys == 0 || max_batch_keys >= (1ull << 30)) return PS_ERR_INVALID_ARG;
     const uint64_t N = cfg->num_workers, S = cfg->slots_per_part;
     out->store_bytes = (size_t)(N * S) * cfg->row_len * 4;
     out->table_bytes = (size_t)cfg->num_keys * 8;
@@ -153,8 +162,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->keysB = (uint32_t*)(ps->ws + l.keysB);
     ps->valsA = (uint32_t*)(ps->ws + l.valsA);
     ps->valsB = (uint32_t*)(ps->ws + l.valsB);
-    ps->hist = (uint32_t*)(ps->ws + l.hist);
-    ps->totals = (uint32_t*)(ps->ws + l.totals);
+    ps->tile_state = (uint32_t*)(ps->ws + l.tile_state);
+    ps->sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl);
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
@@ -172,6 +181,15 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         delete ps;
         return PS_ERR_CUDA;
     }
+    // the side stream's small kernels should not queue behind the gradient kernel's waves of blocks
+    int prio_lo = 0, prio_hi = 0;
+    cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        delete ps;
+        return PS_ERR_CUDA;
+    }
     *out = ps;
     return PS_OK;
 }
@@ -181,6 +199,9 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     cudaSetDevice(ps->cfg.device);
     cudaDeviceSynchronize();
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
+    cudaEventDestroy(ps->ev_fork);
+    cudaEventDestroy(ps->ev_join);
+    cudaStreamDestroy(ps->side);
     delete ps;
     return PS_OK;
 }
@@ -240,8 +261,12 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (!d_i || !d_j || !d_v) return PS_ERR_INVALID_ARG;
     if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    launch_keys_mf(ps, d_i, d_j, n, col_key_base, ps->side);
+    const int which = run_push_sort(ps, (uint32_t)(2 * n), ps->side);
     const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
-    run_push_pipeline(ps, (uint32_t)(2 * n), ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_push_reduce(ps, (uint32_t)(2 * n), which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
     return after_launch();
 }
 
@@ -256,9 +281,14 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     if (dim_complex == 0 || ps->cfg.row_len != 4 * (uint64_t)dim_complex) return PS_ERR_INVALID_ARG;
     if ((3 + (uint64_t)n_neg) * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (rel_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    const uint32_t occ = (uint32_t)((3 + (uint64_t)n_neg) * n);
+    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    launch_keys_kge(ps, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base, ps->side);
+    const int which = run_push_sort(ps, occ, ps->side);
     const uint32_t lb =
         launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex, lr, eps, s);
-    run_push_pipeline(ps, (uint32_t)((3 + (uint64_t)n_neg) * n), ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_push_reduce(ps, occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
     return after_launch();
 }
 
@@ -281,9 +311,13 @@ ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t firs
     uint64_t occ;
     const ps_status_t c = sgns_checks(ps, first_pos, n_centers, corpus_len, window, n_neg, out_key_base, &occ);
     if (c != PS_OK) return c;
+    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    launch_keys_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, ps->side);
+    const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
     const uint32_t lb = launch_step_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
-    run_push_pipeline(ps, (uint32_t)occ, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
     return after_launch();
 }
 
@@ -366,9 +400,14 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     if (cudaMemcpyAsync(d_tok, h_tokens, tok_count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return PS_ERR_CUDA;
     if (n_negs && cudaMemcpyAsync(d_negs, h_negs, n_negs * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return PS_ERR_CUDA;
+    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    launch_keys_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base,
+                     ps->side);
+    const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
     const uint32_t lb = launch_step_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
-    run_push_pipeline(ps, (uint32_t)occ, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
     c = after_launch();
     if (c != PS_OK) return c;
     return finish_host_step(d_loss_accum, h_loss, s);

@@ -15,6 +15,8 @@ constexpr int kSortItems = 8;
 constexpr int kSortTile = kSortThreads * kSortItems;   // keys per sort block
 constexpr int kRadixBits = 8;
 constexpr int kRadix = 1 << kRadixBits;
+constexpr int kMaxSortPasses = 4;                // 32-bit keys
+constexpr int kSortCtlWords = kMaxSortPasses * kRadix + kMaxSortPasses;   // digit histograms of every pass, then tickets
 constexpr int kReduceTile = 32;                  // sorted occurrences per warp in the segmented reduction
 constexpr int kMaxLossBlocks = 4096;
 
@@ -47,8 +49,8 @@ struct ps_store {
     // carved out of the workspace
     psb::DevStatus* status;
     uint32_t *keysA, *keysB, *valsA, *valsB;
-    uint32_t* hist;                 // kRadix x nSortTiles
-    uint32_t* totals;               // kRadix
+    uint32_t* tile_state;           // kMaxSortPasses x nSortTiles x kRadix look-back words
+    uint32_t* sort_ctl;             // kSortCtlWords
     uint32_t* scan_sums;            // block sums of the device-wide scan
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
@@ -61,12 +63,14 @@ struct ps_store {
     uint64_t launches;
     int sm_count;
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
+    cudaStream_t side;              // key extraction and sort of a step run here, beside the gradient kernel
+    cudaEvent_t ev_fork, ev_join;
 };
 
 namespace psb {
 
 struct WsLayout {
-    size_t status, keysA, keysB, valsA, valsB, hist, totals, scan_sums, upd, carry, starters, starter_count,
+    size_t status, keysA, keysB, valsA, valsB, tile_state, sort_ctl, scan_sums, upd, carry, starters, starter_count,
         loss_partial, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
@@ -110,13 +114,25 @@ void launch_prepare_keys(ps_store* ps, const uint64_t* d_keys, uint64_t n, cudaS
 // first `loss_blocks` loss partials to *d_loss_accum (if not null)
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
                        cudaStream_t s);
+// the two halves of the above: sort keysA (returns which buffer holds the result), then reduce and apply
+int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s);
+void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
+                     uint32_t loss_blocks, cudaStream_t s);
 
 // ---- localize.cu ----
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s);
 
 // ---- steps.cu ----
-// Each writes the occurrences' keys to keysA and their update rows to `upd`, and
-// returns the number of per-block loss partials it wrote.
+// launch_keys_* write the keys of a batch's occurrence slots to keysA (they depend on the batch
+// only, so they and the sort can run beside the gradient kernel); launch_step_* write the slots'
+// update rows to `upd` and return the number of per-block loss partials they wrote.
+void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint64_t n, uint64_t col_key_base,
+                    cudaStream_t s);
+void launch_keys_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                     const uint32_t* d_neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_key_base, cudaStream_t s);
+void launch_keys_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
+                      uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs, uint32_t n_neg,
+                      uint64_t out_key_base, cudaStream_t s);
 uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
                         uint64_t col_key_base, float lr, float lambda, cudaStream_t s);
 uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,

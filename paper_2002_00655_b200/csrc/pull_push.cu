@@ -347,9 +347,12 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     }
 }
 
-void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
-                       cudaStream_t s) {
-    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count);
+int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
+    return radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count);
+}
+
+void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
+                     uint32_t loss_blocks, cudaStream_t s) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     const uint32_t* sv = which ? ps->valsB : ps->valsA;
     const uint32_t tiles = div_up_u32(n, kReduceTile);
@@ -362,6 +365,12 @@ void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_l
     PS_LAUNCH(ps, push_fixup_kernel, fix_blocks + 1, 32 * kFixupWarps, s, sk, n, (float4*)ps->store, ps->table,
               ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
               ps->loss_partial, loss_blocks, loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch);
+}
+
+void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
+                       cudaStream_t s) {
+    const int which = run_push_sort(ps, n, s);
+    run_push_reduce(ps, n, which, d_upd, d_loss_accum, loss_blocks, s);
 }
 
 }  // namespace psb

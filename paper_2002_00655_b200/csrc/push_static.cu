@@ -27,8 +27,9 @@ constexpr size_t kOffKeysB = kOffKeysA + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffValsA = kOffKeysB + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffValsB = kOffValsA + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffHist = kOffValsB + pad256(kStaticMaxKeys * 4);
-constexpr size_t kOffTotals = kOffHist + pad256(((kStaticMaxKeys + kSortTile - 1) / kSortTile) * kRadix * 4);
-constexpr size_t kOffCarry = kOffTotals + pad256(kRadix * 4);
+constexpr size_t kOffSortCtl =
+    kOffHist + pad256((size_t)kMaxSortPasses * ((kStaticMaxKeys + kSortTile - 1) / kSortTile) * kRadix * 4);
+constexpr size_t kOffCarry = kOffSortCtl + pad256((size_t)kSortCtlWords * 4);
 constexpr size_t kOffStarters =
     kOffCarry + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 2 * (size_t)kStaticMaxRowLen * 8);
 constexpr size_t kOffStarterCount = kOffStarters + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 4);
@@ -103,8 +104,8 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     tmp.keysB = (uint32_t*)(dev.scratch + kOffKeysB);
     tmp.valsA = (uint32_t*)(dev.scratch + kOffValsA);
     tmp.valsB = (uint32_t*)(dev.scratch + kOffValsB);
-    tmp.hist = (uint32_t*)(dev.scratch + kOffHist);
-    tmp.totals = (uint32_t*)(dev.scratch + kOffTotals);
+    tmp.tile_state = (uint32_t*)(dev.scratch + kOffHist);
+    tmp.sort_ctl = (uint32_t*)(dev.scratch + kOffSortCtl);
     tmp.carry = (double*)(dev.scratch + kOffCarry);
     tmp.starters = (uint32_t*)(dev.scratch + kOffStarters);
     tmp.starter_count = (unsigned int*)(dev.scratch + kOffStarterCount);

@@ -3,68 +3,79 @@
 // them segment by segment (cumulative push, Section 2.1 of the paper) and so
 // that localize sees each distinct key once, in ascending order.
 //
-// Per pass: (1) per-tile digit histograms, (2) one block per digit scans that
-// digit's counts across tiles, (3) each tile ranks its keys stably (warp
-// match + per-warp counters) and scatters.  No inter-block waiting anywhere.
+// One kernel builds the digit histograms of every pass at once (they do not
+// depend on the order of the keys).  Each pass is then a single kernel: a block
+// takes the next tile (an atomic ticket, so every earlier tile is already
+// running or done), ranks its keys stably inside the tile (warp match +
+// per-warp counters), publishes its per-digit counts, obtains the counts of all
+// earlier tiles by looking back over their published words (count-only or
+// running-total, one 32-bit word per tile and digit), and scatters.
+// The only waiting is the look-back; it is bounded, and a block that gives up
+// latches an error and writes nothing.
 #include "ps_internal.cuh"
 
 namespace psb {
 
+constexpr uint32_t kFlagCount = 1u << 30;    // the word holds this tile's count
+constexpr uint32_t kFlagTotal = 2u << 30;    // the word holds the total up to and including this tile
+constexpr uint32_t kValueMask = (1u << 30) - 1u;
+constexpr int kLookbackSpins = 1 << 22;
+constexpr int kLookbackWindow = 8;
+
+// ctl layout: [kMaxPasses][kRadix] histograms, then kMaxPasses tickets.
 __global__ void __launch_bounds__(kSortThreads)
 sort_hist_kernel(const uint32_t* __restrict__ keys, uint32_t n_host, const unsigned int* __restrict__ n_dev,
-                 int shift, uint32_t* __restrict__ counts, uint32_t n_tiles, unsigned int* __restrict__ zero_me) {
-    __shared__ uint32_t h[kRadix];
+                 int n_passes, uint32_t* __restrict__ ctl, uint32_t* __restrict__ tile_state, uint32_t n_tiles,
+                 unsigned int* __restrict__ zero_me) {
+    __shared__ uint32_t h[kMaxSortPasses][kRadix];
     if (zero_me && blockIdx.x == 0 && threadIdx.x == 0) *zero_me = 0u;      // a counter a later kernel of the call uses
     const uint32_t n = n_dev ? tmin<uint32_t>(*n_dev, n_host) : n_host;
-    h[threadIdx.x] = 0;
+    for (int p = 0; p < n_passes; ++p) {
+        h[p][threadIdx.x] = 0;
+        tile_state[((size_t)p * n_tiles + blockIdx.x) * kRadix + threadIdx.x] = 0u;
+    }
     __syncthreads();
     const uint32_t base = blockIdx.x * kSortTile;
 #pragma unroll
     for (int it = 0; it < kSortItems; ++it) {
-        uint32_t idx = base + it * kSortThreads + threadIdx.x;
-        if (idx < n) atomicAdd(&h[(keys[idx] >> shift) & (kRadix - 1)], 1u);
+        const uint32_t idx = base + it * kSortThreads + threadIdx.x;
+        if (idx < n) {
+            const uint32_t key = keys[idx];
+            for (int p = 0; p < n_passes; ++p) atomicAdd(&h[p][(key >> (p * kRadixBits)) & (kRadix - 1)], 1u);
+        }
     }
     __syncthreads();
-    counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
-}
-
-// Block d turns counts[d][0..n_tiles) into its exclusive prefix and writes the digit total.
-__global__ void __launch_bounds__(256)
-sort_scan_kernel(uint32_t* __restrict__ counts, uint32_t n_tiles, uint32_t* __restrict__ totals) {
-    __shared__ uint32_t sm[8];
-    uint32_t* row = counts + (size_t)blockIdx.x * n_tiles;
-    uint32_t running = 0;
-    for (uint32_t c0 = 0; c0 < n_tiles; c0 += 256) {
-        uint32_t i = c0 + threadIdx.x;
-        uint32_t v = i < n_tiles ? row[i] : 0;
-        uint32_t tot;
-        uint32_t ex = block_exclusive_scan_256(v, sm, &tot);
-        if (i < n_tiles) row[i] = running + ex;
-        running += tot;
+    for (int p = 0; p < n_passes; ++p) {
+        const uint32_t c = h[p][threadIdx.x];
+        if (c) atomicAdd(&ctl[p * kRadix + threadIdx.x], c);
     }
-    if (threadIdx.x == 0) totals[blockIdx.x] = running;
 }
 
 template <bool kIota>
 __global__ void __launch_bounds__(kSortThreads)
-sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin,
-                    uint32_t* __restrict__ kout, uint32_t* __restrict__ vout, uint32_t n_host,
-                    const unsigned int* __restrict__ n_dev, int shift, const uint32_t* __restrict__ counts,
-                    uint32_t n_tiles, const uint32_t* __restrict__ totals) {
+sort_pass_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ vin, uint32_t* __restrict__ kout,
+                 uint32_t* __restrict__ vout, uint32_t n_host, const unsigned int* __restrict__ n_dev, int pass,
+                 uint32_t* __restrict__ ctl, uint32_t* __restrict__ tile_state, uint32_t n_tiles, DevStatus* st) {
     __shared__ uint32_t digit_base[kRadix];
     __shared__ uint32_t warp_hist[kSortThreads / 32][kRadix];
     __shared__ uint32_t sm[8];
+    __shared__ uint32_t s_tile;
+    __shared__ int s_gave_up;
     const uint32_t n = n_dev ? tmin<uint32_t>(*n_dev, n_host) : n_host;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    {
-        uint32_t tot;
-        uint32_t ex = block_exclusive_scan_256(totals[tid], sm, &tot);
-        digit_base[tid] = ex + counts[(size_t)tid * n_tiles + blockIdx.x];
-#pragma unroll
-        for (int i = 0; i < kSortThreads / 32; ++i) warp_hist[i][tid] = 0;
+    const int shift = pass * kRadixBits;
+    if (tid == 0) {
+        s_tile = atomicAdd(&ctl[kMaxSortPasses * kRadix + pass], 1u);
+        s_gave_up = 0;
     }
+    uint32_t tot;
+    const uint32_t global_base = block_exclusive_scan_256(ctl[pass * kRadix + tid], sm, &tot);   // has a barrier
+#pragma unroll
+    for (int i = 0; i < kSortThreads / 32; ++i) warp_hist[i][tid] = 0;
     __syncthreads();
-    const uint32_t chunk = blockIdx.x * kSortTile + w * (32 * kSortItems);
+    const uint32_t tile = s_tile;
+    if (tile >= n_tiles) return;
+    const uint32_t chunk = tile * kSortTile + w * (32 * kSortItems);
     uint32_t key[kSortItems], rank[kSortItems];
     const unsigned lt = (1u << lane) - 1u;
 #pragma unroll
@@ -87,15 +98,59 @@ sort_scatter_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict
     }
     __syncthreads();
     {
+        // thread d: this tile's count of digit d; the per-warp counters become offsets inside the tile
         uint32_t run = 0;
 #pragma unroll
         for (int i = 0; i < kSortThreads / 32; ++i) {
-            uint32_t t = warp_hist[i][tid];
+            const uint32_t t = warp_hist[i][tid];
             warp_hist[i][tid] = run;
             run += t;
         }
+        const volatile uint32_t* tile_state_v = tile_state;
+        volatile uint32_t* mine = tile_state + ((size_t)pass * n_tiles + tile) * kRadix + tid;
+        uint32_t before = 0;
+        if (tile == 0) {
+            *mine = kFlagTotal | run;
+        } else {
+            *mine = kFlagCount | run;
+            // Look back over earlier tiles until one of them shows a running total.  The words of
+            // kLookbackWindow tiles are requested together; one that is not published yet is polled.
+            bool done = false;
+            for (uint32_t t = tile; t > 0 && !done; t = t > kLookbackWindow ? t - kLookbackWindow : 0) {
+                uint32_t word[kLookbackWindow];
+#pragma unroll
+                for (int k = 0; k < kLookbackWindow; ++k) {
+                    word[k] = 0u;
+                    if (t > (uint32_t)k) word[k] = *(tile_state_v + ((size_t)pass * n_tiles + (t - 1 - k)) * kRadix + tid);
+                }
+#pragma unroll
+                for (int k = 0; k < kLookbackWindow; ++k) {
+                    if (done || t <= (uint32_t)k) continue;
+                    uint32_t wv = word[k];
+                    int spins = 0;
+                    while ((wv & ~kValueMask) == 0u && spins < kLookbackSpins) {
+                        __nanosleep(32);
+                        wv = *(tile_state_v + ((size_t)pass * n_tiles + (t - 1 - k)) * kRadix + tid);
+                        ++spins;
+                    }
+                    if ((wv & ~kValueMask) == 0u) {
+                        s_gave_up = 1;
+                        done = true;
+                    } else {
+                        before += wv & kValueMask;
+                        if (wv & kFlagTotal) done = true;
+                    }
+                }
+            }
+            *mine = kFlagTotal | (before + run);
+        }
+        digit_base[tid] = global_base + before;
     }
     __syncthreads();
+    if (s_gave_up) {                                    // nothing is written; the call's results are void
+        if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
+        return;
+    }
 #pragma unroll
     for (int it = 0; it < kSortItems; ++it) {
         const uint32_t idx = chunk + it * 32 + lane;
@@ -118,16 +173,17 @@ int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bi
     }
     int which = start;
     if (bits < 1) bits = 1;
-    for (int shift = 0; shift < bits; shift += kRadixBits) {
-        PS_LAUNCH(ps, sort_hist_kernel, n_tiles, kSortThreads, stream, kin, n, n_dev, shift, ps->hist, n_tiles,
-                  shift == 0 ? zero_me : nullptr);
-        PS_LAUNCH(ps, sort_scan_kernel, kRadix, 256, stream, ps->hist, n_tiles, ps->totals);
-        if (iota_vals && shift == 0)
-            PS_LAUNCH(ps, sort_scatter_kernel<true>, n_tiles, kSortThreads, stream, kin, vin, kout, vout, n, n_dev,
-                      shift, ps->hist, n_tiles, ps->totals);
+    const int n_passes = (bits + kRadixBits - 1) / kRadixBits;
+    cudaMemsetAsync(ps->sort_ctl, 0, kSortCtlWords * sizeof(uint32_t), stream);
+    PS_LAUNCH(ps, sort_hist_kernel, n_tiles, kSortThreads, stream, kin, n, n_dev, n_passes, ps->sort_ctl,
+              ps->tile_state, n_tiles, zero_me);
+    for (int pass = 0; pass < n_passes; ++pass) {
+        if (iota_vals && pass == 0)
+            PS_LAUNCH(ps, sort_pass_kernel<true>, n_tiles, kSortThreads, stream, kin, vin, kout, vout, n, n_dev, pass,
+                      ps->sort_ctl, ps->tile_state, n_tiles, ps->status);
         else
-            PS_LAUNCH(ps, sort_scatter_kernel<false>, n_tiles, kSortThreads, stream, kin, vin, kout, vout, n,
-                      n_dev, shift, ps->hist, n_tiles, ps->totals);
+            PS_LAUNCH(ps, sort_pass_kernel<false>, n_tiles, kSortThreads, stream, kin, vin, kout, vout, n, n_dev, pass,
+                      ps->sort_ctl, ps->tile_state, n_tiles, ps->status);
         uint32_t* t;
         t = kin; kin = kout; kout = t;
         t = vin; vin = vout; vout = t;

@@ -53,8 +53,7 @@ __global__ void __launch_bounds__(256)
 mf_step_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, const float* __restrict__ cv,
                uint64_t n, uint64_t col_base, float lr, float lam, const float4* __restrict__ store,
                const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t L4,
-               uint32_t* __restrict__ keys_out, float4* __restrict__ upd, double* __restrict__ loss_partial,
-               DevStatus* st, unsigned int epoch) {
+               float4* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -65,11 +64,7 @@ mf_step_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj,
         const float v = cv[t];
         const uint64_t kw = i, kh = col_base + j;
         if (kw >= col_base || kh >= K) {
-            if (lane == 0) {
-                latch_error(st, epoch, PS_ERR_KEY_RANGE);
-                keys_out[2 * t] = (uint32_t)K;
-                keys_out[2 * t + 1] = (uint32_t)K;
-            }
+            if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
             continue;
         }
         const float4* W = store + phys_row(table[kw], S) * L4;
@@ -122,12 +117,20 @@ mf_step_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj,
         } else {
             for (uint32_t f = lane; f < L4; f += 32) emit(f, W[f], H[f]);
         }
-        if (lane == 0) {
-            keys_out[2 * t] = (uint32_t)kw;
-            keys_out[2 * t + 1] = (uint32_t)kh;
-        }
     }
     block_loss_out(loss, loss_partial);
+}
+
+// keys of the occurrences of a batch of cells: [2t] = row factor, [2t+1] = column factor
+__global__ void __launch_bounds__(256)
+mf_keys_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, uint64_t n, uint64_t col_base,
+               uint64_t K, uint32_t* __restrict__ keys_out, DevStatus* st, unsigned int epoch) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n) return;
+    const uint64_t kw = ci[t], kh = col_base + cj[t];
+    const bool bad = kw >= col_base || kh >= K;
+    if (bad) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+    reinterpret_cast<uint2*>(keys_out)[t] = bad ? make_uint2((uint32_t)K, (uint32_t)K) : make_uint2((uint32_t)kw, (uint32_t)kh);
 }
 
 uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
@@ -135,7 +138,7 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
     const uint32_t L4 = ps->cfg.row_len / 4;
     const uint32_t grid = step_grid(ps, n);
 #define MF_ARGS d_i, d_j, d_v, n, col_key_base, lr, lambda, (const float4*)ps->store, ps->table,                 \
-                ps->cfg.slots_per_part, ps->cfg.num_keys, L4, ps->keysA, (float4*)ps->upd, ps->loss_partial,   \
+                ps->cfg.slots_per_part, ps->cfg.num_keys, L4, (float4*)ps->upd, ps->loss_partial,              \
                 ps->status, ps->epoch
     if (L4 <= 32) PS_LAUNCH(ps, mf_step_kernel<1>, grid, 256, s, MF_ARGS);
     else if (L4 <= 64) PS_LAUNCH(ps, mf_step_kernel<2>, grid, 256, s, MF_ARGS);
@@ -143,6 +146,12 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
     else PS_LAUNCH(ps, mf_step_kernel<0>, grid, 256, s, MF_ARGS);
 #undef MF_ARGS
     return grid;
+}
+
+void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint64_t n, uint64_t col_key_base,
+                    cudaStream_t s) {
+    PS_LAUNCH(ps, mf_keys_kernel, div_up_u32(n, 256), 256, s, d_i, d_j, n, col_key_base, ps->cfg.num_keys, ps->keysA,
+              ps->status, ps->epoch);
 }
 
 // ------------------------------------------------------------- ComplEx ----
@@ -161,8 +170,8 @@ __global__ void __launch_bounds__(256)
 kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                 const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
                 uint32_t n_neg, uint64_t rel_base, uint32_t d, float lr, float eps, const float* __restrict__ store,
-                const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t* __restrict__ keys_out,
-                float* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+                const uint2* __restrict__ table, uint64_t S, uint64_t K, float* __restrict__ upd,
+                double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -186,10 +195,8 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
                 if (lane >= 3) side = neg_side[t * n_neg + (lane - 3)] != 0;
             }
         }
-        uint32_t* kout = keys_out + t * n_slots;
         if (__any_sync(full, bad)) {
             if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
-            if (lane < n_slots) kout[lane] = (uint32_t)K;
             continue;
         }
         uint64_t off = 0;
@@ -301,9 +308,35 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
                 Uu[3 * d + c] = g2_im;
             }
         }
-        if (lane < n_slots) kout[lane] = rep == lane ? (uint32_t)key : (uint32_t)K;
     }
     block_loss_out(loss, loss_partial);
+}
+
+// Keys of the occurrence slots of each data point; a slot that repeats an earlier slot's key, and every
+// slot of a data point with an index out of range, gets the "no key" mark K.
+__global__ void __launch_bounds__(256)
+kge_keys_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
+                const uint32_t* __restrict__ neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_base, uint64_t K,
+                uint32_t* __restrict__ keys_out, DevStatus* st, unsigned int epoch) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n) return;
+    const int n_slots = 3 + (int)n_neg;
+    uint64_t key[32];
+    key[0] = ts[t];
+    key[1] = rel_base + tr[t];
+    key[2] = to[t];
+    bool bad = key[0] >= rel_base || key[2] >= rel_base || key[1] >= K;
+    for (int q = 0; q < (int)n_neg; ++q) {
+        key[3 + q] = neg_ent[t * n_neg + q];
+        bad |= key[3 + q] >= rel_base;
+    }
+    if (bad) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+    uint32_t* kout = keys_out + t * n_slots;
+    for (int u = 0; u < n_slots; ++u) {
+        bool first = true;
+        for (int z = 0; z < u; ++z) first &= key[z] != key[u];
+        kout[u] = (first && !bad) ? (uint32_t)key[u] : (uint32_t)K;
+    }
 }
 
 uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
@@ -311,9 +344,15 @@ uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r,
                          uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s) {
     const uint32_t grid = step_grid(ps, n);
     PS_LAUNCH(ps, kge_step_kernel, grid, 256, s, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim,
-              lr, eps, (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->keysA,
-              ps->upd, ps->loss_partial, ps->status, ps->epoch);
+              lr, eps, (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->upd,
+              ps->loss_partial, ps->status, ps->epoch);
     return grid;
+}
+
+void launch_keys_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                     const uint32_t* d_neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_key_base, cudaStream_t s) {
+    PS_LAUNCH(ps, kge_keys_kernel, div_up_u32(n, 256), 256, s, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base,
+              ps->cfg.num_keys, ps->keysA, ps->status, ps->epoch);
 }
 
 // ---------------------------------------------------------------- SGNS ----
@@ -337,8 +376,8 @@ __global__ void __launch_bounds__(256)
 sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64_t first_pos, uint64_t n_centers,
                  uint64_t T, uint32_t window, const uint32_t* __restrict__ negs, uint32_t n_neg, uint64_t out_base,
                  float lr, const float4* __restrict__ store, const uint2* __restrict__ table, uint64_t S, uint64_t K,
-                 uint32_t L4, uint32_t* __restrict__ keys_out, float4* __restrict__ upd,
-                 double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+                 uint32_t L4, float4* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st,
+                 unsigned int epoch) {
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -351,12 +390,8 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
         const uint64_t lo = p >= window ? p - window : 0;
         const uint64_t hi = p + window < T ? p + window : T - 1;
         const uint64_t z0 = sgns_pairs_before(p, T, window) - pairs0;
-        uint32_t* kout = keys_out + cidx * slots;
         float4* U = upd + cidx * slots * L4;
         const uint32_t wtok = tokens[p - tok_first];
-        // mark every slot unused first; used ones are overwritten below
-        for (uint64_t x = lane; x < slots; x += 32) kout[x] = (uint32_t)K;
-        __syncwarp();
         if (wtok >= out_base) {
             if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
             continue;
@@ -401,7 +436,6 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
                     if (f < L4)
                         U[slot * L4 + f] = make_float4(sc * v[c].x, sc * v[c].y, sc * v[c].z, sc * v[c].w);
                 }
-                if (lane == 0) kout[slot] = (uint32_t)ku;
             }
             ++j;
         }
@@ -411,10 +445,47 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
             const uint32_t f = lane + 32 * c;
             if (f < L4) U[f] = dv[c];
         }
-        if (lane == 0) kout[0] = wtok;
         loss += (double)loss_c;
     }
     block_loss_out(loss, loss_partial);
+}
+
+// Keys of the occurrence slots of each center: slot 0 the center's input vector, then per context
+// 1 + n_neg output vectors; slots of contexts cut off at the stream's ends get the "no key" mark K.
+__global__ void __launch_bounds__(256)
+sgns_keys_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64_t first_pos, uint64_t n_centers,
+                 uint64_t T, uint32_t window, const uint32_t* __restrict__ negs, uint32_t n_neg, uint64_t out_base,
+                 uint64_t K, uint32_t* __restrict__ keys_out, DevStatus* st, unsigned int epoch) {
+    const uint32_t per_ctx = 1 + n_neg;
+    const uint64_t slots = 1 + (uint64_t)2 * window * per_ctx;
+    const uint64_t x = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= n_centers * slots) return;
+    const uint64_t cidx = x / slots, slot = x % slots;
+    const uint64_t p = first_pos + cidx;
+    uint64_t key = K;
+    bool bad = false;
+    if (slot == 0) {
+        const uint32_t w = tokens[p - tok_first];
+        bad = w >= out_base;
+        key = w;
+    } else {
+        const uint64_t lo = p >= window ? p - window : 0;
+        const uint64_t hi = p + window < T ? p + window : T - 1;
+        const uint64_t j = (slot - 1) / per_ctx, i = (slot - 1) % per_ctx;
+        const uint64_t n_left = p - lo;
+        const uint64_t q = j < n_left ? lo + j : lo + j + 1;        // skip the center itself
+        if (q <= hi) {
+            const uint64_t z = sgns_pairs_before(p, T, window) - sgns_pairs_before(first_pos, T, window) + j;
+            const uint32_t word = i == 0 ? tokens[q - tok_first] : negs[z * n_neg + (i - 1)];
+            key = out_base + word;
+            bad = key >= K;
+        }
+    }
+    if (bad) {
+        latch_error(st, epoch, PS_ERR_KEY_RANGE);
+        key = K;
+    }
+    keys_out[x] = (uint32_t)key;
 }
 
 uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
@@ -423,7 +494,7 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
     const uint32_t L4 = ps->cfg.row_len / 4;
     const uint32_t grid = step_grid(ps, n_centers);
 #define SG_ARGS d_tokens, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, lr,   \
-                (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4, ps->keysA,   \
+                (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4,              \
                 (float4*)ps->upd, ps->loss_partial, ps->status, ps->epoch
     if (L4 <= 32) PS_LAUNCH(ps, sgns_step_kernel<1>, grid, 256, s, SG_ARGS);
     else if (L4 <= 64) PS_LAUNCH(ps, sgns_step_kernel<2>, grid, 256, s, SG_ARGS);
@@ -431,6 +502,14 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
     else PS_LAUNCH(ps, sgns_step_kernel<4>, grid, 256, s, SG_ARGS);
 #undef SG_ARGS
     return grid;
+}
+
+void launch_keys_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
+                      uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs, uint32_t n_neg,
+                      uint64_t out_key_base, cudaStream_t s) {
+    const uint64_t total = n_centers * (1 + (uint64_t)2 * window * (1 + n_neg));
+    PS_LAUNCH(ps, sgns_keys_kernel, div_up_u32(total, 256), 256, s, d_tokens, tok_first, first_pos, n_centers,
+              corpus_len, window, d_negs, n_neg, out_key_base, ps->cfg.num_keys, ps->keysA, ps->status, ps->epoch);
 }
 
 }  // namespace psb
