@@ -219,6 +219,16 @@ ps_status_t ps_export_freelists(ps_store_t* ps, uint32_t* h_stacks, uint64_t* h_
 /* Waits for `stream`; returns and clears the first error latched on the device. */
 ps_status_t ps_sync(ps_store_t* ps, void* stream);
 
+/* Latency hiding across steps, after the paper's pre-localization (Section 2.2,
+ * "latency hiding": prepare the next data point's parameters while the current
+ * one is processed).  Off (default): a ps_step_* call reads its batch arrays
+ * only after everything already enqueued on `stream`.  On: the keys of the
+ * batch are extracted and sorted on an internal stream as soon as the call is
+ * made, beside the previous step's kernels, so the batch arrays must be
+ * complete at call time (no writes to them still pending on `stream`).
+ * Results are identical in both modes. */
+ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
+
 /* Number of kernels this handle has launched so far. */
 uint64_t ps_launch_count(const ps_store_t* ps);
 

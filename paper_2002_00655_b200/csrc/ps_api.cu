@@ -27,17 +27,19 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     const size_t reduce_tiles = (mk + kReduceTile - 1) / kReduceTile;
     const size_t row_bytes = (size_t)cfg.row_len * 4;
     l.status = take(sizeof(DevStatus));
-    l.keysA = take(mk * 4);
-    l.keysB = take(mk * 4);
-    l.valsA = take(mk * 4);
-    l.valsB = take(mk * 4);
-    l.tile_state = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
-    l.sort_ctl = take((size_t)kSortCtlWords * 4);
+    for (int b = 0; b < 2; ++b) {
+        l.keysA[b] = take(mk * 4);
+        l.keysB[b] = take(mk * 4);
+        l.valsA[b] = take(mk * 4);
+        l.valsB[b] = take(mk * 4);
+        l.tile_state[b] = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
+        l.sort_ctl[b] = take((size_t)kSortCtlWords * 4);
+        l.starters[b] = take(reduce_tiles * 4);
+        l.starter_count[b] = take(4);
+    }
     l.scan_sums = take(((mk + 255) / 256) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
-    l.starters = take(reduce_tiles * 4);
-    l.starter_count = take(4);
     l.loss_partial = take(kMaxLossBlocks * 8);
     l.staging = take(mk * 8 + 256);
     l.total = off;
@@ -76,6 +78,8 @@ void prof_after(ps_store* ps, cudaStream_t s) {
     p->open = false;
 }
 
+static ps_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? PS_OK : PS_ERR_CUDA; }
+
 static int bits_for(uint64_t max_value) {
     int b = 0;
     while (b < 32 && (max_value >> b) != 0) ++b;
@@ -94,19 +98,39 @@ static ps_status_t check_cfg(const ps_config_t* cfg) {
     return PS_OK;
 }
 
-static ps_status_t cuda_ok(cudaError_t e) { return e == cudaSuccess ? PS_OK : PS_ERR_CUDA; }
 
 // Errors raised by a launch itself (bad configuration) show up here; errors inside kernels
 // are reported through the device status word.
 static ps_status_t after_launch() { return cuda_ok(cudaGetLastError()); }
 
+
+// Calls that sort alternate between the handle's two sets of sort buffers.
+static SortSet* next_set(ps_store* ps) {
+    ps->cur_set ^= 1;
+    SortSet* ss = &ps->sets[ps->cur_set];
+    ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
+    ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl;
+    ps->starters = ss->starters; ps->starter_count = ss->starter_count;
+    return ss;
+}
+
 // The keys of a step's occurrences depend on the batch alone, so their extraction and sort run on the
-// handle's side stream while the gradient kernel runs on the caller's; both meet before the reduction.
-static bool fork_side(ps_store* ps, cudaStream_t s) {
+// handle's side stream while gradient kernels run on the caller's; both meet before the reduction.
+// Ordered mode: the side stream starts after everything already enqueued on the caller's stream.
+// Pipelined mode: it starts as soon as the buffer set's previous user is done, i.e. beside the previous
+// step's kernels; the batch arrays must then be complete when the call is made.
+static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
+    if (ps->pipelined) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
     return cudaEventRecord(ps->ev_join, ps->side) == cudaSuccess && cudaStreamWaitEvent(s, ps->ev_join, 0) == cudaSuccess;
+}
+// after the last kernel of a call that used the set
+static ps_status_t release_set(SortSet* ss, cudaStream_t s) {
+    ss->used = true;
+    if (cudaEventRecord(ss->ev_free, s) != cudaSuccess) return PS_ERR_CUDA;
+    return cuda_ok(cudaGetLastError());
 }
 
 static void next_epoch(ps_store* ps) {
@@ -158,17 +182,23 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->ws_bytes = workspace_bytes;
     const WsLayout l = ws_layout(*cfg, max_batch_keys);
     ps->status = (DevStatus*)(ps->ws + l.status);
-    ps->keysA = (uint32_t*)(ps->ws + l.keysA);
-    ps->keysB = (uint32_t*)(ps->ws + l.keysB);
-    ps->valsA = (uint32_t*)(ps->ws + l.valsA);
-    ps->valsB = (uint32_t*)(ps->ws + l.valsB);
-    ps->tile_state = (uint32_t*)(ps->ws + l.tile_state);
-    ps->sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl);
+    for (int b = 0; b < 2; ++b) {
+        SortSet& ss = ps->sets[b];
+        ss.keysA = (uint32_t*)(ps->ws + l.keysA[b]);
+        ss.keysB = (uint32_t*)(ps->ws + l.keysB[b]);
+        ss.valsA = (uint32_t*)(ps->ws + l.valsA[b]);
+        ss.valsB = (uint32_t*)(ps->ws + l.valsB[b]);
+        ss.tile_state = (uint32_t*)(ps->ws + l.tile_state[b]);
+        ss.sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl[b]);
+        ss.starters = (uint32_t*)(ps->ws + l.starters[b]);
+        ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
+        ss.used = false;
+    }
+    ps->cur_set = 1;
+    next_set(ps);
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
-    ps->starters = (uint32_t*)(ps->ws + l.starters);
-    ps->starter_count = (unsigned int*)(ps->ws + l.starter_count);
     ps->loss_partial = (double*)(ps->ws + l.loss_partial);
     ps->staging = ps->ws + l.staging;
     int sms = 0;
@@ -186,7 +216,9 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
     if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->sets[0].ev_free, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->sets[1].ev_free, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
     }
@@ -201,6 +233,8 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
+    cudaEventDestroy(ps->sets[0].ev_free);
+    cudaEventDestroy(ps->sets[1].ev_free);
     cudaStreamDestroy(ps->side);
     delete ps;
     return PS_OK;
@@ -238,9 +272,10 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
     if (n == 0) return PS_OK;
     if (!d_keys || !d_updates) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    SortSet* ss = next_set(ps);
     launch_prepare_keys(ps, d_keys, n, s);
     run_push_pipeline(ps, (uint32_t)n, d_updates, nullptr, 0, s);
-    return after_launch();
+    return release_set(ss, s);
 }
 
 ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n, void* stream) {
@@ -249,9 +284,10 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     if (n == 0) return PS_OK;
     if (!d_keys) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    SortSet* ss = next_set(ps);
     launch_prepare_keys(ps, d_keys, n, s);
     run_localize(ps, worker, (uint32_t)n, s);
-    return after_launch();
+    return release_set(ss, s);
 }
 
 ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
@@ -261,13 +297,14 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (!d_i || !d_j || !d_v) return PS_ERR_INVALID_ARG;
     if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
-    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    SortSet* ss = next_set(ps);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_mf(ps, d_i, d_j, n, col_key_base, ps->side);
     const int which = run_push_sort(ps, (uint32_t)(2 * n), ps->side);
     const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)(2 * n), which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
-    return after_launch();
+    return release_set(ss, s);
 }
 
 ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
@@ -282,14 +319,15 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     if ((3 + (uint64_t)n_neg) * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (rel_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
     const uint32_t occ = (uint32_t)((3 + (uint64_t)n_neg) * n);
-    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    SortSet* ss = next_set(ps);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_kge(ps, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base, ps->side);
     const int which = run_push_sort(ps, occ, ps->side);
     const uint32_t lb =
         launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex, lr, eps, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
-    return after_launch();
+    return release_set(ss, s);
 }
 
 static ps_status_t sgns_checks(ps_store_t* ps, uint64_t first_pos, uint64_t n_centers, uint64_t corpus_len,
@@ -311,14 +349,15 @@ ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t firs
     uint64_t occ;
     const ps_status_t c = sgns_checks(ps, first_pos, n_centers, corpus_len, window, n_neg, out_key_base, &occ);
     if (c != PS_OK) return c;
-    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    SortSet* ss = next_set(ps);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, ps->side);
     const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
     const uint32_t lb = launch_step_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
-    return after_launch();
+    return release_set(ss, s);
 }
 
 // ---- host-batch variants ----
@@ -345,7 +384,10 @@ ps_status_t ps_step_mf_host(ps_store_t* ps, const uint32_t* h_i, const uint32_t*
         cudaMemcpyAsync(d_j, h_j, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
         cudaMemcpyAsync(d_v, h_v, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return PS_ERR_CUDA;
+    const bool was = ps->pipelined;         // the batch arrives on the caller's stream: order the side stream after it
+    ps->pipelined = false;
     const ps_status_t c = ps_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, d_loss_accum, stream);
+    ps->pipelined = was;
     if (c != PS_OK) return c;
     return finish_host_step(d_loss_accum, h_loss, s);
 }
@@ -371,8 +413,11 @@ ps_status_t ps_step_kge_host(ps_store_t* ps, const uint32_t* h_s, const uint32_t
     if (n_neg && (cudaMemcpyAsync(d_ne, h_neg_ent, n * n_neg * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
                   cudaMemcpyAsync(d_ns, h_neg_side, n * n_neg, cudaMemcpyHostToDevice, s) != cudaSuccess))
         return PS_ERR_CUDA;
+    const bool was = ps->pipelined;         // the batch arrives on the caller's stream: order the side stream after it
+    ps->pipelined = false;
     const ps_status_t c = ps_step_kge(ps, d_s, d_r, d_o, d_ne, d_ns, n, n_neg, rel_key_base, dim_complex, lr, eps,
                                       d_loss_accum, stream);
+    ps->pipelined = was;
     if (c != PS_OK) return c;
     return finish_host_step(d_loss_accum, h_loss, s);
 }
@@ -400,7 +445,10 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     if (cudaMemcpyAsync(d_tok, h_tokens, tok_count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return PS_ERR_CUDA;
     if (n_negs && cudaMemcpyAsync(d_negs, h_negs, n_negs * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return PS_ERR_CUDA;
-    if (!fork_side(ps, s)) return PS_ERR_CUDA;
+    SortSet* ss = next_set(ps);
+    // the batch was just copied on the caller's stream: the side stream has to wait for that
+    if (cudaEventRecord(ps->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) != cudaSuccess)
+        return PS_ERR_CUDA;
     launch_keys_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base,
                      ps->side);
     const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
@@ -408,7 +456,7 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
                                          out_key_base, lr, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
-    c = after_launch();
+    c = release_set(ss, s);
     if (c != PS_OK) return c;
     return finish_host_step(d_loss_accum, h_loss, s);
 }
@@ -470,6 +518,12 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream) {
     if (cudaMemcpy(&code, &ps->status->sticky, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
     if (code != 0 && cudaMemset(&ps->status->sticky, 0, 4) != cudaSuccess) return PS_ERR_CUDA;
     return (ps_status_t)code;
+}
+
+ps_status_t ps_set_pipelining(ps_store_t* ps, int on) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    ps->pipelined = on != 0;
+    return PS_OK;
 }
 
 uint64_t ps_launch_count(const ps_store_t* ps) { return ps ? ps->launches : 0; }

@@ -24,13 +24,25 @@ constexpr int kMaxLossBlocks = 4096;
 // epoch, so no kernel has to clear anything before a call starts.
 struct DevStatus {
     unsigned int sticky;            // first error code since the last ps_sync
-    unsigned int call_err_epoch;    // epoch of the last call that failed on the device
+    unsigned int call_err_epoch[2]; // epoch of the last even / odd call that failed on the device (two calls
+                                    // of one handle can be in flight: one's sort beside the other's kernels)
     unsigned int moved_total;       // localize: number of keys that move in the current call
-    unsigned int pad;
     unsigned long long rows_moved;  // rows relocated by all successful localize calls so far
 };
 
 struct Profile;
+
+// One of the two sets of buffers the key sort and the segment bookkeeping work in.  Calls alternate
+// between the sets so that the sort of one step can run while the previous step is still reducing.
+struct SortSet {
+    uint32_t *keysA, *keysB, *valsA, *valsB;
+    uint32_t* tile_state;
+    uint32_t* sort_ctl;
+    uint32_t* starters;
+    unsigned int* starter_count;
+    cudaEvent_t ev_free;            // recorded after the last kernel that used the set
+    bool used;
+};
 
 }  // namespace psb
 
@@ -65,13 +77,16 @@ struct ps_store {
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
     cudaStream_t side;              // key extraction and sort of a step run here, beside the gradient kernel
     cudaEvent_t ev_fork, ev_join;
+    psb::SortSet sets[2];           // keysA .. starter_count above always point into sets[cur_set]
+    int cur_set;
+    bool pipelined;                 // see ps_set_pipelining
 };
 
 namespace psb {
 
 struct WsLayout {
-    size_t status, keysA, keysB, valsA, valsB, tile_state, sort_ctl, scan_sums, upd, carry, starters, starter_count,
-        loss_partial, staging, total;
+    size_t status, keysA[2], keysB[2], valsA[2], valsB[2], tile_state[2], sort_ctl[2], scan_sums, upd, carry,
+        starters[2], starter_count[2], loss_partial, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
 
@@ -146,10 +161,10 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
 #ifdef __CUDACC__
 __device__ __forceinline__ void latch_error(DevStatus* st, unsigned int epoch, unsigned int code) {
     atomicCAS(&st->sticky, 0u, code);
-    atomicExch(&st->call_err_epoch, epoch);
+    atomicExch(&st->call_err_epoch[epoch & 1u], epoch);
 }
 __device__ __forceinline__ bool call_failed(const DevStatus* st, unsigned int epoch) {
-    return *((const volatile unsigned int*)&st->call_err_epoch) == epoch;
+    return *((const volatile unsigned int*)&st->call_err_epoch[epoch & 1u]) == epoch;
 }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -166,7 +166,10 @@ void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint
 // rounding noise of g into a visible change of the parameter; fp64 sums keep
 // that noise far below the fp32 resolution of the result.  The final AdaGrad
 // expression is evaluated in fp32 on the rounded gradient.
-__global__ void __launch_bounds__(256)
+// kMaxNeg bounds n_neg at compile time so that a data point's values live in registers: for every block
+// of 32 complex dimensions the Re and Im of all its rows are requested together, before any is used.
+template <int kMaxNeg>
+__global__ void __launch_bounds__(256, kMaxNeg <= 10 ? 2 : 1)
 kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                 const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
                 uint32_t n_neg, uint64_t rel_base, uint32_t d, float lr, float eps, const float* __restrict__ store,
@@ -180,7 +183,7 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
     const unsigned full = 0xffffffffu;
     double loss = 0;
     for (uint64_t t = warp; t < n; t += n_warps) {
-        // ---- keys, validity, row offsets, first-slot-with-same-key ----
+        // ---- keys, validity, row offsets, first-slot-with-same-key (lane u holds slot u) ----
         uint64_t key = K;
         int side = 0;
         bool bad = false;
@@ -209,24 +212,45 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
         const float* Srow = store + __shfl_sync(full, off, 0);
         const float* Rrow = store + __shfl_sync(full, off, 1);
         const float* Orow = store + __shfl_sync(full, off, 2);
+        const float* Nrow[kMaxNeg];
+#pragma unroll
+        for (int q = 0; q < kMaxNeg; ++q) Nrow[q] = store + __shfl_sync(full, off, (3 + q) & 31);
+        // bit q: negative q stands in the subject's place / is the first slot with its key
+        const unsigned subj_mask = __ballot_sync(full, lane >= 3 && lane < n_slots && side == 0) >> 3;
+        const unsigned nrep_mask = __ballot_sync(full, lane >= 3 && lane < n_slots && rep == lane) >> 3;
 
-        // ---- pass A: the 1 + n_neg scores; lane q keeps triple q's score ----
+        // ---- pass A: partial scores of the 1 + n_neg triples over this lane's dimensions ----
+        double part[kMaxNeg + 1];
+#pragma unroll
+        for (int q = 0; q <= kMaxNeg; ++q) part[q] = 0.0;
+        for (uint32_t c = lane; c < d; c += 32) {
+            const float a_f = Srow[c], b_f = Srow[d + c], cr_f = Rrow[c], ci_f = Rrow[d + c];
+            const float e_f = Orow[c], f_f = Orow[d + c];
+            float na_f[kMaxNeg], nb_f[kMaxNeg];
+#pragma unroll
+            for (int q = 0; q < kMaxNeg; ++q) {
+                na_f[q] = q < (int)n_neg ? Nrow[q][c] : 0.f;
+                nb_f[q] = q < (int)n_neg ? Nrow[q][d + c] : 0.f;
+            }
+            const double a = a_f, b = b_f, cr = cr_f, ci = ci_f, e = e_f, f = f_f;
+            part[0] += cr * (a * e + b * f) + ci * (a * f - b * e);
+            // (n, r, o): cr (na e + nb f) + ci (na f - nb e);   (s, r, n): cr (a na + b nb) + ci (a nb - b na)
+            const double re_o = cr * e + ci * f, im_o = cr * f - ci * e;        // multiplies (na, nb) for side 0
+            const double re_s = cr * a - ci * b, im_s = cr * b + ci * a;        // multiplies (na, nb) for side 1
+#pragma unroll
+            for (int q = 0; q < kMaxNeg; ++q) {
+                const double na = na_f[q], nb = nb_f[q];
+                part[q + 1] += ((subj_mask >> q) & 1u) ? (na * re_o + nb * im_o) : (na * re_s + nb * im_s);
+            }
+        }
+        // lane q keeps triple q's score
         double phi_mine = 0;
-        for (int q = 0; q <= (int)n_neg; ++q) {
-            const float* Sq = Srow;
-            const float* Oq = Orow;
-            if (q > 0) {
-                const int sd = __shfl_sync(full, side, 2 + q);
-                const float* Nq = store + __shfl_sync(full, off, 2 + q);
-                if (sd == 0) Sq = Nq; else Oq = Nq;
+#pragma unroll
+        for (int q = 0; q <= kMaxNeg; ++q) {
+            if (q <= (int)n_neg) {
+                const double phi = warp_sum_d(part[q]);
+                if (lane == q) phi_mine = phi;
             }
-            double part = 0;
-            for (uint32_t c = lane; c < d; c += 32) {
-                const double a = Sq[c], b = Sq[d + c], cr = Rrow[c], ci = Rrow[d + c], e = Oq[c], f = Oq[d + c];
-                part += cr * (a * e + b * f) + ci * (a * f - b * e);
-            }
-            const double phi = warp_sum_d(part);
-            if (lane == q) phi_mine = phi;
         }
         // lane q: loss term and d loss / d phi of triple q (label +1 for the positive, -1 for negatives)
         double coef = 0, loss_q = 0;
@@ -242,12 +266,12 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
         // With side 1 it stands in the object's place: coef * dphi/dO(s, r).  Summed over the
         // negatives whose key's first slot is this lane.
         double wS = 0, wO = 0;
-        for (int q = 1; q <= (int)n_neg; ++q) {
-            const int rq = __shfl_sync(full, rep, 2 + q);
-            const int sd = __shfl_sync(full, side, 2 + q);
-            const double cf = __shfl_sync(full, coef, q);
-            if (rq == lane) {
-                if (sd == 0) wS += cf; else wO += cf;
+#pragma unroll
+        for (int q = 0; q < kMaxNeg; ++q) {
+            const int rq = __shfl_sync(full, rep, (3 + q) & 31);
+            const double cfq = __shfl_sync(full, coef, (q + 1) & 31);
+            if (q < (int)n_neg && rq == lane) {
+                if ((subj_mask >> q) & 1u) wS += cfq; else wO += cfq;
             }
         }
         const double cf0 = __shfl_sync(full, coef, 0);
@@ -257,55 +281,73 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
 
         // ---- pass B: gradients per block of 32 complex dimensions, AdaGrad, update rows ----
         float* U = upd + (t * n_slots) * L;
+        // -lr g / (sqrt(G + g^2) + eps) with the hardware reciprocal square root and reciprocal (each within
+        // 2 ulp, far inside the fp32 tolerance of the result); x = 0 is kept away from 0 * inf
+        auto adagrad_step = [&](float g, float x) {
+            const float root = x > 0.f ? x * rsqrtf(x) : 0.f;
+            return __fdividef(-lr * g, root + eps);
+        };
+        auto adagrad_out = [&](float* Uu, uint32_t c, double gd_re, double gd_im, float G_re, float G_im) {
+            const float g_re = (float)gd_re, g_im = (float)gd_im;
+            const float g2_re = g_re * g_re, g2_im = g_im * g_im;
+            Uu[c] = adagrad_step(g_re, G_re + g2_re);
+            Uu[d + c] = adagrad_step(g_im, G_im + g2_im);
+            Uu[2 * d + c] = g2_re;
+            Uu[3 * d + c] = g2_im;
+        };
         for (uint32_t c0 = 0; c0 < d; c0 += 32) {
             const uint32_t c = c0 + lane;
             const bool act = c < d;
-            double a = 0, b = 0, cr = 0, ci = 0, e = 0, f = 0;
-            if (act) {
-                a = Srow[c]; b = Srow[d + c]; cr = Rrow[c]; ci = Rrow[d + c]; e = Orow[c]; f = Orow[d + c];
+            const uint32_t cl = act ? c : 0;                 // idle lanes read (and discard) dimension 0
+            // every value this block of dimensions needs, requested before the first use
+            const float a_f = Srow[cl], b_f = Srow[d + cl], cr_f = Rrow[cl], ci_f = Rrow[d + cl];
+            const float e_f = Orow[cl], f_f = Orow[d + cl];
+            const float GS_re = Srow[2 * d + cl], GS_im = Srow[3 * d + cl];
+            const float GR_re = Rrow[2 * d + cl], GR_im = Rrow[3 * d + cl];
+            const float GO_re = Orow[2 * d + cl], GO_im = Orow[3 * d + cl];
+            float na_f[kMaxNeg], nb_f[kMaxNeg], GN_re[kMaxNeg], GN_im[kMaxNeg];
+#pragma unroll
+            for (int q = 0; q < kMaxNeg; ++q) {
+                const bool live = q < (int)n_neg;
+                na_f[q] = live ? Nrow[q][cl] : 0.f;
+                nb_f[q] = live ? Nrow[q][d + cl] : 0.f;
+                GN_re[q] = ((nrep_mask >> q) & 1u) ? Nrow[q][2 * d + cl] : 0.f;
+                GN_im[q] = ((nrep_mask >> q) & 1u) ? Nrow[q][3 * d + cl] : 0.f;
             }
+            const double a = a_f, b = b_f, cr = cr_f, ci = ci_f, e = e_f, f = f_f;
             // directions that do not depend on the negative
             const double dS_re = cr * e + ci * f, dS_im = cr * f - ci * e;      // d phi / d subject, object = o
             const double dO_re = cr * a - ci * b, dO_im = cr * b + ci * a;      // d phi / d object, subject = s
             double gs_re = cf0 * dS_re, gs_im = cf0 * dS_im;
             double go_re = cf0 * dO_re, go_im = cf0 * dO_im;
             double gr_re = cf0 * (a * e + b * f), gr_im = cf0 * (a * f - b * e);
-            for (int q = 1; q <= (int)n_neg; ++q) {
-                const double cf = __shfl_sync(full, coef, q);
-                const int sd = __shfl_sync(full, side, 2 + q);
-                const float* Nq = store + __shfl_sync(full, off, 2 + q);
-                double na = 0, nb = 0;
-                if (act) { na = Nq[c]; nb = Nq[d + c]; }
-                if (sd == 0) {          // triple (n, r, o)
-                    gr_re += cf * (na * e + nb * f); gr_im += cf * (na * f - nb * e);
-                    go_re += cf * (cr * na - ci * nb); go_im += cf * (cr * nb + ci * na);
+#pragma unroll
+            for (int q = 0; q < kMaxNeg; ++q) {
+                const double na = na_f[q], nb = nb_f[q];
+                const double w = __shfl_sync(full, coef, (q + 1) & 31);
+                if ((subj_mask >> q) & 1u) {     // triple (n, r, o)
+                    gr_re += w * (na * e + nb * f); gr_im += w * (na * f - nb * e);
+                    go_re += w * (cr * na - ci * nb); go_im += w * (cr * nb + ci * na);
                 } else {                // triple (s, r, n)
-                    gr_re += cf * (a * na + b * nb); gr_im += cf * (a * nb - b * na);
-                    gs_re += cf * (cr * na + ci * nb); gs_im += cf * (cr * nb - ci * na);
+                    gr_re += w * (a * na + b * nb); gr_im += w * (a * nb - b * na);
+                    gs_re += w * (cr * na + ci * nb); gs_im += w * (cr * nb - ci * na);
                 }
             }
             // negatives that coincide with the subject or the object
             gs_re += wS0 * dS_re + wO0 * dO_re; gs_im += wS0 * dS_im + wO0 * dO_im;
             go_re += wS2 * dS_re + wO2 * dO_re; go_im += wS2 * dS_im + wO2 * dO_im;
             if (rep_o == 0) { gs_re += go_re; gs_im += go_im; }
-            for (int u = 0; u < n_slots; ++u) {
-                const int ru = __shfl_sync(full, rep, u);
-                const double wSu = __shfl_sync(full, wS, u), wOu = __shfl_sync(full, wO, u);
-                const uint64_t offu = __shfl_sync(full, off, u);
-                if (ru != u || !act) continue;
-                double gd_re, gd_im;
-                if (u == 0) { gd_re = gs_re; gd_im = gs_im; }
-                else if (u == 1) { gd_re = gr_re; gd_im = gr_im; }
-                else if (u == 2) { gd_re = go_re; gd_im = go_im; }
-                else { gd_re = wSu * dS_re + wOu * dO_re; gd_im = wSu * dS_im + wOu * dO_im; }
-                const float g_re = (float)gd_re, g_im = (float)gd_im;
-                const float G_re = store[offu + 2 * d + c], G_im = store[offu + 3 * d + c];
-                const float g2_re = g_re * g_re, g2_im = g_im * g_im;
-                float* Uu = U + (uint64_t)u * L;
-                Uu[c] = -lr * g_re / (sqrtf(G_re + g2_re) + eps);
-                Uu[d + c] = -lr * g_im / (sqrtf(G_im + g2_im) + eps);
-                Uu[2 * d + c] = g2_re;
-                Uu[3 * d + c] = g2_im;
+            if (act) {
+                adagrad_out(U, c, gs_re, gs_im, GS_re, GS_im);
+                adagrad_out(U + L, c, gr_re, gr_im, GR_re, GR_im);
+                if (rep_o == 2) adagrad_out(U + 2 * (uint64_t)L, c, go_re, go_im, GO_re, GO_im);
+            }
+#pragma unroll
+            for (int q = 0; q < kMaxNeg; ++q) {
+                const double wSq = __shfl_sync(full, wS, (3 + q) & 31), wOq = __shfl_sync(full, wO, (3 + q) & 31);
+                if (act && ((nrep_mask >> q) & 1u))
+                    adagrad_out(U + (uint64_t)(3 + q) * L, c, wSq * dS_re + wOq * dO_re, wSq * dS_im + wOq * dO_im,
+                                GN_re[q], GN_im[q]);
             }
         }
     }
@@ -343,9 +385,13 @@ uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r,
                          const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
                          uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s) {
     const uint32_t grid = step_grid(ps, n);
-    PS_LAUNCH(ps, kge_step_kernel, grid, 256, s, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim,
-              lr, eps, (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->upd,
-              ps->loss_partial, ps->status, ps->epoch);
+#define KGE_ARGS d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, lr, eps,                     \
+                 (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->upd,         \
+                 ps->loss_partial, ps->status, ps->epoch
+    if (n_neg <= 4) PS_LAUNCH(ps, kge_step_kernel<4>, grid, 256, s, KGE_ARGS);
+    else if (n_neg <= 10) PS_LAUNCH(ps, kge_step_kernel<10>, grid, 256, s, KGE_ARGS);
+    else PS_LAUNCH(ps, kge_step_kernel<29>, grid, 256, s, KGE_ARGS);
+#undef KGE_ARGS
     return grid;
 }
 

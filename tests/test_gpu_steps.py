@@ -212,3 +212,30 @@ def test_host_batch_variants_match_the_device_calls():
                          sc.out_key_base, sc.lr, b.loss, h_loss)
     a.sync()
     assert h_loss[0] == loss_of(a) and (a.export(table=False)[0] == b.export(table=False)[0]).all()
+
+
+# ---------------------------------------------------------- pipelining ----
+def test_pipelined_mode_gives_identical_results():
+    """ps_set_pipelining lets the key sort of step t+1 run beside step t's kernels; nothing may change."""
+    cfg = W.scaled(W.MF_TINY, rows=3000, cols=400, rank=100, n_cells=40 * 2048, batch=2048, col_zipf=1.1, lr=0.0005)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    di, dj, dv = i.cuda(), j.cuda(), v.cuda()
+    out = []
+    for pipelined in (False, True):
+        g, _ = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
+        ps.ps_set_pipelining(g.h, pipelined)
+        torch.cuda.synchronize()
+        rng = np.random.default_rng(1)
+        for b in range(cfg.n_batches):
+            s, c = cfg.batch_range(b)
+            ps.ps_step_mf(g.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+            if b % 7 == 3:
+                g.localize(int(rng.integers(0, 4)), dev(rng.integers(0, cfg.num_keys, size=500)))
+            if b % 11 == 5:
+                keys = rng.integers(0, cfg.num_keys, size=700)
+                g.push(dev(keys), dev((0.01 * rng.normal(size=(700, cfg.rank))).astype(np.float32)))
+        g.sync()
+        out.append((g.export()[0].numpy(), loss_of(g)))
+    assert (out[0][0] == out[1][0]).all() and out[0][1] == out[1][1]
+    assert np.isfinite(out[0][1])
