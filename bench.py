@@ -446,6 +446,7 @@ class StressWorkload:
 
 def make_workload(name):
     table = {"mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
+             "mf_medium": lambda: MFWorkload(W.MF_MEDIUM),
              "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
              "sgns": lambda: SGNSWorkload(W.SGNS), "sgns_tiny": lambda: SGNSWorkload(W.SGNS_TINY),
              "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY)}
@@ -486,8 +487,10 @@ def timed_loop(fn, steps, device, world):
     barrier(world)
     torch.cuda.synchronize(device)
     a.record()
+    t0 = time.perf_counter()
     for k in steps:
         fn(k)
+    timed_loop.host_enqueue_ms = (time.perf_counter() - t0) * 1e3      # host time to enqueue, before any wait
     b.record()
     torch.cuda.synchronize(device)
     barrier(world)
@@ -539,10 +542,28 @@ def run_ours(args):
     torch.cuda.synchronize(device)
     launches0 = ps.ps_launch_count(h)
     moved0 = ps.ps_rows_moved(h)
+    timed = list(range(args.warmup, total))
+    # The launch-bound loop of steps is captured once into a CUDA graph (every step with its own batch
+    # pointers) and replayed with one launch; --no-graph issues the calls one by one instead.
+    graph = None
+    if not args.no_graph and getattr(wl, "graph_ok", True):
+        try:
+            torch.cuda.synchronize(device)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for k in timed:
+                    wl.step(k)
+        except Exception as e:                                 # noqa: BLE001
+            sys.stderr.write(f"graph capture failed ({e}); timing eager launches\n")
+            graph = None
+    launches0 = ps.ps_launch_count(h) if graph is None else launches0
     sampler = ClockSampler(device.index)
     sampler.start()
-    timed = list(range(args.warmup, total))
-    ms = timed_loop(wl.step, timed, device, world)
+    if graph is not None:
+        ms = timed_loop(lambda _k: graph.replay(), [0], device, world)
+    else:
+        ms = timed_loop(wl.step, timed, device, world)
+    host_ms = timed_loop.host_enqueue_ms
     clocks = sampler.stop()
     launches = ps.ps_launch_count(h) - launches0
     moved = ps.ps_rows_moved(h) - moved0
@@ -593,6 +614,8 @@ def run_ours(args):
                        accumulation="per-key sums in f64, state f32",
                        pipelining="off" if args.no_pipelining else "key sort of step t+1 beside step t (ps_set_pipelining)"),
         "gpu_launches": int(launches), "launches_per_step": launches / len(timed),
+        "host_enqueue_ms_per_step": host_ms / len(timed),
+        "launch_mode": "one CUDA graph of all timed steps" if graph is not None else "eager",
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_step": alg,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -661,9 +684,10 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mf_large",
-                    choices=["mf_large", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny"])
+                    choices=["mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host")
     ap.add_argument("--no-pipelining", action="store_true",
                     help="order each step's key sort after all earlier work instead of beside the previous step")
     args = ap.parse_args()

@@ -226,7 +226,11 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream);
  * batch are extracted and sorted on an internal stream as soon as the call is
  * made, beside the previous step's kernels, so the batch arrays must be
  * complete at call time (no writes to them still pending on `stream`).
- * Results are identical in both modes. */
+ * Results are identical in both modes.
+ * The ps_step_* calls (device-batch variants) may be captured into a CUDA graph
+ * on `stream`; the internal stream joins the capture at the first captured call
+ * and is joined back before each call returns.  Begin a capture only when the
+ * handle's earlier work has completed. */
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
 
 /* Number of kernels this handle has launched so far. */

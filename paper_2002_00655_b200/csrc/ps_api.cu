@@ -34,7 +34,7 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.valsB[b] = take(mk * 4);
         l.tile_state[b] = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
         l.sort_ctl[b] = take((size_t)kSortCtlWords * 4);
-        l.starters[b] = take(reduce_tiles * 4);
+        l.starters[b] = take(reduce_tiles * 16);
         l.starter_count[b] = take(4);
     }
     l.scan_sums = take(((mk + 255) / 256) * 4);
@@ -120,7 +120,17 @@ static SortSet* next_set(ps_store* ps) {
 // Pipelined mode: it starts as soon as the buffer set's previous user is done, i.e. beside the previous
 // step's kernels; the batch arrays must then be complete when the call is made.
 static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
-    if (ps->pipelined) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
+    // When the caller's stream enters or leaves a CUDA-graph capture, events recorded on the other side of
+    // that border cannot be waited on, and the side stream has to join (or leave) the capture: the first
+    // call after such a change forks in ordered mode and forgets the older events.
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    unsigned long long id = 0;
+    if (cudaStreamGetCaptureInfo(s, &cs, &id) != cudaSuccess) return false;
+    if (cs != cudaStreamCaptureStatusActive) id = 0;
+    const bool crossed = id != ps->capture_id;
+    ps->capture_id = id;
+    if (crossed) ps->sets[0].used = ps->sets[1].used = false;
+    if (ps->pipelined && !crossed) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
@@ -190,7 +200,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.valsB = (uint32_t*)(ps->ws + l.valsB[b]);
         ss.tile_state = (uint32_t*)(ps->ws + l.tile_state[b]);
         ss.sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl[b]);
-        ss.starters = (uint32_t*)(ps->ws + l.starters[b]);
+        ss.starters = (uint4*)(ps->ws + l.starters[b]);
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;
     }

@@ -38,7 +38,7 @@ struct SortSet {
     uint32_t *keysA, *keysB, *valsA, *valsB;
     uint32_t* tile_state;
     uint32_t* sort_ctl;
-    uint32_t* starters;
+    uint4* starters;
     unsigned int* starter_count;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
     bool used;
@@ -66,7 +66,7 @@ struct ps_store {
     uint32_t* scan_sums;            // block sums of the device-wide scan
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
-    uint32_t* starters;             // tiles that start a border-crossing segment (nReduceTiles)
+    uint4* starters;                // {tile, key, row} of the tiles that start a border-crossing segment
     unsigned int* starter_count;
     double* loss_partial;           // kMaxLossBlocks
     char* staging;                  // host-batch staging, max_keys x 8 bytes
@@ -80,6 +80,7 @@ struct ps_store {
     psb::SortSet sets[2];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
     bool pipelined;                 // see ps_set_pipelining
+    unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
 };
 
 namespace psb {

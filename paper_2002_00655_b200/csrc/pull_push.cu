@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(256)
 push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
                    const float4* __restrict__ upd, float4* __restrict__ store, const uint2* __restrict__ table,
                    uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry,
-                   uint32_t* __restrict__ starters, unsigned int* __restrict__ starter_count,
+                   uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
                    const DevStatus* st, unsigned int epoch) {
     if (call_failed(st, epoch)) return;
     const unsigned full = 0xffffffffu;
@@ -219,7 +219,8 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
     const uint32_t key31 = __shfl_sync(full, key, 31);
     const bool runs_on = key31 < K && next_after == key31;
     // a border-crossing segment starts in this tile iff it runs on and has its head here
-    if (runs_on && head_mask != 0u && lane == 0) starters[atomicAdd(starter_count, 1u)] = tile;
+    if (runs_on && head_mask != 0u && lane == 31)
+        starters[atomicAdd(starter_count, 1u)] = make_uint4(tile, key, (uint32_t)row, (uint32_t)(row >> 32));
     const uint32_t L = L4 * 4;
     for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
         const uint32_t f = f0 + lane;
@@ -275,7 +276,7 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
 __global__ void __launch_bounds__(32 * kFixupWarps)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
-                  const double* __restrict__ carry, const uint32_t* __restrict__ starters,
+                  const double* __restrict__ carry, const uint4* __restrict__ starters,
                   const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
                   uint32_t loss_blocks, double* __restrict__ loss_accum, const DevStatus* st, unsigned int epoch) {
     __shared__ d4 part[kFixupWarps][32];
@@ -299,12 +300,11 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t count = *starter_count;
     const uint32_t L = L4 * 4;
+    const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
     for (uint32_t si = blockIdx.x; si < count; si += gridDim.x - 1) {
-        const uint32_t tile = starters[si];
-        const uint64_t base = (uint64_t)tile * kReduceTile;
-        const uint32_t kl = sk[base + kReduceTile - 1];
-        const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
-        const uint64_t row = phys_row(table[kl], S);
+        const uint4 rec = starters[si];                     // {tile, key, row} as the reduction saw them
+        const uint32_t tile = rec.x, kl = rec.y;
+        const uint64_t row = (uint64_t)rec.z | ((uint64_t)rec.w << 32);
         // last tile of the segment: every later tile whose first key is the segment's key belongs to it
         // (keys are sorted); the block's threads probe 256 tiles at a time
         uint32_t last_tile = tile;
@@ -319,6 +319,14 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             const uint32_t f = f0 + lane;
             const bool act = f < L4;
             d4 a = {0.0, 0.0, 0.0, 0.0};
+            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+            d4 own = {0.0, 0.0, 0.0, 0.0};
+            if (w == 0 && act) {                            // requested early, used after the barrier
+                r = store[row * L4 + f];
+                const double* c = carry + ((uint64_t)tile * 2 + 1) * L + (uint64_t)f * 4;
+                const double2 x = *(const double2*)c, y = *(const double2*)(c + 2);
+                own.x = x.x; own.y = x.y; own.z = y.x; own.w = y.y;
+            }
             if (act) {
 #pragma unroll 4
                 for (uint32_t t2 = tile + 1 + w; t2 <= last_tile; t2 += kFixupWarps) {
@@ -330,14 +338,11 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             part[w][lane] = a;
             __syncthreads();
             if (w == 0 && act) {
-                const double* c = carry + ((uint64_t)tile * 2 + 1) * L + (uint64_t)f * 4;
-                const double2 x = *(const double2*)c, y = *(const double2*)(c + 2);
-                d4 t = {x.x, x.y, y.x, y.y};
+                d4 t = own;
 #pragma unroll
                 for (int i = 0; i < kFixupWarps; ++i) {
                     t.x += part[i][lane].x; t.y += part[i][lane].y; t.z += part[i][lane].z; t.w += part[i][lane].w;
                 }
-                float4 r = store[row * L4 + f];
                 r.x = (float)((double)r.x + t.x); r.y = (float)((double)r.y + t.y);
                 r.z = (float)((double)r.z + t.z); r.w = (float)((double)r.w + t.w);
                 store[row * L4 + f] = r;

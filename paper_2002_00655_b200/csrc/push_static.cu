@@ -32,7 +32,7 @@ constexpr size_t kOffSortCtl =
 constexpr size_t kOffCarry = kOffSortCtl + pad256((size_t)kSortCtlWords * 4);
 constexpr size_t kOffStarters =
     kOffCarry + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 2 * (size_t)kStaticMaxRowLen * 8);
-constexpr size_t kOffStarterCount = kOffStarters + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 4);
+constexpr size_t kOffStarterCount = kOffStarters + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 16);
 constexpr size_t kStaticBytes = kOffStarterCount + 256;
 
 // About 2.3 MB per GPU.  In host code this name is only a handle for the
@@ -107,7 +107,7 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     tmp.tile_state = (uint32_t*)(dev.scratch + kOffHist);
     tmp.sort_ctl = (uint32_t*)(dev.scratch + kOffSortCtl);
     tmp.carry = (double*)(dev.scratch + kOffCarry);
-    tmp.starters = (uint32_t*)(dev.scratch + kOffStarters);
+    tmp.starters = (uint4*)(dev.scratch + kOffStarters);
     tmp.starter_count = (unsigned int*)(dev.scratch + kOffStarterCount);
     tmp.epoch = 1;
     tmp.sm_count = dev.sm_count;

@@ -20,7 +20,7 @@ constexpr uint32_t kFlagCount = 1u << 30;    // the word holds this tile's count
 constexpr uint32_t kFlagTotal = 2u << 30;    // the word holds the total up to and including this tile
 constexpr uint32_t kValueMask = (1u << 30) - 1u;
 constexpr int kLookbackSpins = 1 << 22;
-constexpr int kLookbackWindow = 8;
+constexpr int kLookbackWindow = 16;
 
 // ctl layout: [kMaxPasses][kRadix] histograms, then kMaxPasses tickets.
 __global__ void __launch_bounds__(kSortThreads)

@@ -116,6 +116,9 @@ class MFConfig:
 MF_TINY = MFConfig("mf_tiny", 1_000, 1_000, 8, 100_000, 1_024, 0.01, 0.05, 0.1, 0.1, None)
 MF_LARGE = MFConfig("mf_large", 10_000_000, 1_000_000, 100, 500_000_000, 65_536,
                     0.002, 0.05, 0.1, 0.5, 1.1)
+# a fifth of the large matrix with the same minibatch: for profiler captures, which should hold little memory
+MF_MEDIUM = MFConfig("mf_medium", 2_000_000, 200_000, 100, 100_000_000, 65_536,
+                     0.002, 0.05, 0.1, 0.5, 1.1)
 
 
 def mf_init_rows(cfg: MFConfig, key_start: int, count: int, device) -> torch.Tensor:
