@@ -150,7 +150,7 @@ loc_move_kernel(LocScratch sc, float4* __restrict__ store, uint32_t worker, uint
 // keysA already holds the call's keys (range-checked).
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s) {
     LocScratch sc = loc_scratch(ps);
-    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, nullptr);
+    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, nullptr, 0);
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     uint32_t* owner_keys = which ? ps->keysA : ps->keysB;    // the buffer the sorted keys are not in
     const uint32_t blocks = div_up_u32(n, 256);
@@ -161,7 +161,7 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s) {
     PS_LAUNCH(ps, loc_scan_sums_kernel, 1, 256, s, ps->scan_sums, blocks, ps->status, ps->epoch);
     PS_LAUNCH(ps, loc_assign_kernel, blocks, 256, s, sk, n, ps->table, worker, S, ps->tops, ps->stacks, sc.flag,
               ps->scan_sums, sc, owner_keys, ps->status, ps->epoch);
-    const int w2 = radix_sort_pairs(ps, n, &ps->status->moved_total, ps->owner_bits, true, s, which ^ 1, nullptr);
+    const int w2 = radix_sort_pairs(ps, n, &ps->status->moved_total, ps->owner_bits, true, s, which ^ 1, nullptr, 0);
     const uint32_t* so = w2 ? ps->keysB : ps->keysA;
     const uint32_t* sv = w2 ? ps->valsB : ps->valsA;
     PS_LAUNCH(ps, loc_free_kernel, blocks, 256, s, so, sv, sc.mslot, ps->tops, ps->stacks, S, ps->status, ps->epoch);

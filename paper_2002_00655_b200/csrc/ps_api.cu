@@ -33,13 +33,14 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.valsA[b] = take(mk * 4);
         l.valsB[b] = take(mk * 4);
         l.tile_state[b] = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
-        l.sort_ctl[b] = take((size_t)kSortCtlWords * 4);
+        l.sort_ctl[b] = take(((size_t)kSortCtlWords + (mk + kGroupSpan - 1) / kGroupSpan) * 4);
         l.starters[b] = take(reduce_tiles * 16);
         l.starter_count[b] = take(4);
     }
     l.scan_sums = take(((mk + 255) / 256) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
+    l.group_sum = take(((mk + kGroupSpan - 1) / kGroupSpan) * (size_t)cfg.row_len * 8);
     l.loss_partial = take(kMaxLossBlocks * 8);
     l.staging = take(mk * 8 + 256);
     l.total = off;
@@ -109,7 +110,7 @@ static SortSet* next_set(ps_store* ps) {
     ps->cur_set ^= 1;
     SortSet* ss = &ps->sets[ps->cur_set];
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
-    ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl;
+    ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
     ps->starters = ss->starters; ps->starter_count = ss->starter_count;
     return ss;
 }
@@ -200,6 +201,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.valsB = (uint32_t*)(ps->ws + l.valsB[b]);
         ss.tile_state = (uint32_t*)(ps->ws + l.tile_state[b]);
         ss.sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl[b]);
+        ss.group_done = ss.sort_ctl + kSortCtlWords;
         ss.starters = (uint4*)(ps->ws + l.starters[b]);
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;
@@ -209,6 +211,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
+    ps->group_sum = (double*)(ps->ws + l.group_sum);
     ps->loss_partial = (double*)(ps->ws + l.loss_partial);
     ps->staging = ps->ws + l.staging;
     int sms = 0;

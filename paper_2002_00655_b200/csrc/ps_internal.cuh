@@ -18,6 +18,7 @@ constexpr int kRadix = 1 << kRadixBits;
 constexpr int kMaxSortPasses = 4;                // 32-bit keys
 constexpr int kSortCtlWords = kMaxSortPasses * kRadix + kMaxSortPasses;   // digit histograms of every pass, then tickets
 constexpr int kReduceTile = 32;                  // sorted occurrences per warp in the segmented reduction
+constexpr int kGroupSpan = 64 * kReduceTile;      // sorted positions whose parked parts are pre-added together
 constexpr int kMaxLossBlocks = 4096;
 
 // Device-resident status words.  An error is latched per call with the call's
@@ -38,6 +39,7 @@ struct SortSet {
     uint32_t *keysA, *keysB, *valsA, *valsB;
     uint32_t* tile_state;
     uint32_t* sort_ctl;
+    unsigned int* group_done;
     uint4* starters;
     unsigned int* starter_count;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
@@ -62,7 +64,9 @@ struct ps_store {
     psb::DevStatus* status;
     uint32_t *keysA, *keysB, *valsA, *valsB;
     uint32_t* tile_state;           // kMaxSortPasses x nSortTiles x kRadix look-back words
-    uint32_t* sort_ctl;             // kSortCtlWords
+    uint32_t* sort_ctl;             // kSortCtlWords, followed by group_done
+    unsigned int* group_done;       // per group of 64 reduction tiles: reduction blocks that have finished
+    double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
@@ -86,7 +90,7 @@ struct ps_store {
 namespace psb {
 
 struct WsLayout {
-    size_t status, keysA[2], keysB[2], valsA[2], valsB[2], tile_state[2], sort_ctl[2], scan_sums, upd, carry,
+    size_t status, keysA[2], keysB[2], valsA[2], valsB[2], tile_state[2], sort_ctl[2], scan_sums, upd, carry, group_sum,
         starters[2], starter_count[2], loss_partial, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
@@ -113,9 +117,10 @@ void prof_after(ps_store* ps, cudaStream_t s);
 // implied as 0..n-1 when iota_vals.  If n_dev is not null the element count is
 // read from device memory (n is then an upper bound used for the launch
 // shapes).  Returns 0 if the result is in the A buffers, 1 if in the B buffers.
-// If zero_me is not null the first kernel also sets *zero_me = 0.
+// If zero_me is not null the first kernel also sets *zero_me = 0; the first `zero_groups` words of
+// group_done are cleared together with the sort's own control words.
 int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
-                     cudaStream_t stream, int start, unsigned int* zero_me);
+                     cudaStream_t stream, int start, unsigned int* zero_me, uint32_t zero_groups);
 
 // ---- pull_push.cu ----
 void launch_init_range_partition(ps_store* ps, cudaStream_t s);

@@ -176,6 +176,58 @@ struct d4 {
 
 constexpr int kReduceGroup = 4;     // sorted occurrences whose loads are issued together
 constexpr int kFixupWarps = 8;
+constexpr int kGroupMinSpan = 8 * kReduceTile;   // a group's entering segment is pre-added only if at least this long
+constexpr int kGroupTiles = 64;     // tiles whose parked parts are pre-added per group (8 reduction blocks)
+
+// Tail of the reduction kernel, kept out of line so that it does not weigh on the main loop's registers.
+// The last block to finish in an aligned group of 64 tiles adds up, once, the parked parts of the (long)
+// segment that enters the group from the group before; the fix-up kernel then needs one value per group
+// for a segment that runs through thousands of tiles (a hot key), instead of one per tile.
+__device__ __noinline__ void group_preadd(const uint32_t* __restrict__ sk, uint32_t n, uint32_t L4,
+                                          const double* __restrict__ carry, unsigned int* __restrict__ group_done,
+                                          double* __restrict__ group_sum, uint32_t group, uint64_t gpos, uint32_t kg,
+                                          d4 (*gpart)[32], unsigned int* s_ticket) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t L = L4 * 4;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) *s_ticket = atomicAdd(&group_done[group], 1u);
+    __syncthreads();
+    const uint32_t blocks_in_group = tmin<uint32_t>(kGroupTiles / 8, gridDim.x - group * (kGroupTiles / 8));
+    if (*s_ticket != blocks_in_group - 1) return;
+    __threadfence();
+    // tiles of the group that begin with the entering segment's key: a prefix of the group's tiles
+    const uint64_t tpos = gpos + (uint64_t)threadIdx.x * kReduceTile;
+    const int hit = threadIdx.x < kGroupTiles && tpos < n && sk[tpos] == kg;
+    const uint32_t m = (uint32_t)__syncthreads_count(hit);
+    const uint32_t t0 = group * kGroupTiles;
+    for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
+        const uint32_t f = f0 + lane;
+        const bool act = f < L4;
+        d4 a = {0.0, 0.0, 0.0, 0.0};
+        if (act) {
+#pragma unroll 4
+            for (uint32_t t = w; t < m; t += 8) {
+                const double* c2 = carry + ((uint64_t)(t0 + t) * 2) * L + (uint64_t)f * 4;
+                const double2 x = __ldcg((const double2*)c2), y = __ldcg((const double2*)(c2 + 2));
+                a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
+            }
+        }
+        gpart[w][lane] = a;
+        __syncthreads();
+        if (w == 0 && act) {
+            d4 t = gpart[0][lane];
+#pragma unroll
+            for (int i = 1; i < 8; ++i) {
+                t.x += gpart[i][lane].x; t.y += gpart[i][lane].y; t.z += gpart[i][lane].z; t.w += gpart[i][lane].w;
+            }
+            double* g = group_sum + (uint64_t)group * L + (uint64_t)f * 4;
+            *(double2*)g = make_double2(t.x, t.y);
+            *(double2*)(g + 2) = make_double2(t.z, t.w);
+        }
+        __syncthreads();
+    }
+}
 
 // A warp owns sorted positions [tile*32, tile*32+32).  A segment (run of equal
 // keys) that starts and ends inside the tile is summed in fp64 and applied with
@@ -191,21 +243,23 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
                    const float4* __restrict__ upd, float4* __restrict__ store, const uint2* __restrict__ table,
                    uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry,
                    uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
+                   unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
                    const DevStatus* st, unsigned int epoch) {
+    __shared__ d4 gpart[8][32];
+    __shared__ unsigned int s_ticket;
     if (call_failed(st, epoch)) return;
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t base = (uint64_t)tile * kReduceTile;
-    if (base >= n) return;
-    const uint32_t n_valid = (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base);
+    const uint32_t n_valid = base < n ? (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base) : 0u;
     const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
     const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
     const bool usable = key < K;                    // "no key" marks and padding sort last
     uint64_t row = 0;
     if (usable) row = phys_row(table[key], S);
     uint32_t prev = __shfl_up_sync(full, key, 1);
-    if (lane == 0) prev = base > 0 ? sk[base - 1] : kSentinelPad;
+    if (lane == 0) prev = (base > 0 && base - 1 < n) ? sk[base - 1] : kSentinelPad;
     const uint32_t next_after = (base + kReduceTile < n) ? sk[base + kReduceTile] : kSentinelPad;
     uint32_t next = __shfl_down_sync(full, key, 1);
     if (lane == 31) next = next_after;
@@ -221,6 +275,18 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
     // a border-crossing segment starts in this tile iff it runs on and has its head here
     if (runs_on && head_mask != 0u && lane == 31)
         starters[atomicAdd(starter_count, 1u)] = make_uint4(tile, key, (uint32_t)row, (uint32_t)(row >> 32));
+    // does a segment enter this block's group of 64 tiles from the group before?  (asked here, with the
+    // walk's loads still to come, and needed only after the walk)
+    const uint32_t group = blockIdx.x / (kGroupTiles / 8);
+    const uint64_t gpos = (uint64_t)group * kGroupTiles * kReduceTile;     // first sorted position of the group
+    // Only a segment that also covers the group's first kGroupMinSpan positions is worth it: shorter ones
+    // end within a few tiles and the fix-up kernel takes those tile by tile.
+    uint32_t kg = kSentinelPad, kg_prev = kSentinelPad - 1, kg_far = kSentinelPad - 2;
+    if (gpos > 0 && gpos + kGroupMinSpan - 1 < n) {
+        kg = sk[gpos];
+        kg_prev = sk[gpos - 1];
+        kg_far = sk[gpos + kGroupMinSpan - 1];
+    }
     const uint32_t L = L4 * 4;
     for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
         const uint32_t f = f0 + lane;
@@ -265,6 +331,11 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
             }
         }
     }
+    // ---- The last block to finish in each aligned group of 64 tiles adds up, once, the parked parts of the
+    // segment that enters the group from the group before.  The fix-up kernel then needs one value per group
+    // for a segment that runs through thousands of tiles (a hot key), instead of one per tile.
+    if (!(kg < K && kg_prev == kg && kg_far == kg)) return;     // nothing to pre-add for this group
+    group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, gpart, &s_ticket);
 }
 
 // Blocks work through the list of tiles that start a border-crossing segment.
@@ -276,7 +347,8 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
 __global__ void __launch_bounds__(32 * kFixupWarps)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
-                  const double* __restrict__ carry, const uint4* __restrict__ starters,
+                  const double* __restrict__ carry, const double* __restrict__ group_sum,
+                  const uint4* __restrict__ starters,
                   const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
                   uint32_t loss_blocks, double* __restrict__ loss_accum, const DevStatus* st, unsigned int epoch) {
     __shared__ d4 part[kFixupWarps][32];
@@ -305,15 +377,33 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
         const uint4 rec = starters[si];                     // {tile, key, row} as the reduction saw them
         const uint32_t tile = rec.x, kl = rec.y;
         const uint64_t row = (uint64_t)rec.z | ((uint64_t)rec.w << 32);
-        // last tile of the segment: every later tile whose first key is the segment's key belongs to it
-        // (keys are sorted); the block's threads probe 256 tiles at a time
-        uint32_t last_tile = tile;
-        for (;;) {
-            const uint32_t t2 = last_tile + 1 + threadIdx.x;
-            const int hit = t2 < n_tiles && sk[(uint64_t)t2 * kReduceTile] == kl;
-            const int cnt = __syncthreads_count(hit);         // hits are a prefix of the probed range
-            last_tile += (uint32_t)cnt;
-            if (cnt < (int)blockDim.x) break;
+        // The segment runs through the tiles after `tile` whose first key is its key (keys are sorted).
+        // Up to the end of the starter's group of 64 tiles they are taken one by one; every later group the
+        // segment enters has one pre-added value.
+        const uint32_t group_end = (tile / kGroupTiles + 1) * kGroupTiles;      // first tile of the next group
+        uint32_t last_tile;
+        {
+            const uint32_t t2 = tile + 1 + threadIdx.x;
+            const int hit = threadIdx.x < kGroupTiles && t2 < group_end && t2 < n_tiles &&
+                            sk[(uint64_t)t2 * kReduceTile] == kl;
+            last_tile = tile + (uint32_t)__syncthreads_count(hit);
+        }
+        uint32_t n_groups = 0;                              // later groups with a pre-added value for this segment
+        uint32_t rem_first = 0, rem_cnt = 0;                // tiles of the segment after those groups (fewer than 8)
+        if (last_tile + 1 == group_end) {
+            for (;;) {
+                const uint64_t g2 = (uint64_t)group_end / kGroupTiles + n_groups + threadIdx.x;
+                const uint64_t gp = g2 * kGroupTiles * kReduceTile;
+                const int hit = gp + kGroupMinSpan - 1 < n && sk[gp] == kl && sk[gp + kGroupMinSpan - 1] == kl;
+                const int cnt = __syncthreads_count(hit);     // hits are a prefix of the probed range
+                n_groups += (uint32_t)cnt;
+                if (cnt < (int)blockDim.x) break;
+            }
+            rem_first = group_end + n_groups * kGroupTiles;
+            const uint32_t t2 = rem_first + threadIdx.x;
+            const int hit = threadIdx.x < kGroupMinSpan / kReduceTile && t2 < n_tiles &&
+                            sk[(uint64_t)t2 * kReduceTile] == kl;
+            rem_cnt = (uint32_t)__syncthreads_count(hit);
         }
         for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
             const uint32_t f = f0 + lane;
@@ -331,6 +421,17 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
 #pragma unroll 4
                 for (uint32_t t2 = tile + 1 + w; t2 <= last_tile; t2 += kFixupWarps) {
                     const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
+                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
+                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
+                }
+                for (uint32_t t2 = rem_first + w; t2 < rem_first + rem_cnt; t2 += kFixupWarps) {
+                    const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
+                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
+                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
+                }
+#pragma unroll 4
+                for (uint32_t g2 = w; g2 < n_groups; g2 += kFixupWarps) {
+                    const double* c2 = group_sum + ((uint64_t)group_end / kGroupTiles + g2) * L + (uint64_t)f * 4;
                     const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
                     a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
                 }
@@ -353,7 +454,8 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
 }
 
 int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
-    return radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count);
+    return radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count,
+                            div_up_u32(n, kGroupSpan));
 }
 
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
@@ -365,11 +467,11 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     const uint32_t L4 = ps->cfg.row_len / 4;
     PS_LAUNCH(ps, push_reduce_kernel, blocks, 256, s, sk, sv, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
               ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
-              ps->status, ps->epoch);
+              ps->group_done, ps->group_sum, ps->status, ps->epoch);
     uint32_t fix_blocks = tiles < (uint32_t)ps->sm_count * 8 ? tiles : (uint32_t)ps->sm_count * 8;
     PS_LAUNCH(ps, push_fixup_kernel, fix_blocks + 1, 32 * kFixupWarps, s, sk, n, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
-              ps->loss_partial, loss_blocks, loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch);
+              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->group_sum, ps->starters,
+              ps->starter_count, ps->loss_partial, loss_blocks, loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch);
 }
 
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,

@@ -29,11 +29,13 @@ constexpr size_t kOffValsB = kOffValsA + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffHist = kOffValsB + pad256(kStaticMaxKeys * 4);
 constexpr size_t kOffSortCtl =
     kOffHist + pad256((size_t)kMaxSortPasses * ((kStaticMaxKeys + kSortTile - 1) / kSortTile) * kRadix * 4);
-constexpr size_t kOffCarry = kOffSortCtl + pad256((size_t)kSortCtlWords * 4);
+constexpr size_t kStaticGroups = (kStaticMaxKeys + kGroupSpan - 1) / kGroupSpan;
+constexpr size_t kOffCarry = kOffSortCtl + pad256(((size_t)kSortCtlWords + kStaticGroups) * 4);
 constexpr size_t kOffStarters =
     kOffCarry + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 2 * (size_t)kStaticMaxRowLen * 8);
 constexpr size_t kOffStarterCount = kOffStarters + pad256(((kStaticMaxKeys + kReduceTile - 1) / kReduceTile) * 16);
-constexpr size_t kStaticBytes = kOffStarterCount + 256;
+constexpr size_t kOffGroupSum = kOffStarterCount + 256;
+constexpr size_t kStaticBytes = kOffGroupSum + pad256(kStaticGroups * (size_t)kStaticMaxRowLen * 8);
 
 // About 2.3 MB per GPU.  In host code this name is only a handle for the
 // runtime; the address a kernel can use comes from cudaGetSymbolAddress.
@@ -106,6 +108,8 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     tmp.valsB = (uint32_t*)(dev.scratch + kOffValsB);
     tmp.tile_state = (uint32_t*)(dev.scratch + kOffHist);
     tmp.sort_ctl = (uint32_t*)(dev.scratch + kOffSortCtl);
+    tmp.group_done = tmp.sort_ctl + kSortCtlWords;
+    tmp.group_sum = (double*)(dev.scratch + kOffGroupSum);
     tmp.carry = (double*)(dev.scratch + kOffCarry);
     tmp.starters = (uint4*)(dev.scratch + kOffStarters);
     tmp.starter_count = (unsigned int*)(dev.scratch + kOffStarterCount);

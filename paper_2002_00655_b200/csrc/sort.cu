@@ -164,7 +164,7 @@ sort_pass_kernel(const uint32_t* __restrict__ kin, const uint32_t* __restrict__ 
 }
 
 int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
-                     cudaStream_t stream, int start, unsigned int* zero_me) {
+                     cudaStream_t stream, int start, unsigned int* zero_me, uint32_t zero_groups) {
     if (n == 0) return start;
     const uint32_t n_tiles = div_up_u32(n, kSortTile);
     uint32_t *kin = ps->keysA, *vin = ps->valsA, *kout = ps->keysB, *vout = ps->valsB;
@@ -174,7 +174,7 @@ int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bi
     int which = start;
     if (bits < 1) bits = 1;
     const int n_passes = (bits + kRadixBits - 1) / kRadixBits;
-    cudaMemsetAsync(ps->sort_ctl, 0, kSortCtlWords * sizeof(uint32_t), stream);
+    cudaMemsetAsync(ps->sort_ctl, 0, (kSortCtlWords + (size_t)zero_groups) * sizeof(uint32_t), stream);
     PS_LAUNCH(ps, sort_hist_kernel, n_tiles, kSortThreads, stream, kin, n, n_dev, n_passes, ps->sort_ctl,
               ps->tile_state, n_tiles, zero_me);
     for (int pass = 0; pass < n_passes; ++pass) {
