@@ -111,6 +111,14 @@ void prof_after(ps_store* ps, cudaStream_t s);
         (ps)->launches++;                                                    \
     } while (0)
 
+#define PS_LAUNCH_SMEM(ps, kernel, grid, block, smem, stream, ...)            \
+    do {                                                                     \
+        if ((ps)->prof) psb::prof_before((ps), #kernel, (stream));           \
+        kernel<<<(grid), (block), (smem), (stream)>>>(__VA_ARGS__);          \
+        if ((ps)->prof) psb::prof_after((ps), (stream));                     \
+        (ps)->launches++;                                                    \
+    } while (0)
+
 // ---- sort.cu ----
 // Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key.
 // Input in the A buffers (start = 0) or the B buffers (start = 1); values are

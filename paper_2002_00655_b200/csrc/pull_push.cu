@@ -174,7 +174,19 @@ struct d4 {
     double x, y, z, w;
 };
 
-constexpr int kReduceGroup = 4;     // sorted occurrences whose loads are issued together
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(kPending) : "memory");
+}
+
+constexpr int kReduceGroup = 4;     // sorted occurrences whose copies are issued together
+constexpr int kReduceStages = 3;    // groups in flight per warp
+constexpr size_t kReduceSmem = (size_t)8 * kReduceStages * 2 * kReduceGroup * 32 * sizeof(float4);
 constexpr int kFixupWarps = 8;
 constexpr int kGroupMinSpan = 8 * kReduceTile;   // a group's entering segment is pre-added only if at least this long
 constexpr int kGroupTiles = 64;     // tiles whose parked parts are pre-added per group (8 reduction blocks)
@@ -288,52 +300,66 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
         kg_far = sk[gpos + kGroupMinSpan - 1];
     }
     const uint32_t L = L4 * 4;
+    // Rows are staged through shared memory with asynchronous 16-byte copies: each lane copies, for a group
+    // of kReduceGroup positions, its own float4 of the update row and (where a segment ends) of the target
+    // row, and later reads back exactly what it copied, so no lane ever waits for another.  kReduceStages
+    // groups are kept in flight per warp.
+    extern __shared__ float4 stage_mem[];
+    float4* my_stage = stage_mem + (size_t)(threadIdx.x >> 5) * (kReduceStages * 2 * kReduceGroup * 32) + lane;
+    const int n_groups = ((int)n_valid + kReduceGroup - 1) / kReduceGroup;
     for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
         const uint32_t f = f0 + lane;
         const bool act = f < L4;
-        d4 acc = {0.0, 0.0, 0.0, 0.0};
-        for (int p0 = 0; p0 < (int)n_valid; p0 += kReduceGroup) {
-            float4 u[kReduceGroup], r[kReduceGroup];
-            uint64_t rows[kReduceGroup];
+        auto issue = [&](int g) {
+            float4* slot = my_stage + (size_t)(g % kReduceStages) * (2 * kReduceGroup * 32);
+            if (g < n_groups) {
 #pragma unroll
-            for (int k = 0; k < kReduceGroup; ++k) {
-                const int p = p0 + k;                       // p <= 31 because p0 < n_valid <= 32 and p0 % 4 == 0
-                const uint32_t o = __shfl_sync(full, occ, p);
-                rows[k] = __shfl_sync(full, row, p);
-                const bool ok = (usable_mask >> p) & 1u;
-                const bool ends = ok && ((end_mask >> p) & 1u);
-                const bool parked = ends && (p < first_head || (p == 31 && runs_on));
-                u[k] = (ok && act) ? __ldcs(upd + (uint64_t)o * L4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
-                r[k] = (ends && !parked && act) ? store[rows[k] * L4 + f] : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < kReduceGroup; ++k) {
+                    const int p = g * kReduceGroup + k;     // p <= 31
+                    const uint32_t o = __shfl_sync(full, occ, p);
+                    const uint64_t rw = __shfl_sync(full, row, p);
+                    const bool ok = (usable_mask >> p) & 1u;
+                    const bool ends = ok && ((end_mask >> p) & 1u);
+                    const bool parked = ends && (p < first_head || (p == 31 && runs_on));
+                    if (ok && act) cp_async16(slot + k * 32, upd + (uint64_t)o * L4 + f);
+                    if (ends && !parked && act) cp_async16(slot + (kReduceGroup + k) * 32, store + rw * L4 + f);
+                }
             }
+            cp_async_commit();                              // one (possibly empty) batch per call
+        };
+#pragma unroll
+        for (int g = 0; g < kReduceStages - 1; ++g) issue(g);
+        d4 acc = {0.0, 0.0, 0.0, 0.0};
+        for (int g = 0; g < n_groups; ++g) {
+            issue(g + kReduceStages - 1);
+            cp_async_wait<kReduceStages - 1>();             // group g has landed; later ones may still fly
+            const float4* slot = my_stage + (size_t)(g % kReduceStages) * (2 * kReduceGroup * 32);
 #pragma unroll
             for (int k = 0; k < kReduceGroup; ++k) {
-                const int p = p0 + k;
-                if (!((usable_mask >> p) & 1u)) continue;
-                acc.x += (double)u[k].x; acc.y += (double)u[k].y; acc.z += (double)u[k].z; acc.w += (double)u[k].w;
+                const int p = g * kReduceGroup + k;
+                const uint64_t rw = __shfl_sync(full, row, p);
+                if (!((usable_mask >> p) & 1u) || !act) continue;
+                const float4 u = slot[k * 32];
+                acc.x += (double)u.x; acc.y += (double)u.y; acc.z += (double)u.z; acc.w += (double)u.w;
                 if ((end_mask >> p) & 1u) {
                     const bool from_prev = p < first_head;
                     const bool parked = from_prev || (p == 31 && runs_on);
-                    if (act) {
-                        if (!parked) {
-                            float4 v = r[k];
-                            v.x = (float)((double)v.x + acc.x); v.y = (float)((double)v.y + acc.y);
-                            v.z = (float)((double)v.z + acc.z); v.w = (float)((double)v.w + acc.w);
-                            store[rows[k] * L4 + f] = v;
-                        } else {
-                            double* c = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
-                            *(double2*)c = make_double2(acc.x, acc.y);
-                            *(double2*)(c + 2) = make_double2(acc.z, acc.w);
-                        }
+                    if (!parked) {
+                        float4 v = slot[(kReduceGroup + k) * 32];
+                        v.x = (float)((double)v.x + acc.x); v.y = (float)((double)v.y + acc.y);
+                        v.z = (float)((double)v.z + acc.z); v.w = (float)((double)v.w + acc.w);
+                        store[rw * L4 + f] = v;
+                    } else {
+                        double* c = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
+                        *(double2*)c = make_double2(acc.x, acc.y);
+                        *(double2*)(c + 2) = make_double2(acc.z, acc.w);
                     }
                     acc.x = acc.y = acc.z = acc.w = 0.0;
                 }
             }
         }
+        cp_async_wait<0>();                                 // nothing of this column block is pending any more
     }
-    // ---- The last block to finish in each aligned group of 64 tiles adds up, once, the parked parts of the
-    // segment that enters the group from the group before.  The fix-up kernel then needs one value per group
-    // for a segment that runs through thousands of tiles (a hot key), instead of one per tile.
     if (!(kg < K && kg_prev == kg && kg_far == kg)) return;     // nothing to pre-add for this group
     group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, gpart, &s_ticket);
 }
@@ -465,7 +491,12 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     const uint32_t tiles = div_up_u32(n, kReduceTile);
     const uint32_t blocks = div_up_u32(tiles, 8);
     const uint32_t L4 = ps->cfg.row_len / 4;
-    PS_LAUNCH(ps, push_reduce_kernel, blocks, 256, s, sk, sv, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
+    static bool smem_set = false;
+    if (!smem_set) {
+        cudaFuncSetAttribute(push_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kReduceSmem);
+        smem_set = true;
+    }
+    PS_LAUNCH_SMEM(ps, push_reduce_kernel, blocks, 256, kReduceSmem, s, sk, sv, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
               ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
               ps->group_done, ps->group_sum, ps->status, ps->epoch);
     uint32_t fix_blocks = tiles < (uint32_t)ps->sm_count * 8 ? tiles : (uint32_t)ps->sm_count * 8;

@@ -121,6 +121,76 @@ mf_step_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj,
     block_loss_out(loss, loss_partial);
 }
 
+// Rows of at most 128 values: one float4 per lane and row.  A warp works on kCells cells at a time so
+// that their index, table and row loads are all in flight together (each cell is a chain of three
+// dependent loads; one cell per warp leaves the memory system idle most of the time).
+template <int kCells>
+__global__ void __launch_bounds__(256)
+mf_step_small_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, const float* __restrict__ cv,
+                     uint64_t n, uint64_t col_base, float lr, float lam, const float4* __restrict__ store,
+                     const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t L4,
+                     float4* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st,
+                     unsigned int epoch) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const bool act = (uint32_t)lane < L4;
+    double loss = 0;
+    for (uint64_t t0 = warp * kCells; t0 < n; t0 += n_warps * kCells) {
+        uint64_t kw[kCells], kh[kCells];
+        float v[kCells];
+        bool ok[kCells];
+#pragma unroll
+        for (int c = 0; c < kCells; ++c) {
+            const uint64_t t = t0 + c;
+            ok[c] = t < n;
+            kw[c] = ok[c] ? ci[t] : 0;
+            kh[c] = ok[c] ? col_base + cj[t] : 0;
+            v[c] = ok[c] ? cv[t] : 0.f;
+            if (ok[c] && (kw[c] >= col_base || kh[c] >= K)) {
+                if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+                ok[c] = false;
+            }
+        }
+        uint2 ew[kCells], eh[kCells];
+#pragma unroll
+        for (int c = 0; c < kCells; ++c) {
+            ew[c] = ok[c] ? table[kw[c]] : make_uint2(0, 0);
+            eh[c] = ok[c] ? table[kh[c]] : make_uint2(0, 0);
+        }
+        float4 w[kCells], h[kCells];
+#pragma unroll
+        for (int c = 0; c < kCells; ++c) {
+            const bool ld = ok[c] && act;
+            w[c] = ld ? store[phys_row(ew[c], S) * L4 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+            h[c] = ld ? store[phys_row(eh[c], S) * L4 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int c = 0; c < kCells; ++c) {
+            float dot = w[c].x * h[c].x + w[c].y * h[c].y + w[c].z * h[c].z + w[c].w * h[c].w;
+            float nw = w[c].x * w[c].x + w[c].y * w[c].y + w[c].z * w[c].z + w[c].w * w[c].w;
+            float nh = h[c].x * h[c].x + h[c].y * h[c].y + h[c].z * h[c].z + h[c].w * h[c].w;
+            dot = warp_sum(dot);
+            nw = warp_sum(nw);
+            nh = warp_sum(nh);
+            if (!ok[c]) continue;
+            const float e = v[c] - dot;
+            loss += (double)(0.5f * e * e + 0.5f * lam * (nw + nh));
+            if (act) {
+                const uint64_t t = t0 + c;
+                float4 dw, dh;
+                dw.x = lr * (e * h[c].x - lam * w[c].x); dw.y = lr * (e * h[c].y - lam * w[c].y);
+                dw.z = lr * (e * h[c].z - lam * w[c].z); dw.w = lr * (e * h[c].w - lam * w[c].w);
+                dh.x = lr * (e * w[c].x - lam * h[c].x); dh.y = lr * (e * w[c].y - lam * h[c].y);
+                dh.z = lr * (e * w[c].z - lam * h[c].z); dh.w = lr * (e * w[c].w - lam * h[c].w);
+                upd[(2 * t) * L4 + lane] = dw;
+                upd[(2 * t + 1) * L4 + lane] = dh;
+            }
+        }
+    }
+    block_loss_out(loss, loss_partial);
+}
+
 // keys of the occurrences of a batch of cells: [2t] = row factor, [2t+1] = column factor
 __global__ void __launch_bounds__(256)
 mf_keys_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, uint64_t n, uint64_t col_base,
@@ -140,7 +210,7 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
 #define MF_ARGS d_i, d_j, d_v, n, col_key_base, lr, lambda, (const float4*)ps->store, ps->table,                 \
                 ps->cfg.slots_per_part, ps->cfg.num_keys, L4, (float4*)ps->upd, ps->loss_partial,              \
                 ps->status, ps->epoch
-    if (L4 <= 32) PS_LAUNCH(ps, mf_step_kernel<1>, grid, 256, s, MF_ARGS);
+    if (L4 <= 32) PS_LAUNCH(ps, mf_step_small_kernel<4>, grid, 256, s, MF_ARGS);
     else if (L4 <= 64) PS_LAUNCH(ps, mf_step_kernel<2>, grid, 256, s, MF_ARGS);
     else if (L4 <= 128) PS_LAUNCH(ps, mf_step_kernel<4>, grid, 256, s, MF_ARGS);
     else PS_LAUNCH(ps, mf_step_kernel<0>, grid, 256, s, MF_ARGS);
