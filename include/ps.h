@@ -221,11 +221,12 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream);
 
 /* Latency hiding across steps, after the paper's pre-localization (Section 2.2,
  * "latency hiding": prepare the next data point's parameters while the current
- * one is processed).  Off (default): a ps_step_* call reads its batch arrays
- * only after everything already enqueued on `stream`.  On: the keys of the
- * batch are extracted and sorted on an internal stream as soon as the call is
- * made, beside the previous step's kernels, so the batch arrays must be
- * complete at call time (no writes to them still pending on `stream`).
+ * one is processed).  It concerns ps_step_*, ps_push and ps_localize.
+ * Off (default): such a call reads its batch arrays (indices, keys) only after
+ * everything already enqueued on `stream`.  On: the keys of the batch are
+ * extracted and sorted on an internal stream as soon as the call is made,
+ * beside the kernels of earlier calls, so those arrays must be complete at
+ * call time (no writes to them still pending on `stream`).
  * Results are identical in both modes.
  * The ps_step_* calls (device-batch variants) may be captured into a CUDA graph
  * on `stream`; the internal stream joins the capture at the first captured call

@@ -147,10 +147,9 @@ loc_move_kernel(LocScratch sc, float4* __restrict__ store, uint32_t worker, uint
     }
 }
 
-// keysA already holds the call's keys (range-checked).
-void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s) {
+// The call's keys (range-checked) have been sorted already; `which` says into which buffers.
+void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s) {
     LocScratch sc = loc_scratch(ps);
-    const int which = radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, nullptr, 0);
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     uint32_t* owner_keys = which ? ps->keysA : ps->keysB;    // the buffer the sorted keys are not in
     const uint32_t blocks = div_up_u32(n, 256);

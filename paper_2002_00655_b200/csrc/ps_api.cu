@@ -286,8 +286,11 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
     if (!d_keys || !d_updates) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
-    launch_prepare_keys(ps, d_keys, n, s);
-    run_push_pipeline(ps, (uint32_t)n, d_updates, nullptr, 0, s);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;         // the keys are sorted beside earlier calls' kernels
+    launch_prepare_keys(ps, d_keys, n, ps->side);
+    const int which = run_push_sort(ps, (uint32_t)n, ps->side);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_push_reduce(ps, (uint32_t)n, which, d_updates, nullptr, 0, s);
     return release_set(ss, s);
 }
 
@@ -298,8 +301,11 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     if (!d_keys) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
-    launch_prepare_keys(ps, d_keys, n, s);
-    run_localize(ps, worker, (uint32_t)n, s);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
+    launch_prepare_keys(ps, d_keys, n, ps->side);
+    const int which = radix_sort_pairs(ps, (uint32_t)n, nullptr, ps->key_bits, true, ps->side, 0, nullptr, 0);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_localize(ps, worker, (uint32_t)n, which, s);
     return release_set(ss, s);
 }
 

@@ -149,7 +149,7 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
                      uint32_t loss_blocks, cudaStream_t s);
 
 // ---- localize.cu ----
-void run_localize(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s);
+void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
 
 // ---- steps.cu ----
 // launch_keys_* write the keys of a batch's occurrence slots to keysA (they depend on the batch
