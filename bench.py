@@ -11,10 +11,12 @@ one ps_push and one ps_localize.  Default workload: matrix factorization,
 replica and the value is the sum over replicas.
 
 Prints ONE JSON line: throughput with the batch resident in HBM (`value`),
-the same through the host-buffer entry point (`e2e`), the fraction of the
-measured HBM copy bandwidth that the algorithmic bytes of a step reach
-(`roofline`), a per-kernel time table (`kernels`), and the CPU oracle timed on
-a bounded sample of the same workload (`cpu_baseline`).
+the same through the host-buffer entry point (`e2e`), a per-kernel table with
+each kernel's own bytes over its own time (`kernels`), the row of that table
+with the largest share of a step as a fraction of the measured HBM copy
+bandwidth (`roofline`), the same fraction for the bytes the method must move
+per step over the whole timed step (`roofline_step`), and the CPU oracle timed
+on a bounded sample of the same workload (`cpu_baseline`).
 """
 from __future__ import annotations
 
@@ -111,8 +113,26 @@ def smi_clocks():
 # ----------------------------------------------------------------------------------------
 # workloads
 # ----------------------------------------------------------------------------------------
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/,
+# keyed by (workload, kernel).  An entry is removed when its kernel changes after the capture.
+TRAFFIC = {}
+
+
 def n_unique(*tensors) -> int:
     return int(torch.unique(torch.cat([t.reshape(-1).to(torch.int64) for t in tensors])).numel())
+
+
+def kernel_bytes_of_step(batch_bytes, occ, u, rb, keys_prefix, step_prefix):
+    """Bytes per LAUNCH that each kernel of a step call must move, by kernel-name prefix: what it reads of the
+    batch, the table and the store, and what it has to write for the next kernel (keys, update rows)."""
+    return {
+        keys_prefix: batch_bytes + occ * 4,                      # batch arrays in, one 32-bit key per occurrence out
+        "sort_hist_kernel": occ * 4,
+        "sort_pass_kernel<true>": occ * 12,                      # keys in; keys and occurrence indices out
+        "sort_pass_kernel<false>": occ * 16,
+        step_prefix: batch_bytes + occ * (8 + rb) + occ * rb,    # table entry + row per occurrence in, update row out
+        "push_reduce_kernel": occ * (8 + rb) + u * (8 + 2 * rb), # sorted pair + update row in; row read-modify-write
+    }
 
 
 class MFWorkload:
@@ -179,6 +199,12 @@ class MFWorkload:
         sl = slice(k * b, (k + 1) * b)
         u = n_unique(self.i[sl]) + n_unique(self.j[sl])
         return b * 12 + 2 * b * (8 + self.row_bytes) + u * 2 * self.row_bytes
+
+    def kernel_bytes(self, k):
+        c, b = self.cfg, self.cfg.batch
+        sl = slice(k * b, (k + 1) * b)
+        u = n_unique(self.i[sl]) + n_unique(self.j[sl])
+        return kernel_bytes_of_step(b * 12, 2 * b, u, self.row_bytes, "mf_keys", "mf_step")
 
     # --- oracle leg ---
     def oracle_setup(self, device):
@@ -269,6 +295,11 @@ class KGEWorkload:
         u = n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl])
         return b * (12 + c.n_neg * 5) + occ * (8 + self.row_bytes) + u * 2 * self.row_bytes
 
+    def kernel_bytes(self, k):
+        c, sl, b = self.cfg, self._sl(k), self.cfg.batch
+        u = n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl])
+        return kernel_bytes_of_step(b * (12 + c.n_neg * 5), (3 + c.n_neg) * b, u, self.row_bytes, "kge_keys", "kge_step")
+
     def oracle_setup(self, device):
         from oracle import OracleStore
         c = self.cfg
@@ -355,6 +386,26 @@ class SGNSWorkload:
         occ = c.batch + pairs * (1 + c.n_neg)
         return c.batch * 4 + pairs * (1 + c.n_neg) * 4 + occ * (8 + self.row_bytes) + u * 2 * self.row_bytes
 
+    def _occ_u(self, k):
+        c = self.cfg
+        first = k * c.batch
+        pairs = c.pairs_before(first + c.batch) - c.pairs_before(first)
+        lo = max(0, first - c.window)
+        u = n_unique(self.tokens[first:first + c.batch]) + \
+            n_unique(self.tokens[lo:first + c.batch + c.window], self.negs[k])
+        return pairs, c.batch + pairs * (1 + c.n_neg), u
+
+    def kernel_bytes(self, k):
+        c = self.cfg
+        pairs, occ, u = self._occ_u(k)
+        kb = kernel_bytes_of_step(c.batch * 4 + pairs * (1 + c.n_neg) * 4, occ, u, self.row_bytes,
+                                  "sgns_keys", "sgns_step")
+        # the step kernel writes two source rows per center and one factor per occurrence, not a row per occurrence
+        kb["sgns_step"] += c.batch * 2 * self.row_bytes + occ * 4 - occ * self.row_bytes
+        # ... and the reduction reads a factor per occurrence and those 2 x centers source rows (from L2 after the first touch)
+        kb["push_reduce_kernel"] += occ * 4 + c.batch * 2 * self.row_bytes - occ * self.row_bytes
+        return kb
+
     def oracle_setup(self, device):
         from oracle import OracleStore
         c = self.cfg
@@ -439,6 +490,11 @@ class StressWorkload:
         push = n * (16 + rb) + u * 2 * rb
         loc = c.localize_count * 16                              # rows moved are added from the device counter
         return pull + push + loc
+
+    def kernel_bytes(self, k):
+        n, rb = self.cfg.batch, self.row_bytes
+        u = n_unique(self.keys[k])
+        return {"pull_kernel": n * (16 + 2 * rb), "push_reduce_kernel": n * (8 + rb) + u * (8 + 2 * rb)}
 
     def oracle_setup(self, device):
         return None
@@ -603,8 +659,22 @@ def run_ours(args):
         wl.step(k)
     prof = ps.ps_profile_stop(h)
     tot_us = sum(us for _, us in prof.values()) or 1.0
-    kernels = [{"name": name, "launches_per_step": n / prof_steps, "us_per_step": us / prof_steps,
-                "share": us / tot_us} for name, (n, us) in prof.items()]
+    kb = {}
+    for k in sample_ks:
+        for pre, v in wl.kernel_bytes(k).items():
+            kb[pre] = kb.get(pre, 0.0) + v / len(sample_ks)
+    kernels = []
+    for name, (n, us) in prof.items():
+        row = {"name": name, "launches_per_step": n / prof_steps, "us_per_launch": us / n, "us_per_step": us / prof_steps,
+               "share": us / tot_us, "alg_bytes_per_launch": None, "gbs": None, "frac": None}
+        pre = next((p for p in kb if name.startswith(p)), None)
+        if pre is not None:
+            row["alg_bytes_per_launch"] = kb[pre]
+            row["gbs"] = kb[pre] / (us / n * 1e-6) / 1e9
+            row["frac"] = row["gbs"] / peak
+        kernels.append(row)
+    rated = [r for r in kernels if r["frac"] is not None]
+    dom = max(rated, key=lambda r: r["us_per_step"]) if rated else None
 
     out = {
         "metric": METRIC, "value": value, "unit": f"{wl.example}/s", "n_gpus": world, "steps": len(timed),
@@ -616,11 +686,19 @@ def run_ours(args):
         "gpu_launches": int(launches), "launches_per_step": launches / len(timed),
         "host_enqueue_ms_per_step": host_ms / len(timed),
         "launch_mode": "one CUDA graph of all timed steps" if graph is not None else "eager",
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_step": alg,
-                     "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "scope": "one step = all kernels of one C-ABI call sequence; algorithmic bytes = batch arrays "
-                              "+ occurrences x (8 B table entry + row read) + distinct keys x (row read + row write)"},
+        # `roofline`: the kernel that takes the largest share of a step, its own bytes over its own time (launched
+        # alone, events on its stream, in the per-kernel pass after the timed region).  `roofline_step`: the
+        # bytes the METHOD must move per step (no update rows, no sort traffic) over the whole timed step.
+        "roofline": None if dom is None else {
+            "bound": "hbm", "kernel": dom["name"], "achieved": dom["gbs"], "peak": peak, "unit": "GB/s",
+            "frac": dom["frac"], "traffic": TRAFFIC.get((wl.cfg.name, dom["name"])), "peak_source": peak_src,
+            "algorithmic_bytes_per_launch": dom["alg_bytes_per_launch"], "us_per_launch": dom["us_per_launch"],
+            "frac_of_nominal_8TBs": dom["gbs"] / 8000.0},
+        "roofline_step": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                          "algorithmic_bytes_per_step": alg, "frac_of_nominal_8TBs": achieved / 8000.0,
+                          "scope": "one step = all kernels of one C-ABI call sequence; algorithmic bytes = batch "
+                                   "arrays + occurrences x (8 B table entry + row read) + distinct keys x (row read "
+                                   "+ row write)"},
         "kernels": kernels, "e2e": e2e, "clocks": clocks, "loss_sum": loss if finite else None,
         "loss_finite": finite,
     }

@@ -12,7 +12,10 @@
  * ------------------------------------
  * Memory.   The library never allocates device memory.  Every `d_*` pointer is
  *           DEVICE memory owned by the caller and must stay valid until the
- *           stream has executed the call.  Every `h_*` pointer is HOST memory
+ *           stream has executed the call.  Buffers of rows (`d_vals`,
+ *           `d_out`, `d_updates`) must be 16-byte aligned: they are moved as
+ *           128-bit vectors and by bulk copies; a misaligned one is refused
+ *           with PS_ERR_INVALID_ARG.  Every `h_*` pointer is HOST memory
  *           owned by the caller.  The library owns only the host handle.
  * Streams.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *           Every call except ps_create/ps_destroy/ps_sync/ps_export*, the
@@ -75,7 +78,8 @@ typedef struct {
 /* Sizes of the four device buffers the caller must allocate (256-byte aligned).
  * `max_batch_keys` bounds the key occurrences of any later call: n for
  * pull/push/localize, 2n for ps_step_mf, (3 + n_neg) * n for ps_step_kge,
- * n_centers * (1 + 2 * window * (1 + n_neg)) for ps_step_sgns. */
+ * n_centers * (1 + 2 * window * (1 + n_neg)), and at least 3 * n_centers,
+ * for ps_step_sgns. */
 ps_status_t ps_query_sizes(const ps_config_t* cfg, uint64_t max_batch_keys, ps_sizes_t* out);
 
 /* Creates the host handle around caller-allocated device buffers of at least
@@ -245,8 +249,10 @@ ps_status_t ps_rows_moved(ps_store_t* ps, uint64_t* h_out);
  * their stream.  ps_profile_stop waits for the device, writes one line per
  * kernel, "name launches total_microseconds\n", in first-launch order, into
  * h_report (NUL-terminated, truncated to `capacity` bytes) and turns timing off.
- * The events add a little time between kernels: do not time a run end to end
- * while profiling is on. */
+ * Each bracketed launch first waits for the whole device to go idle, so a time
+ * is that of the kernel running alone (nothing beside it on the internal
+ * stream): calls made while profiling is on run serialised, must not be captured
+ * into a CUDA graph, and must not be timed end to end. */
 ps_status_t ps_profile_start(ps_store_t* ps, uint32_t max_launches);
 ps_status_t ps_profile_stop(ps_store_t* ps, char* h_report, size_t capacity);
 

@@ -68,6 +68,9 @@ void prof_before(ps_store* ps, const char* name, cudaStream_t s) {
         cudaEventDestroy(r.a);
         return;
     }
+    // Every timed launch starts on an idle device, so that a kernel's time is its own and not that of
+    // whatever the other stream runs beside it.  Profiling therefore serialises the calls it covers.
+    cudaDeviceSynchronize();
     cudaEventRecord(r.a, s);
     p->recs.push_back(r);
     p->open = true;
@@ -267,7 +270,7 @@ ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
 ps_status_t ps_set_rows(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_vals, void* stream) {
     PS_BEGIN_CALL(ps);
     if (n == 0) return PS_OK;
-    if (!d_keys || !d_vals) return PS_ERR_INVALID_ARG;
+    if (!d_keys || !d_vals || ((uintptr_t)d_vals & 15)) return PS_ERR_INVALID_ARG;
     launch_set_rows(ps, d_keys, n, d_vals, s);
     return after_launch();
 }
@@ -275,7 +278,7 @@ ps_status_t ps_set_rows(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, cons
 ps_status_t ps_pull(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, float* d_out, void* stream) {
     PS_BEGIN_CALL(ps);
     if (n == 0) return PS_OK;
-    if (!d_keys || !d_out) return PS_ERR_INVALID_ARG;
+    if (!d_keys || !d_out || ((uintptr_t)d_out & 15)) return PS_ERR_INVALID_ARG;
     launch_pull(ps, d_keys, n, d_out, s);
     return after_launch();
 }
@@ -283,7 +286,7 @@ ps_status_t ps_pull(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, float* d
 ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const float* d_updates, void* stream) {
     PS_BEGIN_CALL(ps);
     if (n == 0) return PS_OK;
-    if (!d_keys || !d_updates) return PS_ERR_INVALID_ARG;
+    if (!d_keys || !d_updates || ((uintptr_t)d_updates & 15)) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;         // the keys are sorted beside earlier calls' kernels
@@ -355,7 +358,8 @@ static ps_status_t sgns_checks(ps_store_t* ps, uint64_t first_pos, uint64_t n_ce
     if (ps->cfg.row_len > 512) return PS_ERR_UNSUPPORTED;
     if (out_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
     *occ = n_centers * (1 + (uint64_t)2 * window * (1 + (uint64_t)n_neg));
-    if (*occ > ps->max_keys) return PS_ERR_WORKSPACE;
+    // two source rows per center and one factor per slot share the update buffer
+    if (*occ > ps->max_keys || 3 * n_centers > ps->max_keys) return PS_ERR_WORKSPACE;
     return PS_OK;
 }
 
@@ -375,7 +379,8 @@ ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t firs
     const uint32_t lb = launch_step_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
-    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s,
+                    sgns_scales(ps, n_centers), (uint32_t)(occ / n_centers));
     return release_set(ss, s);
 }
 
@@ -474,7 +479,8 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     const uint32_t lb = launch_step_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
-    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    run_push_reduce(ps, (uint32_t)occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s,
+                    sgns_scales(ps, n_centers), (uint32_t)(occ / n_centers));
     c = release_set(ss, s);
     if (c != PS_OK) return c;
     return finish_host_step(d_loss_accum, h_loss, s);

@@ -143,10 +143,12 @@ void launch_prepare_keys(ps_store* ps, const uint64_t* d_keys, uint64_t n, cudaS
 // first `loss_blocks` loss partials to *d_loss_accum (if not null)
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
                        cudaStream_t s);
-// the two halves of the above: sort keysA (returns which buffer holds the result), then reduce and apply
+// the two halves of the above: sort keysA (returns which buffer holds the result), then reduce and apply.
+// With d_scales, occurrence o contributes d_scales[o] times a shared source row of d_upd: row 2e for slot 0
+// of example e = o / slots, row 2e + 1 for its other slots.
 int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s);
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
-                     uint32_t loss_blocks, cudaStream_t s);
+                     uint32_t loss_blocks, cudaStream_t s, const float* d_scales = nullptr, uint32_t slots = 0);
 
 // ---- localize.cu ----
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
@@ -154,7 +156,8 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
 // ---- steps.cu ----
 // launch_keys_* write the keys of a batch's occurrence slots to keysA (they depend on the batch
 // only, so they and the sort can run beside the gradient kernel); launch_step_* write the slots'
-// update rows to `upd` and return the number of per-block loss partials they wrote.
+// update rows to `upd` (launch_step_sgns: two source rows per center and one factor per slot, to be
+// reduced with run_push_reduce's d_scales) and return the number of per-block loss partials they wrote.
 void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint64_t n, uint64_t col_key_base,
                     cudaStream_t s);
 void launch_keys_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
@@ -167,6 +170,7 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
 uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                          const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
                          uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s);
+float* sgns_scales(ps_store* ps, uint64_t n_centers);     // where launch_step_sgns puts the per-slot factors
 uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
                           uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
                           uint32_t n_neg, uint64_t out_key_base, float lr, cudaStream_t s);

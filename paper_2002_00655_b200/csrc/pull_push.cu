@@ -174,19 +174,48 @@ struct d4 {
     double x, y, z, w;
 };
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    const unsigned dst = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem) : "memory");
+// ---- bulk asynchronous copies global -> shared, reporting to a barrier word in shared memory ----
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int kPending>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(kPending) : "memory");
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
+// one arrival that also announces `bytes` of copies
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// 16-byte aligned source and destination, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
+                     smem_addr(smem)),
+                 "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.
+constexpr unsigned kBarPollLimit = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
+    const unsigned a = smem_addr(bar);
+    for (unsigned i = 0; i < kBarPollLimit; ++i) {
+        unsigned done;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(done)
+            : "r"(a), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
 }
 
-constexpr int kReduceGroup = 4;     // sorted occurrences whose copies are issued together
-constexpr int kReduceStages = 3;    // groups in flight per warp
-constexpr size_t kReduceSmem = (size_t)8 * kReduceStages * 2 * kReduceGroup * 32 * sizeof(float4);
+// Staging of the reduction kernel for rows of up to kCh column blocks (32 float4 each): positions whose
+// copies are asked for together, and groups in flight per warp.  A position takes 2 x kCh x 512 bytes (update
+// row and target row); a warp stages 6 KB (8 KB for kCh = 4), so four (three) blocks of 8 warps fit an SM.
+__host__ __device__ constexpr int reduce_group(int kCh) { return kCh == 1 ? 2 : 1; }
+__host__ __device__ constexpr int reduce_stages(int kCh) { return kCh <= 2 ? 3 : 2; }
+__host__ __device__ constexpr size_t reduce_smem(int kCh) {
+    return (size_t)8 * reduce_stages(kCh) * reduce_group(kCh) * 2 * kCh * 32 * sizeof(float4);
+}
+static_assert(reduce_smem(1) >= 8 * 32 * 32 && reduce_smem(4) <= 64 * 1024, "staging also serves as the pre-add scratch");
 constexpr int kFixupWarps = 8;
 constexpr int kGroupMinSpan = 8 * kReduceTile;   // a group's entering segment is pre-added only if at least this long
 constexpr int kGroupTiles = 64;     // tiles whose parked parts are pre-added per group (8 reduction blocks)
@@ -250,15 +279,21 @@ __device__ __noinline__ void group_preadd(const uint32_t* __restrict__ sk, uint3
 // Every lane looks up the row of its own position's key, so the 32 table reads
 // go out together; then the positions are walked in groups whose update rows
 // and target rows are all requested before the first is used.
+//
+// kScaled: occurrence o does not have an update row of its own.  Its update is scales[o] times a source
+// row shared with other occurrences: the occurrences come in runs of `slots` per example, example e owning
+// source rows 2e (used, by its slot 0) and 2e + 1 (used by all its other slots) of `upd`.
+template <int kCh, bool kScaled>
 __global__ void __launch_bounds__(256)
 push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
-                   const float4* __restrict__ upd, float4* __restrict__ store, const uint2* __restrict__ table,
+                   const float4* __restrict__ upd, const float* __restrict__ scales, uint32_t slots,
+                   float4* __restrict__ store, const uint2* __restrict__ table,
                    uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry,
                    uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
                    unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
-                   const DevStatus* st, unsigned int epoch) {
-    __shared__ d4 gpart[8][32];
+                   DevStatus* st, unsigned int epoch) {
     __shared__ unsigned int s_ticket;
+    __shared__ __align__(8) uint64_t bars[8][3];    // per warp and stage: the barrier word its copies report to
     if (call_failed(st, epoch)) return;
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -266,8 +301,14 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
     const uint64_t base = (uint64_t)tile * kReduceTile;
     const uint32_t n_valid = base < n ? (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base) : 0u;
     const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
-    const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
+    uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
     const bool usable = key < K;                    // "no key" marks and padding sort last
+    float scale = 1.f;
+    if (kScaled && usable) {
+        scale = scales[occ];
+        const uint32_t e = occ / slots;
+        occ = 2u * e + (occ != e * slots ? 1u : 0u);
+    }
     uint64_t row = 0;
     if (usable) row = phys_row(table[key], S);
     uint32_t prev = __shfl_up_sync(full, key, 1);
@@ -300,68 +341,111 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
         kg_far = sk[gpos + kGroupMinSpan - 1];
     }
     const uint32_t L = L4 * 4;
-    // Rows are staged through shared memory with asynchronous 16-byte copies: each lane copies, for a group
-    // of kReduceGroup positions, its own float4 of the update row and (where a segment ends) of the target
-    // row, and later reads back exactly what it copied, so no lane ever waits for another.  kReduceStages
-    // groups are kept in flight per warp.
+    // Rows are staged through shared memory with bulk asynchronous copies: for a group of G positions the
+    // lane that owns a position asks for its whole update row and, where a segment ends, for the target row
+    // (one instruction each for the whole group), the copies report to a barrier word of the warp's own,
+    // and ST groups are kept in flight per warp.
+    constexpr int G = reduce_group(kCh), ST = reduce_stages(kCh);
+    constexpr int kSlotF4 = 2 * G * kCh * 32;                   // float4s of one stage of one warp
     extern __shared__ float4 stage_mem[];
-    float4* my_stage = stage_mem + (size_t)(threadIdx.x >> 5) * (kReduceStages * 2 * kReduceGroup * 32) + lane;
-    const int n_groups = ((int)n_valid + kReduceGroup - 1) / kReduceGroup;
-    for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
-        const uint32_t f = f0 + lane;
-        const bool act = f < L4;
-        auto issue = [&](int g) {
-            float4* slot = my_stage + (size_t)(g % kReduceStages) * (2 * kReduceGroup * 32);
-            if (g < n_groups) {
-#pragma unroll
-                for (int k = 0; k < kReduceGroup; ++k) {
-                    const int p = g * kReduceGroup + k;     // p <= 31
-                    const uint32_t o = __shfl_sync(full, occ, p);
-                    const uint64_t rw = __shfl_sync(full, row, p);
-                    const bool ok = (usable_mask >> p) & 1u;
-                    const bool ends = ok && ((end_mask >> p) & 1u);
-                    const bool parked = ends && (p < first_head || (p == 31 && runs_on));
-                    if (ok && act) cp_async16(slot + k * 32, upd + (uint64_t)o * L4 + f);
-                    if (ends && !parked && act) cp_async16(slot + (kReduceGroup + k) * 32, store + rw * L4 + f);
-                }
+    const int w = threadIdx.x >> 5;
+    float4* my_stage = stage_mem + (size_t)w * (ST * kSlotF4);
+    if (lane < ST) mbar_init(&bars[w][lane], 1);
+    mbar_init_fence();
+    __syncwarp();
+    const int n_groups = ((int)n_valid + G - 1) / G;
+    // positions whose target row is fetched: a segment ends there and is neither parked on the way in nor out
+    const bool fetch_me = usable && (key != next || lane == 31) && !(lane < first_head || (lane == 31 && runs_on));
+    const unsigned fetch_mask = __ballot_sync(full, fetch_me);
+    const unsigned gmask0 = G == 32 ? full : ((1u << G) - 1u);
+    uint32_t uses = 0;                                          // how often the warp has waited so far, per stage: parity
+    bool dead = false;
+    for (uint32_t f0 = 0; f0 < L4 && !dead; f0 += 32 * kCh) {   // one round unless a row is longer than 128 kCh floats
+        const uint32_t chunk4 = tmin<uint32_t>(L4 - f0, 32u * kCh);
+        const uint32_t chunk_bytes = chunk4 * 16u;
+        const uint32_t fl = f0 + lane;
+        auto issue = [&](int g, int stage) {
+            if (g >= n_groups) return;
+            const unsigned gm = gmask0 << (g * G);
+            const uint32_t n_rows = __popc(usable_mask & gm) + __popc(fetch_mask & gm);
+            if (n_rows == 0) return;                            // nothing to wait for either: see the walk
+            if (lane == g * G) mbar_expect_tx(&bars[w][stage], n_rows * chunk_bytes);
+            __syncwarp();
+            if ((gm >> lane) & 1u) {
+                float4* dst = my_stage + (size_t)stage * kSlotF4 + (size_t)(lane - g * G) * (2 * kCh * 32);
+                if (usable) bulk_g2s(dst, upd + (uint64_t)occ * L4 + f0, chunk_bytes, &bars[w][stage]);
+                if (fetch_me) bulk_g2s(dst + kCh * 32, store + row * L4 + f0, chunk_bytes, &bars[w][stage]);
             }
-            cp_async_commit();                              // one (possibly empty) batch per call
         };
 #pragma unroll
-        for (int g = 0; g < kReduceStages - 1; ++g) issue(g);
-        d4 acc = {0.0, 0.0, 0.0, 0.0};
-        for (int g = 0; g < n_groups; ++g) {
-            issue(g + kReduceStages - 1);
-            cp_async_wait<kReduceStages - 1>();             // group g has landed; later ones may still fly
-            const float4* slot = my_stage + (size_t)(g % kReduceStages) * (2 * kReduceGroup * 32);
+        for (int g = 0; g < ST - 1; ++g) issue(g, g);
+        d4 acc[kCh];
 #pragma unroll
-            for (int k = 0; k < kReduceGroup; ++k) {
-                const int p = g * kReduceGroup + k;
-                const uint64_t rw = __shfl_sync(full, row, p);
-                if (!((usable_mask >> p) & 1u) || !act) continue;
-                const float4 u = slot[k * 32];
-                acc.x += (double)u.x; acc.y += (double)u.y; acc.z += (double)u.z; acc.w += (double)u.w;
-                if ((end_mask >> p) & 1u) {
-                    const bool from_prev = p < first_head;
-                    const bool parked = from_prev || (p == 31 && runs_on);
-                    if (!parked) {
-                        float4 v = slot[(kReduceGroup + k) * 32];
-                        v.x = (float)((double)v.x + acc.x); v.y = (float)((double)v.y + acc.y);
-                        v.z = (float)((double)v.z + acc.z); v.w = (float)((double)v.w + acc.w);
-                        store[rw * L4 + f] = v;
+        for (int c = 0; c < kCh; ++c) acc[c] = d4{0.0, 0.0, 0.0, 0.0};
+        int st_use = 0, st_fill = ST - 1;
+        for (int g = 0; g < n_groups; ++g) {
+            __syncwarp();                                       // every lane is done reading the stage to be refilled
+            issue(g + ST - 1, st_fill);
+            const unsigned gm = gmask0 << (g * G);
+            const float4* slot = my_stage + (size_t)st_use * kSlotF4 + lane;
+            if (usable_mask & gm) {
+                const uint32_t parity = (uses >> st_use) & 1u;
+                if (!mbar_wait(&bars[w][st_use], parity) && !mbar_wait(&bars[w][st_use], parity)) {
+                    if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
+                    dead = true;                                // a copy that does not arrive: give the call up
+                    break;
+                }
+                uses ^= 1u << st_use;
+            }
+            st_use = st_use + 1 == ST ? 0 : st_use + 1;
+            st_fill = st_fill + 1 == ST ? 0 : st_fill + 1;
+#pragma unroll
+            for (int k = 0; k < G; ++k) {
+                const int p = g * G + k;
+                const float sc = kScaled ? __shfl_sync(full, scale, p) : 1.f;
+                if (!((usable_mask >> p) & 1u)) continue;
+                const double d = (double)sc;
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    if (fl + 32 * c >= L4) continue;
+                    const float4 u = slot[(k * 2 * kCh + c) * 32];
+                    if (kScaled) {
+                        acc[c].x += d * (double)u.x; acc[c].y += d * (double)u.y;
+                        acc[c].z += d * (double)u.z; acc[c].w += d * (double)u.w;
                     } else {
-                        double* c = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
-                        *(double2*)c = make_double2(acc.x, acc.y);
-                        *(double2*)(c + 2) = make_double2(acc.z, acc.w);
+                        acc[c].x += (double)u.x; acc[c].y += (double)u.y;
+                        acc[c].z += (double)u.z; acc[c].w += (double)u.w;
                     }
-                    acc.x = acc.y = acc.z = acc.w = 0.0;
+                }
+                if (!((end_mask >> p) & 1u)) continue;
+                const uint64_t rw = __shfl_sync(full, row, p);
+                const bool from_prev = p < first_head;
+                const bool parked = from_prev || (p == 31 && runs_on);
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    const uint32_t f = fl + 32 * c;
+                    if (f < L4) {
+                        if (!parked) {
+                            float4 v = slot[(k * 2 * kCh + kCh + c) * 32];
+                            v.x = (float)((double)v.x + acc[c].x); v.y = (float)((double)v.y + acc[c].y);
+                            v.z = (float)((double)v.z + acc[c].z); v.w = (float)((double)v.w + acc[c].w);
+                            store[rw * L4 + f] = v;
+                        } else {
+                            double* cs = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
+                            *(double2*)cs = make_double2(acc[c].x, acc[c].y);
+                            *(double2*)(cs + 2) = make_double2(acc[c].z, acc[c].w);
+                        }
+                    }
+                    acc[c] = d4{0.0, 0.0, 0.0, 0.0};
                 }
             }
         }
-        cp_async_wait<0>();                                 // nothing of this column block is pending any more
+        __syncwarp();
     }
     if (!(kg < K && kg_prev == kg && kg_far == kg)) return;     // nothing to pre-add for this group
-    group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, gpart, &s_ticket);
+    // the staging memory is free by now (every warp has waited for all its copies) and serves as scratch
+    group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
+                 &s_ticket);
 }
 
 // Blocks work through the list of tiles that start a border-crossing segment.
@@ -485,20 +569,41 @@ int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
 }
 
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
-                     uint32_t loss_blocks, cudaStream_t s) {
+                     uint32_t loss_blocks, cudaStream_t s, const float* d_scales, uint32_t slots) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     const uint32_t* sv = which ? ps->valsB : ps->valsA;
     const uint32_t tiles = div_up_u32(n, kReduceTile);
     const uint32_t blocks = div_up_u32(tiles, 8);
     const uint32_t L4 = ps->cfg.row_len / 4;
-    static bool smem_set = false;
-    if (!smem_set) {
-        cudaFuncSetAttribute(push_reduce_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kReduceSmem);
-        smem_set = true;
+#define REDUCE_ARGS sk, sv, n, (const float4*)d_upd, d_scales, slots, (float4*)ps->store, ps->table,                 \
+                    ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters,                \
+                    ps->starter_count, ps->group_done, ps->group_sum, ps->status, ps->epoch
+#define REDUCE_LAUNCH(kCh, kScaled)                                                                                  \
+    do {                                                                                                             \
+        static bool smem_set = false;                                                                                \
+        if (!smem_set) {                                                                                             \
+            cudaFuncSetAttribute(push_reduce_kernel<kCh, kScaled>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                                 (int)reduce_smem(kCh));                                                             \
+            smem_set = true;                                                                                         \
+        }                                                                                                            \
+        if (ps->prof) prof_before(ps, "push_reduce_kernel<" #kCh "," #kScaled ">", s);                               \
+        push_reduce_kernel<kCh, kScaled><<<blocks, 256, reduce_smem(kCh), s>>>(REDUCE_ARGS);                         \
+        if (ps->prof) prof_after(ps, s);                                                                             \
+        ps->launches++;                                                                                              \
+    } while (0)
+    if (d_scales) {
+        if (L4 <= 32) REDUCE_LAUNCH(1, true);
+        else if (L4 <= 64) REDUCE_LAUNCH(2, true);
+        else if (L4 <= 96) REDUCE_LAUNCH(3, true);
+        else REDUCE_LAUNCH(4, true);
+    } else {
+        if (L4 <= 32) REDUCE_LAUNCH(1, false);
+        else if (L4 <= 64) REDUCE_LAUNCH(2, false);
+        else if (L4 <= 96) REDUCE_LAUNCH(3, false);
+        else REDUCE_LAUNCH(4, false);
     }
-    PS_LAUNCH_SMEM(ps, push_reduce_kernel, blocks, 256, kReduceSmem, s, sk, sv, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters, ps->starter_count,
-              ps->group_done, ps->group_sum, ps->status, ps->epoch);
+#undef REDUCE_LAUNCH
+#undef REDUCE_ARGS
     uint32_t fix_blocks = tiles < (uint32_t)ps->sm_count * 8 ? tiles : (uint32_t)ps->sm_count * 8;
     PS_LAUNCH(ps, push_fixup_kernel, fix_blocks + 1, 32 * kFixupWarps, s, sk, n, (float4*)ps->store, ps->table,
               ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->group_sum, ps->starters,

@@ -80,7 +80,7 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     if (row_len % 4 != 0 || row_len > kStaticMaxRowLen) return PS_ERR_UNSUPPORTED;
     if (n > kStaticMaxKeys) return PS_ERR_WORKSPACE;
     if (n == 0) return PS_OK;
-    if (!d_keys || !d_updates) return PS_ERR_INVALID_ARG;
+    if (!d_keys || !d_updates || ((uintptr_t)d_updates & 15) || ((uintptr_t)d_store & 15)) return PS_ERR_INVALID_ARG;
     int device = -1;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return PS_ERR_CUDA;
     PerDevice dev;

@@ -487,26 +487,38 @@ __device__ __forceinline__ uint64_t sgns_pairs_before(uint64_t p, uint64_t T, ui
 
 // Occurrence slots of center number c of the batch: slot_base = c * (1 + 2W(1 + n_neg));
 // slot_base = the center's input vector; then per context j (ascending position) 1 + n_neg output vectors.
+// The update of an output vector is a multiple of the center's input vector, the same vector for all of
+// the center's slots, so it is not written out per slot: the kernel writes, per center, two source rows
+// (2c: the summed update of the input vector; 2c + 1: a copy of the input vector as it was before the
+// batch) and one factor per slot (1 for slot 0); the reduction multiplies as it adds.
+// A warp takes one center at a time.  The output-vector slots are handled 32 at a time: every lane first
+// resolves one slot (word -> key -> table entry -> row address), so those lookups are in flight together;
+// the rows are then read four slots at a time, all loads of the four before the first dot product.
 template <int kCh>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64_t first_pos, uint64_t n_centers,
                  uint64_t T, uint32_t window, const uint32_t* __restrict__ negs, uint32_t n_neg, uint64_t out_base,
                  float lr, const float4* __restrict__ store, const uint2* __restrict__ table, uint64_t S, uint64_t K,
-                 uint32_t L4, float4* __restrict__ upd, double* __restrict__ loss_partial, DevStatus* st,
-                 unsigned int epoch) {
+                 uint32_t L4, float4* __restrict__ upd, float* __restrict__ scales, double* __restrict__ loss_partial,
+                 DevStatus* st, unsigned int epoch) {
+    const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t per_ctx = 1 + n_neg;
     const uint64_t slots = 1 + (uint64_t)2 * window * per_ctx;
     const uint64_t pairs0 = sgns_pairs_before(first_pos, T, window);
+    constexpr int kQuad = 4;
     double loss = 0;
     for (uint64_t cidx = warp; cidx < n_centers; cidx += n_warps) {
         const uint64_t p = first_pos + cidx;
         const uint64_t lo = p >= window ? p - window : 0;
         const uint64_t hi = p + window < T ? p + window : T - 1;
         const uint64_t z0 = sgns_pairs_before(p, T, window) - pairs0;
-        float4* U = upd + cidx * slots * L4;
+        const uint32_t n_left = (uint32_t)(p - lo);
+        const uint32_t n_out = (uint32_t)(hi - lo) * per_ctx;   // contexts (the center itself excluded) x (1 + n_neg)
+        float4* U = upd + cidx * 2 * L4;
+        float* F = scales + cidx * slots;
         const uint32_t wtok = tokens[p - tok_first];
         if (wtok >= out_base) {
             if (lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
@@ -522,45 +534,80 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
         }
         float loss_c = 0.f;
         bool bad = false;
-        uint32_t j = 0;
-        for (uint64_t q = lo; q <= hi; ++q) {
-            if (q == p) continue;
-            const uint64_t z = z0 + j;
-            for (uint32_t i = 0; i <= n_neg; ++i) {
-                const uint32_t word = i == 0 ? tokens[q - tok_first] : negs[z * n_neg + (i - 1)];
+        for (uint32_t t0 = 0; t0 < n_out; t0 += 32) {
+            // this lane's slot of the round
+            const uint32_t t = t0 + lane;
+            uint64_t my_row = 0;
+            bool my_ok = false;
+            if (t < n_out) {
+                const uint32_t j = t / per_ctx, i = t - j * per_ctx;
+                const uint64_t q = j < n_left ? lo + j : lo + j + 1;            // skip the center itself
+                const uint32_t word = i == 0 ? tokens[q - tok_first] : negs[(z0 + j) * n_neg + (i - 1)];
                 const uint64_t ku = out_base + word;
-                const uint64_t slot = 1 + (uint64_t)j * per_ctx + i;
-                if (ku >= K) { bad = true; continue; }
-                const float4* Urow = store + phys_row(table[ku], S) * L4;
-                float4 u[kCh];
-                float x = 0.f;
-#pragma unroll
-                for (int c = 0; c < kCh; ++c) {
-                    const uint32_t f = lane + 32 * c;
-                    u[c] = f < L4 ? Urow[f] : make_float4(0.f, 0.f, 0.f, 0.f);
-                    x += v[c].x * u[c].x + v[c].y * u[c].y + v[c].z * u[c].z + v[c].w * u[c].w;
-                }
-                x = warp_sum(x);
-                const float y = i == 0 ? 1.f : 0.f;
-                const float g = sigmoidf(x) - y;
-                loss_c += i == 0 ? softplusf(-x) : softplusf(x);
-                const float sc = -lr * g;
-#pragma unroll
-                for (int c = 0; c < kCh; ++c) {
-                    const uint32_t f = lane + 32 * c;
-                    dv[c].x += sc * u[c].x; dv[c].y += sc * u[c].y; dv[c].z += sc * u[c].z; dv[c].w += sc * u[c].w;
-                    if (f < L4)
-                        U[slot * L4 + f] = make_float4(sc * v[c].x, sc * v[c].y, sc * v[c].z, sc * v[c].w);
+                if (ku < K) {
+                    my_row = phys_row(table[ku], S);
+                    my_ok = true;
+                } else {
+                    bad = true;
                 }
             }
-            ++j;
+            const unsigned ok_mask = __ballot_sync(full, my_ok);
+            const uint32_t in_round = tmin<uint32_t>(32u, n_out - t0);
+            float my_scale = 0.f;                                               // factor of this lane's slot
+            for (uint32_t b = 0; b < in_round; b += kQuad) {
+                float4 u[kQuad][kCh];
+                float x[kQuad];
+#pragma unroll
+                for (int a = 0; a < kQuad; ++a) {
+                    const uint64_t r = __shfl_sync(full, my_row, (b + a) & 31);
+                    const bool ok = (ok_mask >> (b + a)) & 1u;                  // b + a <= 31; bits past the round are 0
+                    const float4* Urow = store + r * L4;
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        const uint32_t f = lane + 32 * c;
+                        u[a][c] = (ok && f < L4) ? Urow[f] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+#pragma unroll
+                for (int a = 0; a < kQuad; ++a) {
+                    x[a] = 0.f;
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c)
+                        x[a] += v[c].x * u[a][c].x + v[c].y * u[a][c].y + v[c].z * u[a][c].z + v[c].w * u[a][c].w;
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                    for (int a = 0; a < kQuad; ++a) x[a] += __shfl_xor_sync(full, x[a], o);
+                }
+#pragma unroll
+                for (int a = 0; a < kQuad; ++a) {
+                    if (!((ok_mask >> (b + a)) & 1u)) continue;
+                    const uint32_t tt = t0 + b + a;
+                    const bool positive = tt % per_ctx == 0;
+                    const float g = sigmoidf(x[a]) - (positive ? 1.f : 0.f);
+                    loss_c += positive ? softplusf(-x[a]) : softplusf(x[a]);
+                    const float sc = -lr * g;
+                    if (lane == (int)(b + a)) my_scale = sc;
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        dv[c].x += sc * u[a][c].x; dv[c].y += sc * u[a][c].y;
+                        dv[c].z += sc * u[a][c].z; dv[c].w += sc * u[a][c].w;
+                    }
+                }
+            }
+            if (my_ok) F[1 + t] = my_scale;
         }
-        if (bad && lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+        if (__any_sync(full, bad) && lane == 0) latch_error(st, epoch, PS_ERR_KEY_RANGE);
 #pragma unroll
         for (int c = 0; c < kCh; ++c) {
             const uint32_t f = lane + 32 * c;
-            if (f < L4) U[f] = dv[c];
+            if (f < L4) {
+                U[f] = dv[c];
+                U[L4 + f] = v[c];
+            }
         }
+        if (lane == 0) F[0] = 1.f;
         loss += (double)loss_c;
     }
     block_loss_out(loss, loss_partial);
@@ -604,6 +651,9 @@ sgns_keys_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
     keys_out[x] = (uint32_t)key;
 }
 
+// the per-slot factors follow the 2 n_centers source rows in the update buffer
+float* sgns_scales(ps_store* ps, uint64_t n_centers) { return ps->upd + n_centers * 2 * ps->cfg.row_len; }
+
 uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
                           uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
                           uint32_t n_neg, uint64_t out_key_base, float lr, cudaStream_t s) {
@@ -611,7 +661,7 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
     const uint32_t grid = step_grid(ps, n_centers);
 #define SG_ARGS d_tokens, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, lr,   \
                 (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4,              \
-                (float4*)ps->upd, ps->loss_partial, ps->status, ps->epoch
+                (float4*)ps->upd, sgns_scales(ps, n_centers), ps->loss_partial, ps->status, ps->epoch
     if (L4 <= 32) PS_LAUNCH(ps, sgns_step_kernel<1>, grid, 256, s, SG_ARGS);
     else if (L4 <= 64) PS_LAUNCH(ps, sgns_step_kernel<2>, grid, 256, s, SG_ARGS);
     else if (L4 <= 96) PS_LAUNCH(ps, sgns_step_kernel<3>, grid, 256, s, SG_ARGS);
