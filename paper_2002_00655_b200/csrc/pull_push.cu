@@ -448,12 +448,14 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
                  &s_ticket);
 }
 
-// Blocks work through the list of tiles that start a border-crossing segment.
-// For one such segment the block's warps add the parked partials of the tiles
-// it runs through (warp w takes every 8th tile), the eight warp sums are added
-// in warp order to the starting tile's own partial, and the row is updated.
-// The shape of this sum depends only on the sorted positions.  The last block
-// adds the call's loss partials, in index order.
+// Warps work through the list of tiles that start a border-crossing segment, one segment per warp at a
+// time.  The warp finds the parked partials the segment has left behind (32 probes at a time): those of
+// the tiles it runs through in the starter's group, then one pre-added value per later group, then the
+// tiles after the last such group.  Up to eight partials the warp adds itself, in position order, to the
+// starting tile's own partial, and updates the row; longer walks are shared by the block's warps.
+// The shape of every sum depends only on the sorted positions.  The last block adds the call's loss
+// partials, in index order.
+template <int kCh>
 __global__ void __launch_bounds__(32 * kFixupWarps)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
@@ -461,7 +463,6 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                   const uint4* __restrict__ starters,
                   const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
                   uint32_t loss_blocks, double* __restrict__ loss_accum, const DevStatus* st, unsigned int epoch) {
-    __shared__ d4 part[kFixupWarps][32];
     if (call_failed(st, epoch)) return;
     if (blockIdx.x == gridDim.x - 1) {
         if (loss_accum) {                           // fixed-shape sum: strided per thread, then a tree
@@ -479,87 +480,148 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
         }
         return;
     }
+    const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t count = *starter_count;
     const uint32_t L = L4 * 4;
     const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
-    for (uint32_t si = blockIdx.x; si < count; si += gridDim.x - 1) {
-        const uint4 rec = starters[si];                     // {tile, key, row} as the reduction saw them
-        const uint32_t tile = rec.x, kl = rec.y;
-        const uint64_t row = (uint64_t)rec.z | ((uint64_t)rec.w << 32);
-        // The segment runs through the tiles after `tile` whose first key is its key (keys are sorted).
-        // Up to the end of the starter's group of 64 tiles they are taken one by one; every later group the
-        // segment enters has one pre-added value.
-        const uint32_t group_end = (tile / kGroupTiles + 1) * kGroupTiles;      // first tile of the next group
-        uint32_t last_tile;
-        {
-            const uint32_t t2 = tile + 1 + threadIdx.x;
-            const int hit = threadIdx.x < kGroupTiles && t2 < group_end && t2 < n_tiles &&
-                            sk[(uint64_t)t2 * kReduceTile] == kl;
-            last_tile = tile + (uint32_t)__syncthreads_count(hit);
-        }
-        uint32_t n_groups = 0;                              // later groups with a pre-added value for this segment
-        uint32_t rem_first = 0, rem_cnt = 0;                // tiles of the segment after those groups (fewer than 8)
-        if (last_tile + 1 == group_end) {
-            for (;;) {
-                const uint64_t g2 = (uint64_t)group_end / kGroupTiles + n_groups + threadIdx.x;
-                const uint64_t gp = g2 * kGroupTiles * kReduceTile;
-                const int hit = gp + kGroupMinSpan - 1 < n && sk[gp] == kl && sk[gp + kGroupMinSpan - 1] == kl;
-                const int cnt = __syncthreads_count(hit);     // hits are a prefix of the probed range
-                n_groups += (uint32_t)cnt;
-                if (cnt < (int)blockDim.x) break;
-            }
-            rem_first = group_end + n_groups * kGroupTiles;
-            const uint32_t t2 = rem_first + threadIdx.x;
-            const int hit = threadIdx.x < kGroupMinSpan / kReduceTile && t2 < n_tiles &&
-                            sk[(uint64_t)t2 * kReduceTile] == kl;
-            rem_cnt = (uint32_t)__syncthreads_count(hit);
-        }
-        for (uint32_t f0 = 0; f0 < L4; f0 += 32) {
-            const uint32_t f = f0 + lane;
-            const bool act = f < L4;
-            d4 a = {0.0, 0.0, 0.0, 0.0};
-            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-            d4 own = {0.0, 0.0, 0.0, 0.0};
-            if (w == 0 && act) {                            // requested early, used after the barrier
-                r = store[row * L4 + f];
-                const double* c = carry + ((uint64_t)tile * 2 + 1) * L + (uint64_t)f * 4;
-                const double2 x = *(const double2*)c, y = *(const double2*)(c + 2);
-                own.x = x.x; own.y = x.y; own.z = y.x; own.w = y.y;
-            }
-            if (act) {
-#pragma unroll 4
-                for (uint32_t t2 = tile + 1 + w; t2 <= last_tile; t2 += kFixupWarps) {
-                    const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
-                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
-                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
-                }
-                for (uint32_t t2 = rem_first + w; t2 < rem_first + rem_cnt; t2 += kFixupWarps) {
-                    const double* c2 = carry + ((uint64_t)t2 * 2) * L + (uint64_t)f * 4;
-                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
-                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
-                }
-#pragma unroll 4
-                for (uint32_t g2 = w; g2 < n_groups; g2 += kFixupWarps) {
-                    const double* c2 = group_sum + ((uint64_t)group_end / kGroupTiles + g2) * L + (uint64_t)f * 4;
-                    const double2 x = *(const double2*)c2, y = *(const double2*)(c2 + 2);
-                    a.x += x.x; a.y += x.y; a.z += y.x; a.w += y.y;
-                }
-            }
-            part[w][lane] = a;
-            __syncthreads();
-            if (w == 0 && act) {
-                d4 t = own;
+    const uint32_t n_warps = (gridDim.x - 1) * kFixupWarps;
+    // what a warp found out about its segment, for the block to share the work of a long one
+    struct Walk {
+        uint32_t tile, last_tile, group0, n_groups, rem_first, rem_cnt, is_long;
+        uint64_t row;
+    };
+    __shared__ Walk walks[kFixupWarps];
+    __shared__ d4 part[kFixupWarps][kCh][32];
+    // one parked partial added to a[]: base is its f = 0 element
+    auto add = [&](d4* a, uint32_t f0, const double* base) {
 #pragma unroll
-                for (int i = 0; i < kFixupWarps; ++i) {
-                    t.x += part[i][lane].x; t.y += part[i][lane].y; t.z += part[i][lane].z; t.w += part[i][lane].w;
-                }
-                r.x = (float)((double)r.x + t.x); r.y = (float)((double)r.y + t.y);
-                r.z = (float)((double)r.z + t.z); r.w = (float)((double)r.w + t.w);
-                store[row * L4 + f] = r;
+        for (int c = 0; c < kCh; ++c) {
+            const uint32_t f = f0 + lane + 32 * c;
+            if (f < L4) {
+                const double2 x = *(const double2*)(base + (uint64_t)f * 4);
+                const double2 y = *(const double2*)(base + (uint64_t)f * 4 + 2);
+                a[c].x += x.x; a[c].y += x.y; a[c].z += y.x; a[c].w += y.y;
             }
-            __syncthreads();
         }
+    };
+    // adds parked partial number i of the walk (tiles of the starter's group, then groups, then the rest)
+    auto add_nth = [&](d4* a, uint32_t f0, const Walk& k, uint32_t i) {
+        const uint32_t n1 = k.last_tile - k.tile;
+        if (i < n1) add(a, f0, carry + ((uint64_t)(k.tile + 1 + i) * 2) * L);
+        else if (i < n1 + k.n_groups) add(a, f0, group_sum + ((uint64_t)k.group0 + (i - n1)) * L);
+        else add(a, f0, carry + ((uint64_t)(k.rem_first + (i - n1 - k.n_groups)) * 2) * L);
+    };
+    for (uint32_t s0 = blockIdx.x * kFixupWarps; s0 < count; s0 += n_warps) {      // same trip count for all warps
+        const uint32_t si = s0 + w;
+        Walk k = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (si < count) {
+            const uint4 rec = starters[si];                 // {tile, key, row} as the reduction saw them
+            const uint32_t kl = rec.y;
+            k.tile = rec.x;
+            k.row = (uint64_t)rec.z | ((uint64_t)rec.w << 32);
+            // The segment runs through the tiles after `tile` whose first key is its key (keys are sorted,
+            // so they form a run).  Up to the end of the starter's group of 64 tiles they are taken one by
+            // one; every later group the segment enters has one pre-added value.
+            const uint32_t group_end = (k.tile / kGroupTiles + 1) * kGroupTiles;    // first tile of the next group
+            const uint32_t walk_end = tmin<uint32_t>(group_end, n_tiles);
+            k.last_tile = k.tile;
+            for (uint32_t t0 = k.tile + 1; t0 < walk_end; t0 += 32) {
+                const uint32_t t2 = t0 + lane;
+                const unsigned m = __ballot_sync(full, t2 < walk_end && sk[(uint64_t)t2 * kReduceTile] == kl);
+                k.last_tile += (uint32_t)__popc(m);
+                if (m != full) break;
+            }
+            k.group0 = group_end / kGroupTiles;
+            if (k.last_tile + 1 == group_end) {
+                for (;;) {
+                    const uint64_t g2 = (uint64_t)k.group0 + k.n_groups + lane;
+                    const uint64_t gp = g2 * kGroupTiles * kReduceTile;
+                    const unsigned m = __ballot_sync(
+                        full, gp + kGroupMinSpan - 1 < n && sk[gp] == kl && sk[gp + kGroupMinSpan - 1] == kl);
+                    k.n_groups += (uint32_t)__popc(m);      // hits are a prefix of the probed range
+                    if (m != full) break;
+                }
+                k.rem_first = group_end + k.n_groups * kGroupTiles;
+                const uint32_t t2 = k.rem_first + lane;
+                k.rem_cnt = (uint32_t)__popc(__ballot_sync(
+                    full, lane < kGroupMinSpan / kReduceTile && t2 < n_tiles && sk[(uint64_t)t2 * kReduceTile] == kl));
+            }
+            const uint32_t n_parts = k.last_tile - k.tile + k.n_groups + k.rem_cnt;
+            k.is_long = n_parts > kFixupWarps ? 1u : 0u;
+            if (!k.is_long) {                               // a short walk: this warp alone, partials in position order
+                for (uint32_t f0 = 0; f0 < L4; f0 += 32 * kCh) {
+                    d4 a[kCh];
+                    float4 r[kCh];
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        const uint32_t f = f0 + lane + 32 * c;
+                        a[c] = d4{0.0, 0.0, 0.0, 0.0};
+                        r[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (f < L4) r[c] = store[k.row * L4 + f];
+                    }
+                    add(a, f0, carry + ((uint64_t)k.tile * 2 + 1) * L);
+                    for (uint32_t i = 0; i < n_parts; ++i) add_nth(a, f0, k, i);
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        const uint32_t f = f0 + lane + 32 * c;
+                        if (f < L4) {
+                            float4 v = r[c];
+                            v.x = (float)((double)v.x + a[c].x); v.y = (float)((double)v.y + a[c].y);
+                            v.z = (float)((double)v.z + a[c].z); v.w = (float)((double)v.w + a[c].w);
+                            store[k.row * L4 + f] = v;
+                        }
+                    }
+                }
+            }
+        }
+        if (lane == 0) walks[w] = k;
+        __syncthreads();
+        // long walks: the block's warps share one (warp w takes every 8th partial), the eight warp sums are
+        // added in warp order to the starting tile's own partial, and warp 0 updates the row
+        for (int j = 0; j < kFixupWarps; ++j) {
+            if (!walks[j].is_long) continue;                // the same decision in every warp
+            const Walk kj = walks[j];
+            const uint32_t n_parts = kj.last_tile - kj.tile + kj.n_groups + kj.rem_cnt;
+            for (uint32_t f0 = 0; f0 < L4; f0 += 32 * kCh) {
+                d4 a[kCh];
+                float4 r[kCh];
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    const uint32_t f = f0 + lane + 32 * c;
+                    a[c] = d4{0.0, 0.0, 0.0, 0.0};
+                    r[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (w == 0 && f < L4) r[c] = store[kj.row * L4 + f];       // asked for early, used after the barrier
+                }
+#pragma unroll 2
+                for (uint32_t i = w; i < n_parts; i += kFixupWarps) add_nth(a, f0, kj, i);
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) part[w][c][lane] = a[c];
+                __syncthreads();
+                if (w == 0) {
+                    d4 t[kCh];
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) t[c] = d4{0.0, 0.0, 0.0, 0.0};
+                    add(t, f0, carry + ((uint64_t)kj.tile * 2 + 1) * L);
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        const uint32_t f = f0 + lane + 32 * c;
+                        if (f >= L4) continue;
+#pragma unroll
+                        for (int i = 0; i < kFixupWarps; ++i) {
+                            t[c].x += part[i][c][lane].x; t[c].y += part[i][c][lane].y;
+                            t[c].z += part[i][c][lane].z; t[c].w += part[i][c][lane].w;
+                        }
+                        float4 v = r[c];
+                        v.x = (float)((double)v.x + t[c].x); v.y = (float)((double)v.y + t[c].y);
+                        v.z = (float)((double)v.z + t[c].z); v.w = (float)((double)v.w + t[c].w);
+                        store[kj.row * L4 + f] = v;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        __syncthreads();                                    // walks[] is rewritten in the next round
     }
 }
 
@@ -604,10 +666,16 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     }
 #undef REDUCE_LAUNCH
 #undef REDUCE_ARGS
-    uint32_t fix_blocks = tiles < (uint32_t)ps->sm_count * 8 ? tiles : (uint32_t)ps->sm_count * 8;
-    PS_LAUNCH(ps, push_fixup_kernel, fix_blocks + 1, 32 * kFixupWarps, s, sk, n, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->group_sum, ps->starters,
-              ps->starter_count, ps->loss_partial, loss_blocks, loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch);
+    // a warp per listed segment; there are fewer segments in the list than tiles
+    const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8);
+#define FIXUP_ARGS sk, n, (float4*)ps->store, ps->table, ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4,   \
+                   ps->carry, ps->group_sum, ps->starters, ps->starter_count, ps->loss_partial, loss_blocks,      \
+                   loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch
+    if (L4 <= 32) PS_LAUNCH(ps, push_fixup_kernel<1>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else if (L4 <= 64) PS_LAUNCH(ps, push_fixup_kernel<2>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else if (L4 <= 96) PS_LAUNCH(ps, push_fixup_kernel<3>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else PS_LAUNCH(ps, push_fixup_kernel<4>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
+#undef FIXUP_ARGS
 }
 
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,
