@@ -27,7 +27,7 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     const size_t reduce_tiles = (mk + kReduceTile - 1) / kReduceTile;
     const size_t row_bytes = (size_t)cfg.row_len * 4;
     l.status = take(sizeof(DevStatus));
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kSortSets; ++b) {
         l.keysA[b] = take(mk * 4);
         l.keysB[b] = take(mk * 4);
         l.valsA[b] = take(mk * 4);
@@ -41,7 +41,8 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
     l.group_sum = take(((mk + kGroupSpan - 1) / kGroupSpan) * (size_t)cfg.row_len * 8);
-    l.loss_partial = take(kMaxLossBlocks * 8);
+    l.loss_partial = take(tmax<size_t>(kMaxLossBlocks, mk / 256 + 1) * 8);
+    l.apply_rows = take(mk * 8);
     l.staging = take(mk * 8 + 256);
     l.total = off;
     return l;
@@ -108,9 +109,9 @@ static ps_status_t check_cfg(const ps_config_t* cfg) {
 static ps_status_t after_launch() { return cuda_ok(cudaGetLastError()); }
 
 
-// Calls that sort alternate between the handle's two sets of sort buffers.
+// Calls that sort rotate through the handle's sets of sort buffers.
 static SortSet* next_set(ps_store* ps) {
-    ps->cur_set ^= 1;
+    ps->cur_set = (ps->cur_set + 1) % kSortSets;
     SortSet* ss = &ps->sets[ps->cur_set];
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
     ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
@@ -133,7 +134,8 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
     if (cs != cudaStreamCaptureStatusActive) id = 0;
     const bool crossed = id != ps->capture_id;
     ps->capture_id = id;
-    if (crossed) ps->sets[0].used = ps->sets[1].used = false;
+    if (crossed)
+        for (int b = 0; b < kSortSets; ++b) ps->sets[b].used = false;
     if (ps->pipelined && !crossed) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
@@ -196,7 +198,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->ws_bytes = workspace_bytes;
     const WsLayout l = ws_layout(*cfg, max_batch_keys);
     ps->status = (DevStatus*)(ps->ws + l.status);
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kSortSets; ++b) {
         SortSet& ss = ps->sets[b];
         ss.keysA = (uint32_t*)(ps->ws + l.keysA[b]);
         ss.keysB = (uint32_t*)(ps->ws + l.keysB[b]);
@@ -209,13 +211,14 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;
     }
-    ps->cur_set = 1;
+    ps->cur_set = kSortSets - 1;
     next_set(ps);
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
     ps->group_sum = (double*)(ps->ws + l.group_sum);
     ps->loss_partial = (double*)(ps->ws + l.loss_partial);
+    ps->apply_rows = (uint64_t*)(ps->ws + l.apply_rows);
     ps->staging = ps->ws + l.staging;
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0) {
@@ -232,12 +235,15 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
     if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->sets[0].ev_free, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->sets[1].ev_free, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
     }
+    for (int b = 0; b < kSortSets; ++b)
+        if (cudaEventCreateWithFlags(&ps->sets[b].ev_free, cudaEventDisableTiming) != cudaSuccess) {
+            delete ps;
+            return PS_ERR_CUDA;
+        }
     *out = ps;
     return PS_OK;
 }
@@ -249,8 +255,7 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
-    cudaEventDestroy(ps->sets[0].ev_free);
-    cudaEventDestroy(ps->sets[1].ev_free);
+    for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
     cudaStreamDestroy(ps->side);
     delete ps;
     return PS_OK;
@@ -323,6 +328,12 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_mf(ps, d_i, d_j, n, col_key_base, ps->side);
     const int which = run_push_sort(ps, (uint32_t)(2 * n), ps->side);
+    if (ps->cfg.row_len <= 512) {
+        // gradient and reduction in one kernel over the sorted occurrences: no update rows
+        if (!join_side(ps, s)) return PS_ERR_CUDA;
+        run_mf_fused(ps, (uint32_t)n, which, d_i, d_j, d_v, col_key_base, lr, lambda, d_loss_accum, s);
+        return release_set(ss, s);
+    }
     const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)(2 * n), which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);

@@ -20,21 +20,25 @@ constexpr int kSortCtlWords = kMaxSortPasses * kRadix + kMaxSortPasses;   // dig
 constexpr int kReduceTile = 32;                  // sorted occurrences per warp in the segmented reduction
 constexpr int kGroupSpan = 64 * kReduceTile;      // sorted positions whose parked parts are pre-added together
 constexpr int kMaxLossBlocks = 4096;
+constexpr int kSortSets = 3;                     // calls whose key sort may be in flight at once (see SortSet)
 
 // Device-resident status words.  An error is latched per call with the call's
 // epoch, so no kernel has to clear anything before a call starts.
 struct DevStatus {
     unsigned int sticky;            // first error code since the last ps_sync
-    unsigned int call_err_epoch[2]; // epoch of the last even / odd call that failed on the device (two calls
-                                    // of one handle can be in flight: one's sort beside the other's kernels)
+    unsigned int call_err_epoch[4]; // epoch of the last call with that epoch mod 4 that failed on the device (up
+                                    // to kSortSets calls of one handle are in flight: later ones' sorts beside
+                                    // the current one's kernels)
     unsigned int moved_total;       // localize: number of keys that move in the current call
     unsigned long long rows_moved;  // rows relocated by all successful localize calls so far
 };
 
+static_assert(kSortSets <= 4, "one error-epoch word per call in flight");
+
 struct Profile;
 
-// One of the two sets of buffers the key sort and the segment bookkeeping work in.  Calls alternate
-// between the sets so that the sort of one step can run while the previous step is still reducing.
+// One of the kSortSets sets of buffers the key sort and the segment bookkeeping work in.  Calls rotate
+// through the sets so that the sorts of the next steps can run while earlier steps are still reducing.
 struct SortSet {
     uint32_t *keysA, *keysB, *valsA, *valsB;
     uint32_t* tile_state;
@@ -72,7 +76,8 @@ struct ps_store {
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
     uint4* starters;                // {tile, key, row} of the tiles that start a border-crossing segment
     unsigned int* starter_count;
-    double* loss_partial;           // kMaxLossBlocks
+    double* loss_partial;           // max(kMaxLossBlocks, one per 256 key occurrences)
+    uint64_t* apply_rows;           // per sorted position: address of the row staged there, or all ones
     char* staging;                  // host-batch staging, max_keys x 8 bytes
     // host state
     uint32_t epoch;
@@ -81,7 +86,7 @@ struct ps_store {
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
     cudaStream_t side;              // key extraction and sort of a step run here, beside the gradient kernel
     cudaEvent_t ev_fork, ev_join;
-    psb::SortSet sets[2];           // keysA .. starter_count above always point into sets[cur_set]
+    psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
     bool pipelined;                 // see ps_set_pipelining
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
@@ -90,8 +95,9 @@ struct ps_store {
 namespace psb {
 
 struct WsLayout {
-    size_t status, keysA[2], keysB[2], valsA[2], valsB[2], tile_state[2], sort_ctl[2], scan_sums, upd, carry, group_sum,
-        starters[2], starter_count[2], loss_partial, staging, total;
+    size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
+        sort_ctl[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        loss_partial, apply_rows, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
 
@@ -150,6 +156,11 @@ int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s);
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
                      uint32_t loss_blocks, cudaStream_t s, const float* d_scales = nullptr, uint32_t slots = 0);
 
+// MF step working on the sorted occurrences directly (rows of at most 512 values): gradient, reduction,
+// then the fix-up launch that also moves the staged rows into the store
+void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
+                  uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, cudaStream_t s);
+
 // ---- localize.cu ----
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
 
@@ -179,10 +190,10 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
 #ifdef __CUDACC__
 __device__ __forceinline__ void latch_error(DevStatus* st, unsigned int epoch, unsigned int code) {
     atomicCAS(&st->sticky, 0u, code);
-    atomicExch(&st->call_err_epoch[epoch & 1u], epoch);
+    atomicExch(&st->call_err_epoch[epoch & 3u], epoch);
 }
 __device__ __forceinline__ bool call_failed(const DevStatus* st, unsigned int epoch) {
-    return *((const volatile unsigned int*)&st->call_err_epoch[epoch & 1u]) == epoch;
+    return *((const volatile unsigned int*)&st->call_err_epoch[epoch & 3u]) == epoch;
 }
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

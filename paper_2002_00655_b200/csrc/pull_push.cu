@@ -448,6 +448,200 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
                  &s_ticket);
 }
 
+// ------------------------------------------------- MF: gradient inside the reduction ----
+// One minibatch of matrix factorization without update rows.  The occurrences (2t: row factor of cell t,
+// 2t + 1: its column factor) arrive sorted by key, as for a push.  For every sorted position the warp
+// fetches the PARTNER row (the other factor of the cell) and, where a segment's part in the tile begins,
+// the key's own row; e = v - <own, partner> is formed on the spot and lr (e partner - lambda own) is
+// added, in fp64, to the segment's sum.  Since other warps still read rows as they were before the call,
+// nothing is written to the store here: a segment that lies inside the tile leaves its new row in
+// `staged` (indexed by the sorted position of its end) and the row's address in `apply_row`; the
+// fix-up launch, which runs after every read of this kernel, moves those rows in and finishes the
+// segments that cross tile borders from their parked partial sums, exactly as for a push.
+// The loss of a cell is taken at its row-factor occurrence.
+template <int kCh>
+__global__ void __launch_bounds__(256)
+mf_fused_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
+                const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, const float* __restrict__ cv,
+                uint32_t col_base, float lr, float lam, const float4* __restrict__ store,
+                const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
+                float4* __restrict__ staged, uint64_t* __restrict__ apply_row, double* __restrict__ carry,
+                uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
+                unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
+                double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+    __shared__ unsigned int s_ticket;
+    __shared__ __align__(8) uint64_t bars[8][3];
+    __shared__ double wl[8];
+    if (call_failed(st, epoch)) return;
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t base = (uint64_t)tile * kReduceTile;
+    const uint32_t n_valid = base < n ? (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base) : 0u;
+    const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
+    const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
+    const bool usable = key < K;                    // cells with a key out of range carry the "no key" mark
+    uint64_t row = 0, prow = 0;
+    float val = 0.f;
+    if (usable) {
+        const uint32_t t = occ >> 1;
+        const uint32_t pkey = (occ & 1u) ? ci[t] : col_base + cj[t];
+        val = cv[t];
+        row = phys_row(table[key], S);
+        prow = phys_row(table[pkey], S);            // in range: the key extraction marked the cell otherwise
+    }
+    const unsigned side0_mask = __ballot_sync(full, usable && !(occ & 1u));
+    uint32_t prev = __shfl_up_sync(full, key, 1);
+    if (lane == 0) prev = (base > 0 && base - 1 < n) ? sk[base - 1] : kSentinelPad;
+    const uint32_t next_after = (base + kReduceTile < n) ? sk[base + kReduceTile] : kSentinelPad;
+    uint32_t next = __shfl_down_sync(full, key, 1);
+    if (lane == 31) next = next_after;
+    const unsigned head_mask = __ballot_sync(full, key != prev);
+    const unsigned usable_mask = __ballot_sync(full, usable);
+    const unsigned end_mask = __ballot_sync(full, usable && (key != next || lane == 31));
+    const int first_head = head_mask ? (__ffs(head_mask) - 1) : 32;
+    const uint32_t key31 = __shfl_sync(full, key, 31);
+    const bool runs_on = key31 < K && next_after == key31;
+    if (runs_on && head_mask != 0u && lane == 31)
+        starters[atomicAdd(starter_count, 1u)] = make_uint4(tile, key, (uint32_t)row, (uint32_t)(row >> 32));
+    const uint32_t group = blockIdx.x / (kGroupTiles / 8);
+    const uint64_t gpos = (uint64_t)group * kGroupTiles * kReduceTile;
+    uint32_t kg = kSentinelPad, kg_prev = kSentinelPad - 1, kg_far = kSentinelPad - 2;
+    if (gpos > 0 && gpos + kGroupMinSpan - 1 < n) {
+        kg = sk[gpos];
+        kg_prev = sk[gpos - 1];
+        kg_far = sk[gpos + kGroupMinSpan - 1];
+    }
+    const uint32_t L = L4 * 4;
+    // positions where the part of a segment that lies in this tile begins: its own row is fetched there
+    const bool begin_me = usable && (lane == 0 || key != prev);
+    const unsigned begin_mask = __ballot_sync(full, begin_me);
+    // positions whose segment ends here and lies wholly inside the tile: the new row is staged there
+    const bool stage_me = usable && (key != next || lane == 31) && !(lane < first_head || (lane == 31 && runs_on));
+    if (lane < n_valid) apply_row[base + lane] = stage_me ? row : ~0ull;
+    constexpr int G = reduce_group(kCh), ST = reduce_stages(kCh);
+    constexpr int kSlotF4 = 2 * G * kCh * 32;
+    extern __shared__ float4 stage_mem[];
+    float4* my_stage = stage_mem + (size_t)w * (ST * kSlotF4);
+    if (lane < ST) mbar_init(&bars[w][lane], 1);
+    mbar_init_fence();
+    __syncwarp();
+    const int n_groups = ((int)n_valid + G - 1) / G;
+    const unsigned gmask0 = (1u << G) - 1u;
+    const uint32_t chunk_bytes = L4 * 16u;           // rows of at most 32 kCh float4: one round
+    uint32_t uses = 0;
+    bool dead = false;
+    auto issue = [&](int g, int stage) {
+        if (g >= n_groups) return;
+        const unsigned gm = gmask0 << (g * G);
+        const uint32_t n_rows = __popc(usable_mask & gm) + __popc(begin_mask & gm);
+        if (n_rows == 0) return;
+        if (lane == g * G) mbar_expect_tx(&bars[w][stage], n_rows * chunk_bytes);
+        __syncwarp();
+        if ((gm >> lane) & 1u) {
+            float4* dst = my_stage + (size_t)stage * kSlotF4 + (size_t)(lane - g * G) * (2 * kCh * 32);
+            if (usable) bulk_g2s(dst, store + prow * L4, chunk_bytes, &bars[w][stage]);
+            if (begin_me) bulk_g2s(dst + kCh * 32, store + row * L4, chunk_bytes, &bars[w][stage]);
+        }
+    };
+#pragma unroll
+    for (int g = 0; g < ST - 1; ++g) issue(g, g);
+    d4 acc[kCh];
+    float4 own[kCh];
+#pragma unroll
+    for (int c = 0; c < kCh; ++c) {
+        acc[c] = d4{0.0, 0.0, 0.0, 0.0};
+        own[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float nw = 0.f;                                 // this lane's share of |own|^2
+    double loss = 0;                                // this lane's share of the tile's loss
+    int st_use = 0, st_fill = ST - 1;
+    for (int g = 0; g < n_groups; ++g) {
+        __syncwarp();
+        issue(g + ST - 1, st_fill);
+        const unsigned gm = gmask0 << (g * G);
+        const float4* slot = my_stage + (size_t)st_use * kSlotF4 + lane;
+        if (usable_mask & gm) {
+            const uint32_t parity = (uses >> st_use) & 1u;
+            if (!mbar_wait(&bars[w][st_use], parity) && !mbar_wait(&bars[w][st_use], parity)) {
+                if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
+                dead = true;
+                break;
+            }
+            uses ^= 1u << st_use;
+        }
+        st_use = st_use + 1 == ST ? 0 : st_use + 1;
+        st_fill = st_fill + 1 == ST ? 0 : st_fill + 1;
+#pragma unroll
+        for (int k = 0; k < G; ++k) {
+            const int p = g * G + k;
+            const float v = __shfl_sync(full, val, p);
+            if (!((usable_mask >> p) & 1u)) continue;
+            if ((begin_mask >> p) & 1u) {
+                nw = 0.f;
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    own[c] = lane + 32 * c < L4 ? slot[(k * 2 * kCh + kCh + c) * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
+                    nw += own[c].x * own[c].x + own[c].y * own[c].y + own[c].z * own[c].z + own[c].w * own[c].w;
+                }
+            }
+            float4 h[kCh];
+            float dot = 0.f, nh = 0.f;
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                h[c] = lane + 32 * c < L4 ? slot[(k * 2 * kCh + c) * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
+                dot += own[c].x * h[c].x + own[c].y * h[c].y + own[c].z * h[c].z + own[c].w * h[c].w;
+                nh += h[c].x * h[c].x + h[c].y * h[c].y + h[c].z * h[c].z + h[c].w * h[c].w;
+            }
+            dot = warp_sum(dot);
+            const float e = v - dot;
+            // the cell's loss: the lanes keep their shares of the two squared norms, lane 0 adds the squared error
+            if ((side0_mask >> p) & 1u) loss += (double)(0.5f * lam * (nw + nh) + (lane == 0 ? 0.5f * e * e : 0.f));
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                acc[c].x += (double)(lr * (e * h[c].x - lam * own[c].x));
+                acc[c].y += (double)(lr * (e * h[c].y - lam * own[c].y));
+                acc[c].z += (double)(lr * (e * h[c].z - lam * own[c].z));
+                acc[c].w += (double)(lr * (e * h[c].w - lam * own[c].w));
+            }
+            if (!((end_mask >> p) & 1u)) continue;
+            const bool from_prev = p < first_head;
+            const bool parked = from_prev || (p == 31 && runs_on);
+#pragma unroll
+            for (int c = 0; c < kCh; ++c) {
+                const uint32_t f = lane + 32 * c;
+                if (f < L4) {
+                    if (!parked) {
+                        float4 r = own[c];
+                        r.x = (float)((double)r.x + acc[c].x); r.y = (float)((double)r.y + acc[c].y);
+                        r.z = (float)((double)r.z + acc[c].z); r.w = (float)((double)r.w + acc[c].w);
+                        staged[(base + p) * L4 + f] = r;
+                    } else {
+                        double* cs = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
+                        *(double2*)cs = make_double2(acc[c].x, acc[c].y);
+                        *(double2*)(cs + 2) = make_double2(acc[c].z, acc[c].w);
+                    }
+                }
+                acc[c] = d4{0.0, 0.0, 0.0, 0.0};
+            }
+        }
+    }
+    __syncwarp();
+    (void)dead;
+    // per-block loss partial, fixed order
+    loss = warp_sum_d(loss);
+    if (lane == 0) wl[w] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0;
+        for (int i = 0; i < 8; ++i) t += wl[i];
+        loss_partial[blockIdx.x] = t;
+    }
+    if (!(kg < K && kg_prev == kg && kg_far == kg)) return;
+    group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
+                 &s_ticket);
+}
+
 // Warps work through the list of tiles that start a border-crossing segment, one segment per warp at a
 // time.  The warp finds the parked partials the segment has left behind (32 probes at a time): those of
 // the tiles it runs through in the starter's group, then one pre-added value per later group, then the
@@ -462,9 +656,44 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                   const double* __restrict__ carry, const double* __restrict__ group_sum,
                   const uint4* __restrict__ starters,
                   const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
-                  uint32_t loss_blocks, double* __restrict__ loss_accum, const DevStatus* st, unsigned int epoch) {
+                  uint32_t loss_blocks, double* __restrict__ loss_accum, uint32_t fix_blocks,
+                  const float4* __restrict__ staged, const uint64_t* __restrict__ apply_row,
+                  const DevStatus* st, unsigned int epoch) {
     if (call_failed(st, epoch)) return;
-    if (blockIdx.x == gridDim.x - 1) {
+    if (blockIdx.x > fix_blocks) {
+        // Blocks past the loss block move staged rows into the store (calls that stage rows only): a warp
+        // looks at 32 sorted positions at a time and copies the rows staged there, four in flight at once.
+        const unsigned full = 0xffffffffu;
+        const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+        const uint64_t stride = (uint64_t)(gridDim.x - fix_blocks - 1) * kFixupWarps * 32;
+        for (uint64_t b0 = ((uint64_t)(blockIdx.x - fix_blocks - 1) * kFixupWarps + w) * 32; b0 < n; b0 += stride) {
+            const uint64_t r = b0 + lane < n ? apply_row[b0 + lane] : ~0ull;
+            unsigned m = __ballot_sync(full, r != ~0ull);
+            while (m) {
+                int q[4];
+                uint64_t rr[4];
+                float4 x[4][kCh];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    q[a] = m ? __ffs(m) - 1 : -1;
+                    m &= m - 1;                              // 0 stays 0
+                    rr[a] = __shfl_sync(full, r, q[a] & 31);
+                }
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c)
+                        if (q[a] >= 0 && lane + 32 * c < L4) x[a][c] = staged[(b0 + q[a]) * L4 + lane + 32 * c];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c)
+                        if (q[a] >= 0 && lane + 32 * c < L4) store[rr[a] * L4 + lane + 32 * c] = x[a][c];
+            }
+        }
+        return;
+    }
+    if (blockIdx.x == fix_blocks) {
         if (loss_accum) {                           // fixed-shape sum: strided per thread, then a tree
             __shared__ double ws[kFixupWarps];
             double t = 0;
@@ -485,7 +714,7 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     const uint32_t count = *starter_count;
     const uint32_t L = L4 * 4;
     const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
-    const uint32_t n_warps = (gridDim.x - 1) * kFixupWarps;
+    const uint32_t n_warps = fix_blocks * kFixupWarps;
     // what a warp found out about its segment, for the block to share the work of a long one
     struct Walk {
         uint32_t tile, last_tile, group0, n_groups, rem_first, rem_cnt, is_long;
@@ -630,6 +859,59 @@ int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
                             div_up_u32(n, kGroupSpan));
 }
 
+// The launch that follows a reduction: finishes the border-crossing segments, adds the loss partials and,
+// for calls that staged new rows instead of writing them (apply), moves those into the store.
+static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d_loss_accum, uint32_t loss_blocks,
+                         bool apply, cudaStream_t s) {
+    const uint32_t tiles = div_up_u32(n, kReduceTile);
+    const uint32_t L4 = ps->cfg.row_len / 4;
+    // a warp per listed segment; there are fewer segments in the list than tiles
+    const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8);
+    const uint32_t apply_blocks = apply ? tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8) : 0;
+    const uint32_t grid = fix_blocks + 1 + apply_blocks;
+#define FIXUP_ARGS sk, n, (float4*)ps->store, ps->table, ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4,   \
+                   ps->carry, ps->group_sum, ps->starters, ps->starter_count, ps->loss_partial, loss_blocks,      \
+                   loss_blocks ? d_loss_accum : nullptr, fix_blocks, (const float4*)ps->upd, ps->apply_rows,      \
+                   ps->status, ps->epoch
+    if (L4 <= 32) PS_LAUNCH(ps, push_fixup_kernel<1>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else if (L4 <= 64) PS_LAUNCH(ps, push_fixup_kernel<2>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else if (L4 <= 96) PS_LAUNCH(ps, push_fixup_kernel<3>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
+    else PS_LAUNCH(ps, push_fixup_kernel<4>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
+#undef FIXUP_ARGS
+}
+
+// The MF step on sorted occurrences (which: buffer that holds the sort's result); rows of at most 512 values.
+void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
+                  uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, cudaStream_t s) {
+    const uint32_t* sk = which ? ps->keysB : ps->keysA;
+    const uint32_t* sv = which ? ps->valsB : ps->valsA;
+    const uint32_t n = 2 * n_cells;
+    const uint32_t tiles = div_up_u32(n, kReduceTile);
+    const uint32_t blocks = div_up_u32(tiles, 8);
+    const uint32_t L4 = ps->cfg.row_len / 4;
+#define FUSED_ARGS sk, sv, n, d_i, d_j, d_v, (uint32_t)col_key_base, lr, lambda, (const float4*)ps->store, ps->table, \
+                   ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, (float4*)ps->upd, ps->apply_rows,          \
+                   ps->carry, ps->starters, ps->starter_count, ps->group_done, ps->group_sum, ps->loss_partial,       \
+                   ps->status, ps->epoch
+#define FUSED_LAUNCH(kCh)                                                                                            \
+    do {                                                                                                             \
+        static bool smem_set = false;                                                                                \
+        if (!smem_set) {                                                                                             \
+            cudaFuncSetAttribute(mf_fused_kernel<kCh>, cudaFuncAttributeMaxDynamicSharedMemorySize,                  \
+                                 (int)reduce_smem(kCh));                                                             \
+            smem_set = true;                                                                                         \
+        }                                                                                                            \
+        PS_LAUNCH_SMEM(ps, mf_fused_kernel<kCh>, blocks, 256, reduce_smem(kCh), s, FUSED_ARGS);                      \
+    } while (0)
+    if (L4 <= 32) FUSED_LAUNCH(1);
+    else if (L4 <= 64) FUSED_LAUNCH(2);
+    else if (L4 <= 96) FUSED_LAUNCH(3);
+    else FUSED_LAUNCH(4);
+#undef FUSED_LAUNCH
+#undef FUSED_ARGS
+    launch_fixup(ps, sk, n, d_loss_accum, d_loss_accum ? blocks : 0, true, s);
+}
+
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
                      uint32_t loss_blocks, cudaStream_t s, const float* d_scales, uint32_t slots) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
@@ -666,16 +948,7 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     }
 #undef REDUCE_LAUNCH
 #undef REDUCE_ARGS
-    // a warp per listed segment; there are fewer segments in the list than tiles
-    const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8);
-#define FIXUP_ARGS sk, n, (float4*)ps->store, ps->table, ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4,   \
-                   ps->carry, ps->group_sum, ps->starters, ps->starter_count, ps->loss_partial, loss_blocks,      \
-                   loss_blocks ? d_loss_accum : nullptr, ps->status, ps->epoch
-    if (L4 <= 32) PS_LAUNCH(ps, push_fixup_kernel<1>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
-    else if (L4 <= 64) PS_LAUNCH(ps, push_fixup_kernel<2>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
-    else if (L4 <= 96) PS_LAUNCH(ps, push_fixup_kernel<3>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
-    else PS_LAUNCH(ps, push_fixup_kernel<4>, fix_blocks + 1, 32 * kFixupWarps, s, FIXUP_ARGS);
-#undef FIXUP_ARGS
+    launch_fixup(ps, sk, n, d_loss_accum, loss_blocks, false, s);
 }
 
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,

@@ -580,14 +580,20 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
 #pragma unroll
                     for (int a = 0; a < kQuad; ++a) x[a] += __shfl_xor_sync(full, x[a], o);
                 }
+                // lane a < 4 turns the a-th score of the four into the slot's factor and loss term
+                float xa = x[0];
+#pragma unroll
+                for (int a = 1; a < kQuad; ++a) xa = lane == a ? x[a] : xa;
+                float sc_mine = 0.f;
+                if (lane < kQuad && ((ok_mask >> (b + lane)) & 1u)) {
+                    const bool positive = (t0 + b + lane) % per_ctx == 0;
+                    sc_mine = -lr * (sigmoidf(xa) - (positive ? 1.f : 0.f));
+                    loss_c += positive ? softplusf(-xa) : softplusf(xa);
+                }
 #pragma unroll
                 for (int a = 0; a < kQuad; ++a) {
+                    const float sc = __shfl_sync(full, sc_mine, a);
                     if (!((ok_mask >> (b + a)) & 1u)) continue;
-                    const uint32_t tt = t0 + b + a;
-                    const bool positive = tt % per_ctx == 0;
-                    const float g = sigmoidf(x[a]) - (positive ? 1.f : 0.f);
-                    loss_c += positive ? softplusf(-x[a]) : softplusf(x[a]);
-                    const float sc = -lr * g;
                     if (lane == (int)(b + a)) my_scale = sc;
 #pragma unroll
                     for (int c = 0; c < kCh; ++c) {
@@ -608,9 +614,9 @@ sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64
             }
         }
         if (lane == 0) F[0] = 1.f;
-        loss += (double)loss_c;
+        loss += (double)loss_c;                             // this lane's share (lanes 0..3 hold the terms)
     }
-    block_loss_out(loss, loss_partial);
+    block_loss_out(warp_sum_d(loss), loss_partial);
 }
 
 // Keys of the occurrence slots of each center: slot 0 the center's input vector, then per context
