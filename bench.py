@@ -127,9 +127,6 @@ def kernel_bytes_of_step(batch_bytes, occ, u, rb, keys_prefix, step_prefix):
     batch, the table and the store, and what it has to write for the next kernel (keys, update rows)."""
     return {
         keys_prefix: batch_bytes + occ * 4,                      # batch arrays in, one 32-bit key per occurrence out
-        "sort_hist_kernel": occ * 4,
-        "sort_pass_kernel<true>": occ * 12,                      # keys in; keys and occurrence indices out
-        "sort_pass_kernel<false>": occ * 16,
         step_prefix: batch_bytes + occ * (8 + rb) + occ * rb,    # table entry + row per occurrence in, update row out
         "push_reduce_kernel": occ * (8 + rb) + u * (8 + 2 * rb), # sorted pair + update row in; row read-modify-write
     }

@@ -160,7 +160,7 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
     PS_LAUNCH(ps, loc_scan_sums_kernel, 1, 256, s, ps->scan_sums, blocks, ps->status, ps->epoch);
     PS_LAUNCH(ps, loc_assign_kernel, blocks, 256, s, sk, n, ps->table, worker, S, ps->tops, ps->stacks, sc.flag,
               ps->scan_sums, sc, owner_keys, ps->status, ps->epoch);
-    const int w2 = radix_sort_pairs(ps, n, &ps->status->moved_total, ps->owner_bits, true, s, which ^ 1, nullptr, 0);
+    const int w2 = radix_sort_pairs(ps, n, &ps->status->moved_total, ps->owner_bits, s, which ^ 1, nullptr, 0);
     const uint32_t* so = w2 ? ps->keysB : ps->keysA;
     const uint32_t* sv = w2 ? ps->valsB : ps->valsA;
     PS_LAUNCH(ps, loc_free_kernel, blocks, 256, s, so, sv, sc.mslot, ps->tops, ps->stacks, S, ps->status, ps->epoch);

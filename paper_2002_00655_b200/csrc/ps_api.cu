@@ -23,8 +23,11 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         return at;
     };
     const uint64_t mk = max_keys ? max_keys : 1;
-    const size_t sort_tiles = (mk + kSortTile - 1) / kSortTile;
-    const size_t reduce_tiles = (mk + kReduceTile - 1) / kReduceTile;
+    const size_t sort_tiles = (mk + kSortTile / 2 - 1) / (kSortTile / 2);   // the sort's blocks, at its shortest tile
+    // tiles of the reduction: 32 positions, or 8 for the matrix-factorization step on rows of at most 128 values
+    const size_t tile_len = cfg.row_len <= 128 ? 8 : kReduceTile;
+    const size_t reduce_tiles = (mk + tile_len - 1) / tile_len;
+    const size_t groups = (mk + tile_len * 64 - 1) / (tile_len * 64);
     const size_t row_bytes = (size_t)cfg.row_len * 4;
     l.status = take(sizeof(DevStatus));
     for (int b = 0; b < kSortSets; ++b) {
@@ -33,14 +36,15 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.valsA[b] = take(mk * 4);
         l.valsB[b] = take(mk * 4);
         l.tile_state[b] = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
-        l.sort_ctl[b] = take(((size_t)kSortCtlWords + (mk + kGroupSpan - 1) / kGroupSpan) * 4);
+        l.sort_ctl[b] = take(((size_t)kSortCtlWords + groups) * 4);
+        l.rec[b] = take(mk * 16);
         l.starters[b] = take(reduce_tiles * 16);
         l.starter_count[b] = take(4);
     }
     l.scan_sums = take(((mk + 255) / 256) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
-    l.group_sum = take(((mk + kGroupSpan - 1) / kGroupSpan) * (size_t)cfg.row_len * 8);
+    l.group_sum = take(groups * (size_t)cfg.row_len * 8);
     l.loss_partial = take(tmax<size_t>(kMaxLossBlocks, mk / 256 + 1) * 8);
     l.apply_rows = take(mk * 8);
     l.staging = take(mk * 8 + 256);
@@ -115,7 +119,7 @@ static SortSet* next_set(ps_store* ps) {
     SortSet* ss = &ps->sets[ps->cur_set];
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
     ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
-    ps->starters = ss->starters; ps->starter_count = ss->starter_count;
+    ps->starters = ss->starters; ps->starter_count = ss->starter_count; ps->rec = ss->rec;
     return ss;
 }
 
@@ -136,7 +140,10 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
     ps->capture_id = id;
     if (crossed)
         for (int b = 0; b < kSortSets; ++b) ps->sets[b].used = false;
-    if (ps->pipelined && !crossed) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
+    // a sort that reads the location table (the matrix-factorization records) must come after a call that rewrote it
+    const bool ordered = crossed || ps->table_dirty;
+    ps->table_dirty = false;
+    if (ps->pipelined && !ordered) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
@@ -189,6 +196,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->cfg = *cfg;
     ps->max_keys = max_batch_keys;
     ps->key_bits = bits_for(cfg->num_keys);                 // keys 0..K, K marks "no key"
+    ps->sort_blocks_cap = div_up_u32(max_batch_keys, kSortTile / 2);
     ps->owner_bits = bits_for(cfg->num_workers - 1);
     ps->store = (float*)d_store;
     ps->table = (uint2*)d_table;
@@ -207,6 +215,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.tile_state = (uint32_t*)(ps->ws + l.tile_state[b]);
         ss.sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl[b]);
         ss.group_done = ss.sort_ctl + kSortCtlWords;
+        ss.rec = (uint4*)(ps->ws + l.rec[b]);
         ss.starters = (uint4*)(ps->ws + l.starters[b]);
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;
@@ -230,6 +239,12 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         delete ps;
         return PS_ERR_CUDA;
     }
+    // the sort's grid barrier re-arms itself after every use, but has to start from zero
+    for (int b = 0; b < kSortSets; ++b)
+        if (cudaMemset(ps->sets[b].sort_ctl, 0, kSortCtlWords * sizeof(uint32_t)) != cudaSuccess) {
+            delete ps;
+            return PS_ERR_CUDA;
+        }
     // the side stream's small kernels should not queue behind the gradient kernel's waves of blocks
     int prio_lo = 0, prio_hi = 0;
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
@@ -269,6 +284,7 @@ ps_status_t ps_destroy(ps_store_t* ps) {
 ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
     PS_BEGIN_CALL(ps);
     launch_init_range_partition(ps, s);
+    ps->table_dirty = true;
     return after_launch();
 }
 
@@ -295,8 +311,8 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;         // the keys are sorted beside earlier calls' kernels
-    launch_prepare_keys(ps, d_keys, n, ps->side);
-    const int which = run_push_sort(ps, (uint32_t)n, ps->side);
+    const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, ps->starter_count,
+                                        div_up_u32(n, kGroupSpan));
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)n, which, d_updates, nullptr, 0, s);
     return release_set(ss, s);
@@ -310,10 +326,10 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
-    launch_prepare_keys(ps, d_keys, n, ps->side);
-    const int which = radix_sort_pairs(ps, (uint32_t)n, nullptr, ps->key_bits, true, ps->side, 0, nullptr, 0);
+    const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, nullptr, 0);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_localize(ps, worker, (uint32_t)n, which, s);
+    ps->table_dirty = true;
     return release_set(ss, s);
 }
 
@@ -326,12 +342,14 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
-    launch_keys_mf(ps, d_i, d_j, n, col_key_base, ps->side);
-    const int which = run_push_sort(ps, (uint32_t)(2 * n), ps->side);
-    if (ps->cfg.row_len <= 512) {
+    // rows short enough to be staged whole, and row numbers that fit the 32-bit fields of the sort's records
+    const bool fused = ps->cfg.row_len <= 128 && (uint64_t)ps->cfg.num_workers * ps->cfg.slots_per_part < (1ull << 32);
+    const int which = radix_sort_mf(ps, d_i, d_j, d_v, (uint32_t)n, col_key_base, fused, ps->side, ps->starter_count,
+                                    div_up_u32(2 * n, fused ? 64 * 8 : kGroupSpan));
+    if (fused) {
         // gradient and reduction in one kernel over the sorted occurrences: no update rows
         if (!join_side(ps, s)) return PS_ERR_CUDA;
-        run_mf_fused(ps, (uint32_t)n, which, d_i, d_j, d_v, col_key_base, lr, lambda, d_loss_accum, s);
+        run_mf_fused(ps, (uint32_t)n, which, col_key_base, lr, lambda, d_loss_accum, s);
         return release_set(ss, s);
     }
     const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
@@ -553,6 +571,11 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream) {
     unsigned int code = 0;
     if (cudaMemcpy(&code, &ps->status->sticky, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
     if (code != 0 && cudaMemset(&ps->status->sticky, 0, 4) != cudaSuccess) return PS_ERR_CUDA;
+    if (code == PS_ERR_CUDA) {                  // a sort that gave up inside its grid barrier leaves it mid-count
+        if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;
+        for (int b = 0; b < kSortSets; ++b)
+            if (cudaMemset(ps->sets[b].sort_ctl, 0, kSortCtlWords * sizeof(uint32_t)) != cudaSuccess) return PS_ERR_CUDA;
+    }
     return (ps_status_t)code;
 }
 

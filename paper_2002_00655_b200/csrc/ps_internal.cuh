@@ -44,6 +44,7 @@ struct SortSet {
     uint32_t* tile_state;
     uint32_t* sort_ctl;
     unsigned int* group_done;
+    uint4* rec;
     uint4* starters;
     unsigned int* starter_count;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
@@ -56,6 +57,7 @@ struct ps_store {
     ps_config_t cfg;
     uint64_t max_keys;
     int key_bits;                   // bits needed for keys 0..K inclusive (K is the "no key" mark)
+    uint32_t sort_blocks_cap;       // blocks the sort's digit counters (tile_state) have room for
     int owner_bits;
     // caller-owned device buffers
     float* store;
@@ -67,8 +69,9 @@ struct ps_store {
     // carved out of the workspace
     psb::DevStatus* status;
     uint32_t *keysA, *keysB, *valsA, *valsB;
-    uint32_t* tile_state;           // kMaxSortPasses x nSortTiles x kRadix look-back words
-    uint32_t* sort_ctl;             // kSortCtlWords, followed by group_done
+    uint32_t* tile_state;           // kMaxSortPasses x sort blocks x kRadix digit counters
+    uint32_t* sort_ctl;             // the sort's grid barrier (two words) in kSortCtlWords, followed by group_done
+    uint4* rec;                     // MF: {key, cell value, row of the key, row of the other factor} per sorted position
     unsigned int* group_done;       // per group of 64 reduction tiles: reduction blocks that have finished
     double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
@@ -89,6 +92,7 @@ struct ps_store {
     psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
     bool pipelined;                 // see ps_set_pipelining
+    bool table_dirty;               // the location table was rewritten since the side stream last waited for the caller's
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
 };
 
@@ -96,7 +100,7 @@ namespace psb {
 
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
-        sort_ctl[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        sort_ctl[kSortSets], rec[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
         loss_partial, apply_rows, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
@@ -126,15 +130,22 @@ void prof_after(ps_store* ps, cudaStream_t s);
     } while (0)
 
 // ---- sort.cu ----
-// Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key.
-// Input in the A buffers (start = 0) or the B buffers (start = 1); values are
-// implied as 0..n-1 when iota_vals.  If n_dev is not null the element count is
-// read from device memory (n is then an upper bound used for the launch
-// shapes).  Returns 0 if the result is in the A buffers, 1 if in the B buffers.
-// If zero_me is not null the first kernel also sets *zero_me = 0; the first `zero_groups` words of
-// group_done are cleared together with the sort's own control words.
-int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, bool iota_vals,
-                     cudaStream_t stream, int start, unsigned int* zero_me, uint32_t zero_groups);
+// Stable LSD radix sort of (key, value) pairs on the low `bits` bits of the key, one cooperative launch.
+// Values are the positions 0..n-1 of the input.  Input in the A buffers (start = 0) or the B buffers
+// (start = 1).  If n_dev is not null the element count is read from device memory (n is then an upper
+// bound used for the launch shape).  Returns 0 if the result is in the A buffers, 1 if in the B buffers.
+// Before its first grid barrier the kernel clears *zero_me (if not null) and the first `zero_groups`
+// words of group_done.
+int radix_sort_pairs(ps_store* ps, uint32_t n, const unsigned int* n_dev, int bits, cudaStream_t stream, int start,
+                     unsigned int* zero_me, uint32_t zero_groups);
+// the same on range-checked 64-bit caller keys (no separate key kernel); key_bits bits
+int radix_sort_keys64(ps_store* ps, const uint64_t* d_keys, uint32_t n, cudaStream_t stream, unsigned int* zero_me,
+                      uint32_t zero_groups);
+// the 2 n_cells occurrences of a batch of matrix cells (2t: row factor, 2t + 1: column factor), keys taken
+// from the batch arrays inside the sort; with `records` the last pass writes ps->rec beside the sorted keys
+int radix_sort_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint32_t n_cells,
+                  uint64_t col_key_base, bool records, cudaStream_t stream, unsigned int* zero_me,
+                  uint32_t zero_groups);
 
 // ---- pull_push.cu ----
 void launch_init_range_partition(ps_store* ps, cudaStream_t s);
@@ -158,8 +169,8 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
 
 // MF step working on the sorted occurrences directly (rows of at most 512 values): gradient, reduction,
 // then the fix-up launch that also moves the staged rows into the store
-void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
-                  uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, cudaStream_t s);
+void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
+                  double* d_loss_accum, cudaStream_t s);
 
 // ---- localize.cu ----
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
@@ -169,8 +180,6 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
 // only, so they and the sort can run beside the gradient kernel); launch_step_* write the slots'
 // update rows to `upd` (launch_step_sgns: two source rows per center and one factor per slot, to be
 // reduced with run_push_reduce's d_scales) and return the number of per-block loss partials they wrote.
-void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint64_t n, uint64_t col_key_base,
-                    cudaStream_t s);
 void launch_keys_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                      const uint32_t* d_neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_key_base, cudaStream_t s);
 void launch_keys_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,

@@ -227,18 +227,18 @@ constexpr int kGroupTiles = 64;     // tiles whose parked parts are pre-added pe
 __device__ __noinline__ void group_preadd(const uint32_t* __restrict__ sk, uint32_t n, uint32_t L4,
                                           const double* __restrict__ carry, unsigned int* __restrict__ group_done,
                                           double* __restrict__ group_sum, uint32_t group, uint64_t gpos, uint32_t kg,
-                                          d4 (*gpart)[32], unsigned int* s_ticket) {
+                                          d4 (*gpart)[32], unsigned int* s_ticket, uint32_t tile_len,
+                                          uint32_t arrivals) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t L = L4 * 4;
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) *s_ticket = atomicAdd(&group_done[group], 1u);
     __syncthreads();
-    const uint32_t blocks_in_group = tmin<uint32_t>(kGroupTiles / 8, gridDim.x - group * (kGroupTiles / 8));
-    if (*s_ticket != blocks_in_group - 1) return;
+    if (*s_ticket != arrivals - 1) return;              // `arrivals` blocks work on the group's tiles
     __threadfence();
     // tiles of the group that begin with the entering segment's key: a prefix of the group's tiles
-    const uint64_t tpos = gpos + (uint64_t)threadIdx.x * kReduceTile;
+    const uint64_t tpos = gpos + (uint64_t)threadIdx.x * tile_len;
     const int hit = threadIdx.x < kGroupTiles && tpos < n && sk[tpos] == kg;
     const uint32_t m = (uint32_t)__syncthreads_count(hit);
     const uint32_t t0 = group * kGroupTiles;
@@ -445,201 +445,239 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
     if (!(kg < K && kg_prev == kg && kg_far == kg)) return;     // nothing to pre-add for this group
     // the staging memory is free by now (every warp has waited for all its copies) and serves as scratch
     group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
-                 &s_ticket);
+                 &s_ticket, kReduceTile, tmin<uint32_t>(kGroupTiles / 8, gridDim.x - group * (kGroupTiles / 8)));
 }
 
 // ------------------------------------------------- MF: gradient inside the reduction ----
 // One minibatch of matrix factorization without update rows.  The occurrences (2t: row factor of cell t,
-// 2t + 1: its column factor) arrive sorted by key, as for a push.  For every sorted position the warp
-// fetches the PARTNER row (the other factor of the cell) and, where a segment's part in the tile begins,
-// the key's own row; e = v - <own, partner> is formed on the spot and lr (e partner - lambda own) is
-// added, in fp64, to the segment's sum.  Since other warps still read rows as they were before the call,
-// nothing is written to the store here: a segment that lies inside the tile leaves its new row in
-// `staged` (indexed by the sorted position of its end) and the row's address in `apply_row`; the
-// fix-up launch, which runs after every read of this kernel, moves those rows in and finishes the
-// segments that cross tile borders from their parked partial sums, exactly as for a push.
-// The loss of a cell is taken at its row-factor occurrence.
-template <int kCh>
-__global__ void __launch_bounds__(256)
-mf_fused_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
-                const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, const float* __restrict__ cv,
-                uint32_t col_base, float lr, float lam, const float4* __restrict__ store,
-                const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
-                float4* __restrict__ staged, uint64_t* __restrict__ apply_row, double* __restrict__ carry,
-                uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
-                unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
-                double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
+// 2t + 1: its column factor) arrive sorted by key, as for a push, each with a record {key, value of the
+// cell, row of the key, row of the cell's other factor} written by the sort.  For every sorted position
+// the PARTNER row (the other factor) is fetched and, where a segment's part in a tile begins, the key's
+// own row; e = v - <own, partner> is formed on the spot and lr (e partner - lambda own) is added to the
+// segment's sum.
+//
+// The kernel is bound by instruction issue, not by memory, if a whole warp works on one position (a row
+// of 100 values keeps 25 lanes busy for one instruction while the bookkeeping of the position costs
+// dozens).  So a position is handled by EIGHT lanes: a warp covers 32 consecutive positions as four tiles
+// of kMfTile = 8 positions, one per group of eight lanes, and every instruction of the walk serves four
+// positions.  A lane holds every eighth float4 of a row.  Tiles of eight positions are the unit of the
+// border logic: a segment's part that crosses a tile border parks its fp64 partial sum (slot 0 of the tile
+// it enters, slot 1 of the tile it leaves) and the fix-up launch adds the parts up, as for a push.
+// A segment of exactly one position needs no fp64 sum: own + update is formed in fp32, which rounds the
+// same exact sum once.
+//
+// Column-factor keys sort after row-factor keys, so the two sides are two ranges of positions, and the
+// step runs this kernel twice.  First the column side: it reads row factors as partners and leaves its new
+// rows in `staged` (the fix-up launch moves them into the store).  Then the row side: its partners are
+// column factors, which nothing has overwritten, and nobody reads a row factor any more except the group
+// that owns its segment, so new rows go straight into the store.  The loss of a cell is taken at its
+// row-factor occurrence.
+constexpr int kMfTile = 8;
+constexpr int kMfStages = 3;
+constexpr size_t kMfSmem = (size_t)8 * kMfStages * 4 * 64 * sizeof(float4);     // warp x stage x group x {partner, own}
+
+enum : uint32_t { kFUsable = 1, kFBegin = 2, kFEnd = 4, kFParked = 8, kFFromPrev = 16, kFSide0 = 32, kFSingle = 64 };
+
+template <int kC>
+__global__ void __launch_bounds__(256, 2)
+mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, uint32_t n, uint32_t lo, uint32_t hi,
+              uint32_t first_block, int in_place, uint32_t col_base, float lr, float lam, float4* store, uint32_t K,
+              uint32_t L4, float4* __restrict__ staged, uint64_t* __restrict__ apply_row, double* __restrict__ carry,
+              uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
+              unsigned int* __restrict__ group_done, double* __restrict__ group_sum, uint32_t extra_group,
+              double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
     __shared__ unsigned int s_ticket;
-    __shared__ __align__(8) uint64_t bars[8][3];
+    __shared__ __align__(8) uint64_t bars[8][kMfStages];
     __shared__ double wl[8];
+    extern __shared__ float4 stage_mem[];
     if (call_failed(st, epoch)) return;
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t base = (uint64_t)tile * kReduceTile;
-    const uint32_t n_valid = base < n ? (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base) : 0u;
-    const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
-    const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
-    const bool usable = key < K;                    // cells with a key out of range carry the "no key" mark
-    uint64_t row = 0, prow = 0;
-    float val = 0.f;
-    if (usable) {
-        const uint32_t t = occ >> 1;
-        const uint32_t pkey = (occ & 1u) ? ci[t] : col_base + cj[t];
-        val = cv[t];
-        row = phys_row(table[key], S);
-        prow = phys_row(table[pkey], S);            // in range: the key extraction marked the cell otherwise
-    }
-    const unsigned side0_mask = __ballot_sync(full, usable && !(occ & 1u));
+    const int sg = lane >> 3, l8 = lane & 7;
+    const uint32_t gb = first_block + blockIdx.x;                   // block number over all sorted positions
+    const uint32_t tile32 = gb * 8 + w;
+    const uint64_t base = (uint64_t)tile32 * 32;
+    const uint64_t pos = base + lane;
+    const bool inside = pos >= lo && pos < hi;                      // hi <= n
+    const uint4 me = inside ? rec[pos] : make_uint4(kSentinelPad, 0u, 0u, 0u);
+    const uint32_t key = me.x;
+    const bool usable = key < K;
+    const float val = __uint_as_float(me.y);
+    const uint32_t row = me.z, prow = me.w;
     uint32_t prev = __shfl_up_sync(full, key, 1);
     if (lane == 0) prev = (base > 0 && base - 1 < n) ? sk[base - 1] : kSentinelPad;
-    const uint32_t next_after = (base + kReduceTile < n) ? sk[base + kReduceTile] : kSentinelPad;
     uint32_t next = __shfl_down_sync(full, key, 1);
-    if (lane == 31) next = next_after;
-    const unsigned head_mask = __ballot_sync(full, key != prev);
+    if (lane == 31) next = (base + 32 < n) ? sk[base + 32] : kSentinelPad;
+    const bool head = key != prev;
+    const unsigned head_mask = __ballot_sync(full, head);
     const unsigned usable_mask = __ballot_sync(full, usable);
-    const unsigned end_mask = __ballot_sync(full, usable && (key != next || lane == 31));
-    const int first_head = head_mask ? (__ffs(head_mask) - 1) : 32;
-    const uint32_t key31 = __shfl_sync(full, key, 31);
-    const bool runs_on = key31 < K && next_after == key31;
-    if (runs_on && head_mask != 0u && lane == 31)
-        starters[atomicAdd(starter_count, 1u)] = make_uint4(tile, key, (uint32_t)row, (uint32_t)(row >> 32));
-    const uint32_t group = blockIdx.x / (kGroupTiles / 8);
-    const uint64_t gpos = (uint64_t)group * kGroupTiles * kReduceTile;
+    // the head of this position's segment, if it lies in the warp's 32 positions
+    const unsigned at_or_below = head_mask & (0xffffffffu >> (31 - lane));
+    const int seg_head = at_or_below ? 31 - __clz(at_or_below) : -1;
+    const bool from_prev = usable && seg_head < 8 * sg;             // the segment came in from an earlier tile
+    const bool begin_me = usable && (l8 == 0 || head);              // the own row is fetched here
+    const bool end_me = usable && (l8 == 7 || key != next);         // the segment's part in the tile ends here
+    const bool runs_on = end_me && key == next;                     // ... and goes on in the next tile
+    const bool parked = end_me && (from_prev || runs_on);
+    const bool stage_me = end_me && !parked;                        // a whole segment ends here: new row
+    const uint32_t tile8 = tile32 * 4 + sg;
+    if (runs_on && !from_prev) starters[atomicAdd(starter_count, 1u)] = make_uint4(tile8, key, row, 0u);
+    if (!in_place && inside) apply_row[pos] = stage_me ? (uint64_t)row : ~0ull;
+    const unsigned begin_mask = __ballot_sync(full, begin_me);
+    const uint32_t flags = (usable ? kFUsable : 0u) | (begin_me ? kFBegin : 0u) | (end_me ? kFEnd : 0u) |
+                           (parked ? kFParked : 0u) | (from_prev ? kFFromPrev : 0u) |
+                           ((usable && key < col_base) ? kFSide0 : 0u) | ((begin_me && stage_me) ? kFSingle : 0u);
+    // where a finished row goes: the store row (row side) or the staging row of the position (column side)
+    const uint64_t dst_row = in_place ? (uint64_t)row : pos;
+    // does a long segment enter this block's group of 64 tiles from the group before?
+    constexpr uint32_t kTilesPerBlock = 8 * 4;
+    const uint32_t group = gb / (kGroupTiles / kTilesPerBlock);
+    const uint64_t gpos = (uint64_t)group * kGroupTiles * kMfTile;
     uint32_t kg = kSentinelPad, kg_prev = kSentinelPad - 1, kg_far = kSentinelPad - 2;
-    if (gpos > 0 && gpos + kGroupMinSpan - 1 < n) {
+    if (gpos > 0 && gpos + 8 * kMfTile - 1 < n) {
         kg = sk[gpos];
         kg_prev = sk[gpos - 1];
-        kg_far = sk[gpos + kGroupMinSpan - 1];
+        kg_far = sk[gpos + 8 * kMfTile - 1];
     }
     const uint32_t L = L4 * 4;
-    // positions where the part of a segment that lies in this tile begins: its own row is fetched there
-    const bool begin_me = usable && (lane == 0 || key != prev);
-    const unsigned begin_mask = __ballot_sync(full, begin_me);
-    // positions whose segment ends here and lies wholly inside the tile: the new row is staged there
-    const bool stage_me = usable && (key != next || lane == 31) && !(lane < first_head || (lane == 31 && runs_on));
-    if (lane < n_valid) apply_row[base + lane] = stage_me ? row : ~0ull;
-    constexpr int G = reduce_group(kCh), ST = reduce_stages(kCh);
-    constexpr int kSlotF4 = 2 * G * kCh * 32;
-    extern __shared__ float4 stage_mem[];
-    float4* my_stage = stage_mem + (size_t)w * (ST * kSlotF4);
-    if (lane < ST) mbar_init(&bars[w][lane], 1);
+    float4* my_stage = stage_mem + (size_t)w * (kMfStages * 4 * 64);
+    // Rows reach shared memory as bulk asynchronous copies of whole rows, issued by the lane that holds the
+    // position; all copies of a walk step report to one barrier word of the warp.  (Per-lane 16-byte
+    // asynchronous copies were measured too: 26 and 43 us per side against 20 and 20 with bulk copies.)
+    if (lane < kMfStages) mbar_init(&bars[w][lane], 1);
     mbar_init_fence();
     __syncwarp();
-    const int n_groups = ((int)n_valid + G - 1) / G;
-    const unsigned gmask0 = (1u << G) - 1u;
-    const uint32_t chunk_bytes = L4 * 16u;           // rows of at most 32 kCh float4: one round
-    uint32_t uses = 0;
-    bool dead = false;
-    auto issue = [&](int g, int stage) {
-        if (g >= n_groups) return;
-        const unsigned gm = gmask0 << (g * G);
-        const uint32_t n_rows = __popc(usable_mask & gm) + __popc(begin_mask & gm);
+    const uint32_t row_bytes = L4 * 16u;
+    // asks for the rows of the four positions of walk step s2 (one per group)
+    auto issue = [&](int s2, int stage) {
+        if (s2 >= kMfTile) return;
+        const unsigned sm = 0x01010101u << s2;
+        const uint32_t n_rows = __popc(usable_mask & sm) + __popc(begin_mask & sm);
         if (n_rows == 0) return;
-        if (lane == g * G) mbar_expect_tx(&bars[w][stage], n_rows * chunk_bytes);
+        if (lane == 0) mbar_expect_tx(&bars[w][stage], n_rows * row_bytes);
         __syncwarp();
-        if ((gm >> lane) & 1u) {
-            float4* dst = my_stage + (size_t)stage * kSlotF4 + (size_t)(lane - g * G) * (2 * kCh * 32);
-            if (usable) bulk_g2s(dst, store + prow * L4, chunk_bytes, &bars[w][stage]);
-            if (begin_me) bulk_g2s(dst + kCh * 32, store + row * L4, chunk_bytes, &bars[w][stage]);
+        if (l8 == s2 && usable) {
+            float4* dst = my_stage + (size_t)(stage * 4 + sg) * 64;
+            bulk_g2s(dst, store + (uint64_t)prow * L4, row_bytes, &bars[w][stage]);
+            if (begin_me) bulk_g2s(dst + 32, store + (uint64_t)row * L4, row_bytes, &bars[w][stage]);
         }
     };
 #pragma unroll
-    for (int g = 0; g < ST - 1; ++g) issue(g, g);
-    d4 acc[kCh];
-    float4 own[kCh];
+    for (int s2 = 0; s2 < kMfStages - 1; ++s2) issue(s2, s2);
+    d4 acc[kC];
+    float4 own[kC];
 #pragma unroll
-    for (int c = 0; c < kCh; ++c) {
+    for (int c = 0; c < kC; ++c) {
         acc[c] = d4{0.0, 0.0, 0.0, 0.0};
         own[c] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    float nw = 0.f;                                 // this lane's share of |own|^2
-    double loss = 0;                                // this lane's share of the tile's loss
-    int st_use = 0, st_fill = ST - 1;
-    for (int g = 0; g < n_groups; ++g) {
-        __syncwarp();
-        issue(g + ST - 1, st_fill);
-        const unsigned gm = gmask0 << (g * G);
-        const float4* slot = my_stage + (size_t)st_use * kSlotF4 + lane;
-        if (usable_mask & gm) {
+    float nw = 0.f, loss_f = 0.f;                   // this lane's share of |own|^2 and of the tile's loss
+    uint32_t uses = 0;
+    int st_use = 0, st_fill = kMfStages - 1;
+#pragma unroll 1
+    for (int s2 = 0; s2 < kMfTile; ++s2) {
+        __syncwarp();                               // every lane is done reading the stage to be refilled
+        issue(s2 + kMfStages - 1, st_fill);
+        const unsigned sm = 0x01010101u << s2;
+        if (usable_mask & sm) {
             const uint32_t parity = (uses >> st_use) & 1u;
             if (!mbar_wait(&bars[w][st_use], parity) && !mbar_wait(&bars[w][st_use], parity)) {
                 if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
-                dead = true;
-                break;
+                break;                              // a copy that does not arrive: give the call up
             }
             uses ^= 1u << st_use;
         }
-        st_use = st_use + 1 == ST ? 0 : st_use + 1;
-        st_fill = st_fill + 1 == ST ? 0 : st_fill + 1;
+        const float4* slot = my_stage + (size_t)(st_use * 4 + sg) * 64 + l8;
+        st_use = st_use + 1 == kMfStages ? 0 : st_use + 1;
+        st_fill = st_fill + 1 == kMfStages ? 0 : st_fill + 1;
+        const int src = 8 * sg + s2;
+        const uint32_t f = __shfl_sync(full, flags, src);
+        const float v = __shfl_sync(full, val, src);
+        const uint64_t drow = __shfl_sync(full, dst_row, src);
+        const bool live = f & kFUsable;
+        if (f & kFBegin) {
+            nw = 0.f;
 #pragma unroll
-        for (int k = 0; k < G; ++k) {
-            const int p = g * G + k;
-            const float v = __shfl_sync(full, val, p);
-            if (!((usable_mask >> p) & 1u)) continue;
-            if ((begin_mask >> p) & 1u) {
-                nw = 0.f;
+            for (int c = 0; c < kC; ++c) {
+                own[c] = (uint32_t)(l8 + 8 * c) < L4 ? slot[32 + 8 * c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                nw += own[c].x * own[c].x + own[c].y * own[c].y + own[c].z * own[c].z + own[c].w * own[c].w;
+                acc[c] = d4{0.0, 0.0, 0.0, 0.0};
+            }
+        }
+        float4 h[kC];
+        float dot = 0.f, nh = 0.f;
 #pragma unroll
-                for (int c = 0; c < kCh; ++c) {
-                    own[c] = lane + 32 * c < L4 ? slot[(k * 2 * kCh + kCh + c) * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
-                    nw += own[c].x * own[c].x + own[c].y * own[c].y + own[c].z * own[c].z + own[c].w * own[c].w;
+        for (int c = 0; c < kC; ++c) {
+            h[c] = (live && (uint32_t)(l8 + 8 * c) < L4) ? slot[8 * c] : make_float4(0.f, 0.f, 0.f, 0.f);
+            dot += own[c].x * h[c].x + own[c].y * h[c].y + own[c].z * h[c].z + own[c].w * h[c].w;
+            nh += h[c].x * h[c].x + h[c].y * h[c].y + h[c].z * h[c].z + h[c].w * h[c].w;
+        }
+        dot += __shfl_xor_sync(full, dot, 1);
+        dot += __shfl_xor_sync(full, dot, 2);
+        dot += __shfl_xor_sync(full, dot, 4);
+        const float e = v - dot;
+        // the cell's loss: the lanes keep their shares of the two squared norms, one lane adds the squared error
+        if (f & kFSide0) loss_f += 0.5f * lam * (nw + nh) + (l8 == 0 ? 0.5f * e * e : 0.f);
+        if (f & kFSingle) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                if ((uint32_t)(l8 + 8 * c) < L4) {
+                    float4 r;
+                    r.x = own[c].x + lr * (e * h[c].x - lam * own[c].x);
+                    r.y = own[c].y + lr * (e * h[c].y - lam * own[c].y);
+                    r.z = own[c].z + lr * (e * h[c].z - lam * own[c].z);
+                    r.w = own[c].w + lr * (e * h[c].w - lam * own[c].w);
+                    if (in_place) store[drow * L4 + l8 + 8 * c] = r;
+                    else staged[drow * L4 + l8 + 8 * c] = r;
                 }
             }
-            float4 h[kCh];
-            float dot = 0.f, nh = 0.f;
+        } else if (live) {
 #pragma unroll
-            for (int c = 0; c < kCh; ++c) {
-                h[c] = lane + 32 * c < L4 ? slot[(k * 2 * kCh + c) * 32] : make_float4(0.f, 0.f, 0.f, 0.f);
-                dot += own[c].x * h[c].x + own[c].y * h[c].y + own[c].z * h[c].z + own[c].w * h[c].w;
-                nh += h[c].x * h[c].x + h[c].y * h[c].y + h[c].z * h[c].z + h[c].w * h[c].w;
-            }
-            dot = warp_sum(dot);
-            const float e = v - dot;
-            // the cell's loss: the lanes keep their shares of the two squared norms, lane 0 adds the squared error
-            if ((side0_mask >> p) & 1u) loss += (double)(0.5f * lam * (nw + nh) + (lane == 0 ? 0.5f * e * e : 0.f));
-#pragma unroll
-            for (int c = 0; c < kCh; ++c) {
+            for (int c = 0; c < kC; ++c) {
                 acc[c].x += (double)(lr * (e * h[c].x - lam * own[c].x));
                 acc[c].y += (double)(lr * (e * h[c].y - lam * own[c].y));
                 acc[c].z += (double)(lr * (e * h[c].z - lam * own[c].z));
                 acc[c].w += (double)(lr * (e * h[c].w - lam * own[c].w));
             }
-            if (!((end_mask >> p) & 1u)) continue;
-            const bool from_prev = p < first_head;
-            const bool parked = from_prev || (p == 31 && runs_on);
+            if (f & kFEnd) {
 #pragma unroll
-            for (int c = 0; c < kCh; ++c) {
-                const uint32_t f = lane + 32 * c;
-                if (f < L4) {
-                    if (!parked) {
+                for (int c = 0; c < kC; ++c) {
+                    const uint32_t fi = l8 + 8 * c;
+                    if (fi >= L4) continue;
+                    if (f & kFParked) {
+                        double* cs = carry + ((uint64_t)tile8 * 2 + ((f & kFFromPrev) ? 0 : 1)) * L + (uint64_t)fi * 4;
+                        *(double2*)cs = make_double2(acc[c].x, acc[c].y);
+                        *(double2*)(cs + 2) = make_double2(acc[c].z, acc[c].w);
+                    } else {
                         float4 r = own[c];
                         r.x = (float)((double)r.x + acc[c].x); r.y = (float)((double)r.y + acc[c].y);
                         r.z = (float)((double)r.z + acc[c].z); r.w = (float)((double)r.w + acc[c].w);
-                        staged[(base + p) * L4 + f] = r;
-                    } else {
-                        double* cs = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L + (uint64_t)f * 4;
-                        *(double2*)cs = make_double2(acc[c].x, acc[c].y);
-                        *(double2*)(cs + 2) = make_double2(acc[c].z, acc[c].w);
+                        if (in_place) store[drow * L4 + fi] = r;
+                        else staged[drow * L4 + fi] = r;
                     }
                 }
-                acc[c] = d4{0.0, 0.0, 0.0, 0.0};
             }
         }
     }
-    __syncwarp();
-    (void)dead;
-    // per-block loss partial, fixed order
-    loss = warp_sum_d(loss);
-    if (lane == 0) wl[w] = loss;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        double t = 0;
-        for (int i = 0; i < 8; ++i) t += wl[i];
-        loss_partial[blockIdx.x] = t;
+    __syncthreads();                                // the staging memory is scratch from here on
+    // per-block loss partial, fixed order (only the row side has loss terms)
+    if (in_place) {
+        const double lw = warp_sum_d((double)loss_f);
+        if (lane == 0) wl[w] = lw;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double t = 0;
+            for (int i = 0; i < 8; ++i) t += wl[i];
+            loss_partial[gb] = t;
+        }
     }
     if (!(kg < K && kg_prev == kg && kg_far == kg)) return;
+    // blocks that work on the group's tiles: those of the launch, plus one if a block runs in both launches
+    const uint32_t n_blocks_all = (uint32_t)(((uint64_t)n + 255) / 256);
+    const uint32_t arrivals = tmin<uint32_t>(kGroupTiles / kTilesPerBlock, n_blocks_all - group * (kGroupTiles / kTilesPerBlock)) +
+                              (group == extra_group ? 1u : 0u);
     group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
-                 &s_ticket);
+                 &s_ticket, kMfTile, arrivals);
 }
 
 // Warps work through the list of tiles that start a border-crossing segment, one segment per warp at a
@@ -657,8 +695,8 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                   const uint4* __restrict__ starters,
                   const unsigned int* __restrict__ starter_count, const double* __restrict__ loss_partial,
                   uint32_t loss_blocks, double* __restrict__ loss_accum, uint32_t fix_blocks,
-                  const float4* __restrict__ staged, const uint64_t* __restrict__ apply_row,
-                  const DevStatus* st, unsigned int epoch) {
+                  const float4* __restrict__ staged, const uint64_t* __restrict__ apply_row, uint32_t tile_len,
+                  uint32_t apply_lo, const DevStatus* st, unsigned int epoch) {
     if (call_failed(st, epoch)) return;
     if (blockIdx.x > fix_blocks) {
         // Blocks past the loss block move staged rows into the store (calls that stage rows only): a warp
@@ -666,26 +704,27 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
         const unsigned full = 0xffffffffu;
         const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
         const uint64_t stride = (uint64_t)(gridDim.x - fix_blocks - 1) * kFixupWarps * 32;
-        for (uint64_t b0 = ((uint64_t)(blockIdx.x - fix_blocks - 1) * kFixupWarps + w) * 32; b0 < n; b0 += stride) {
+        for (uint64_t b0 = apply_lo + ((uint64_t)(blockIdx.x - fix_blocks - 1) * kFixupWarps + w) * 32; b0 < n; b0 += stride) {
             const uint64_t r = b0 + lane < n ? apply_row[b0 + lane] : ~0ull;
             unsigned m = __ballot_sync(full, r != ~0ull);
+            constexpr int kFly = kCh == 1 ? 8 : 4;           // rows in flight per warp
             while (m) {
-                int q[4];
-                uint64_t rr[4];
-                float4 x[4][kCh];
+                int q[kFly];
+                uint64_t rr[kFly];
+                float4 x[kFly][kCh];
 #pragma unroll
-                for (int a = 0; a < 4; ++a) {
+                for (int a = 0; a < kFly; ++a) {
                     q[a] = m ? __ffs(m) - 1 : -1;
                     m &= m - 1;                              // 0 stays 0
                     rr[a] = __shfl_sync(full, r, q[a] & 31);
                 }
 #pragma unroll
-                for (int a = 0; a < 4; ++a)
+                for (int a = 0; a < kFly; ++a)
 #pragma unroll
                     for (int c = 0; c < kCh; ++c)
-                        if (q[a] >= 0 && lane + 32 * c < L4) x[a][c] = staged[(b0 + q[a]) * L4 + lane + 32 * c];
+                        if (q[a] >= 0 && lane + 32 * c < L4) x[a][c] = __ldcs(staged + (b0 + q[a]) * L4 + lane + 32 * c);
 #pragma unroll
-                for (int a = 0; a < 4; ++a)
+                for (int a = 0; a < kFly; ++a)
 #pragma unroll
                     for (int c = 0; c < kCh; ++c)
                         if (q[a] >= 0 && lane + 32 * c < L4) store[rr[a] * L4 + lane + 32 * c] = x[a][c];
@@ -713,7 +752,8 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const uint32_t count = *starter_count;
     const uint32_t L = L4 * 4;
-    const uint32_t n_tiles = (uint32_t)(((uint64_t)n + kReduceTile - 1) / kReduceTile);
+    const uint32_t n_tiles = (uint32_t)(((uint64_t)n + tile_len - 1) / tile_len);
+    const uint32_t min_span = 8 * tile_len;                 // shortest entering segment a group pre-adds
     const uint32_t n_warps = fix_blocks * kFixupWarps;
     // what a warp found out about its segment, for the block to share the work of a long one
     struct Walk {
@@ -734,12 +774,42 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             }
         }
     };
-    // adds parked partial number i of the walk (tiles of the starter's group, then groups, then the rest)
-    auto add_nth = [&](d4* a, uint32_t f0, const Walk& k, uint32_t i) {
+    // where parked partial number i of the walk lies (tiles of the starter's group, then groups, then the rest)
+    auto nth = [&](const Walk& k, uint32_t i) -> const double* {
         const uint32_t n1 = k.last_tile - k.tile;
-        if (i < n1) add(a, f0, carry + ((uint64_t)(k.tile + 1 + i) * 2) * L);
-        else if (i < n1 + k.n_groups) add(a, f0, group_sum + ((uint64_t)k.group0 + (i - n1)) * L);
-        else add(a, f0, carry + ((uint64_t)(k.rem_first + (i - n1 - k.n_groups)) * 2) * L);
+        if (i < n1) return carry + ((uint64_t)(k.tile + 1 + i) * 2) * L;
+        if (i < n1 + k.n_groups) return group_sum + ((uint64_t)k.group0 + (i - n1)) * L;
+        return carry + ((uint64_t)(k.rem_first + (i - n1 - k.n_groups)) * 2) * L;
+    };
+    // Adds partials number i0, i0 + stride, ... (below n_parts) to a[], in that order; kB of them are requested
+    // together before the first is added, so a walk costs one round trip per kB partials.
+    constexpr int kB = kCh == 1 ? 8 : (kCh == 2 ? 4 : 2);
+    auto add_range = [&](d4* a, uint32_t f0, const Walk& k, uint32_t i0, uint32_t stride, uint32_t n_parts) {
+        for (uint32_t i = i0; i < n_parts; i += kB * stride) {
+            double2 x[kB][kCh], y[kB][kCh];
+#pragma unroll
+            for (int b = 0; b < kB; ++b) {
+                const uint32_t ib = i + b * stride;
+                const double* base = nth(k, ib < n_parts ? ib : i);
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    const uint32_t f = f0 + lane + 32 * c;
+                    x[b][c] = y[b][c] = make_double2(0.0, 0.0);
+                    if (ib < n_parts && f < L4) {
+                        x[b][c] = *(const double2*)(base + (uint64_t)f * 4);
+                        y[b][c] = *(const double2*)(base + (uint64_t)f * 4 + 2);
+                    }
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < kB; ++b) {
+                if (i + b * stride >= n_parts) break;
+#pragma unroll
+                for (int c = 0; c < kCh; ++c) {
+                    a[c].x += x[b][c].x; a[c].y += x[b][c].y; a[c].z += y[b][c].x; a[c].w += y[b][c].y;
+                }
+            }
+        }
     };
     for (uint32_t s0 = blockIdx.x * kFixupWarps; s0 < count; s0 += n_warps) {      // same trip count for all warps
         const uint32_t si = s0 + w;
@@ -757,7 +827,7 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             k.last_tile = k.tile;
             for (uint32_t t0 = k.tile + 1; t0 < walk_end; t0 += 32) {
                 const uint32_t t2 = t0 + lane;
-                const unsigned m = __ballot_sync(full, t2 < walk_end && sk[(uint64_t)t2 * kReduceTile] == kl);
+                const unsigned m = __ballot_sync(full, t2 < walk_end && sk[(uint64_t)t2 * tile_len] == kl);
                 k.last_tile += (uint32_t)__popc(m);
                 if (m != full) break;
             }
@@ -765,16 +835,16 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             if (k.last_tile + 1 == group_end) {
                 for (;;) {
                     const uint64_t g2 = (uint64_t)k.group0 + k.n_groups + lane;
-                    const uint64_t gp = g2 * kGroupTiles * kReduceTile;
+                    const uint64_t gp = g2 * kGroupTiles * tile_len;
                     const unsigned m = __ballot_sync(
-                        full, gp + kGroupMinSpan - 1 < n && sk[gp] == kl && sk[gp + kGroupMinSpan - 1] == kl);
+                        full, gp + min_span - 1 < n && sk[gp] == kl && sk[gp + min_span - 1] == kl);
                     k.n_groups += (uint32_t)__popc(m);      // hits are a prefix of the probed range
                     if (m != full) break;
                 }
                 k.rem_first = group_end + k.n_groups * kGroupTiles;
                 const uint32_t t2 = k.rem_first + lane;
                 k.rem_cnt = (uint32_t)__popc(__ballot_sync(
-                    full, lane < kGroupMinSpan / kReduceTile && t2 < n_tiles && sk[(uint64_t)t2 * kReduceTile] == kl));
+                    full, lane < 8 && t2 < n_tiles && sk[(uint64_t)t2 * tile_len] == kl));
             }
             const uint32_t n_parts = k.last_tile - k.tile + k.n_groups + k.rem_cnt;
             k.is_long = n_parts > kFixupWarps ? 1u : 0u;
@@ -790,7 +860,7 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                         if (f < L4) r[c] = store[k.row * L4 + f];
                     }
                     add(a, f0, carry + ((uint64_t)k.tile * 2 + 1) * L);
-                    for (uint32_t i = 0; i < n_parts; ++i) add_nth(a, f0, k, i);
+                    add_range(a, f0, k, 0, 1, n_parts);
 #pragma unroll
                     for (int c = 0; c < kCh; ++c) {
                         const uint32_t f = f0 + lane + 32 * c;
@@ -822,8 +892,7 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                     r[c] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (w == 0 && f < L4) r[c] = store[kj.row * L4 + f];       // asked for early, used after the barrier
                 }
-#pragma unroll 2
-                for (uint32_t i = w; i < n_parts; i += kFixupWarps) add_nth(a, f0, kj, i);
+                add_range(a, f0, kj, w, kFixupWarps, n_parts);
 #pragma unroll
                 for (int c = 0; c < kCh; ++c) part[w][c][lane] = a[c];
                 __syncthreads();
@@ -855,24 +924,25 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
 }
 
 int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
-    return radix_sort_pairs(ps, n, nullptr, ps->key_bits, true, s, 0, ps->starter_count,
-                            div_up_u32(n, kGroupSpan));
+    return radix_sort_pairs(ps, n, nullptr, ps->key_bits, s, 0, ps->starter_count, div_up_u32(n, kGroupSpan));
 }
 
-// The launch that follows a reduction: finishes the border-crossing segments, adds the loss partials and,
-// for calls that staged new rows instead of writing them (apply), moves those into the store.
+// The launch that follows a reduction: finishes the border-crossing segments (tiles of tile_len positions), adds the
+// loss partials and, for calls that staged new rows instead of writing them, moves the rows staged at
+// positions apply_lo .. n into the store.
 static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d_loss_accum, uint32_t loss_blocks,
-                         bool apply, cudaStream_t s) {
-    const uint32_t tiles = div_up_u32(n, kReduceTile);
+                         bool apply, uint32_t tile_len, uint32_t apply_lo, cudaStream_t s) {
+    const uint32_t tiles = div_up_u32(n, tile_len);
     const uint32_t L4 = ps->cfg.row_len / 4;
     // a warp per listed segment; there are fewer segments in the list than tiles
     const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8);
-    const uint32_t apply_blocks = apply ? tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8) : 0;
+    const uint32_t apply_blocks =
+        apply ? tmax<uint32_t>(1u, tmin<uint32_t>(div_up_u32(n - apply_lo, 32 * kFixupWarps), (uint32_t)ps->sm_count * 8)) : 0;
     const uint32_t grid = fix_blocks + 1 + apply_blocks;
 #define FIXUP_ARGS sk, n, (float4*)ps->store, ps->table, ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4,   \
                    ps->carry, ps->group_sum, ps->starters, ps->starter_count, ps->loss_partial, loss_blocks,      \
                    loss_blocks ? d_loss_accum : nullptr, fix_blocks, (const float4*)ps->upd, ps->apply_rows,      \
-                   ps->status, ps->epoch
+                   tile_len, apply_lo, ps->status, ps->epoch
     if (L4 <= 32) PS_LAUNCH(ps, push_fixup_kernel<1>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
     else if (L4 <= 64) PS_LAUNCH(ps, push_fixup_kernel<2>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
     else if (L4 <= 96) PS_LAUNCH(ps, push_fixup_kernel<3>, grid, 32 * kFixupWarps, s, FIXUP_ARGS);
@@ -880,36 +950,42 @@ static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d
 #undef FIXUP_ARGS
 }
 
-// The MF step on sorted occurrences (which: buffer that holds the sort's result); rows of at most 512 values.
-void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
-                  uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, cudaStream_t s) {
+// The MF step on sorted occurrences (which: buffer that holds the sorted keys; the records are in ps->rec); rows
+// of at most 128 values.  Column side first (new rows staged), then the row side (new rows written in place),
+// then the fix-up launch, which also moves the staged column rows into the store.
+void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
+                  double* d_loss_accum, cudaStream_t s) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
-    const uint32_t* sv = which ? ps->valsB : ps->valsA;
     const uint32_t n = 2 * n_cells;
-    const uint32_t tiles = div_up_u32(n, kReduceTile);
-    const uint32_t blocks = div_up_u32(tiles, 8);
     const uint32_t L4 = ps->cfg.row_len / 4;
-#define FUSED_ARGS sk, sv, n, d_i, d_j, d_v, (uint32_t)col_key_base, lr, lambda, (const float4*)ps->store, ps->table, \
-                   ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, (float4*)ps->upd, ps->apply_rows,          \
-                   ps->carry, ps->starters, ps->starter_count, ps->group_done, ps->group_sum, ps->loss_partial,       \
-                   ps->status, ps->epoch
-#define FUSED_LAUNCH(kCh)                                                                                            \
+    const uint32_t all_blocks = div_up_u32(n, 256);
+    const uint32_t row_blocks = div_up_u32(n_cells, 256);               // blocks 0 .. row_blocks work on the row side
+    const uint32_t col_first = n_cells / 256;                           // blocks col_first .. all_blocks on the column side
+    // a block that holds positions of both sides runs in both launches: one more arrival for its group of tiles
+    const uint32_t extra_group = (n_cells % 256) ? col_first / (kGroupTiles / 32) : 0xFFFFFFFFu;
+#define SUB_ARGS(lo, hi, first, in_place)                                                                            \
+    sk, ps->rec, n, (uint32_t)(lo), (uint32_t)(hi), (uint32_t)(first), (int)(in_place), (uint32_t)col_key_base, lr,  \
+        lambda, (float4*)ps->store, (uint32_t)ps->cfg.num_keys, L4, (float4*)ps->upd, ps->apply_rows, ps->carry,     \
+        ps->starters, ps->starter_count, ps->group_done, ps->group_sum, extra_group, ps->loss_partial, ps->status,  \
+        ps->epoch
+#define SUB_LAUNCH(kC)                                                                                               \
     do {                                                                                                             \
         static bool smem_set = false;                                                                                \
         if (!smem_set) {                                                                                             \
-            cudaFuncSetAttribute(mf_fused_kernel<kCh>, cudaFuncAttributeMaxDynamicSharedMemorySize,                  \
-                                 (int)reduce_smem(kCh));                                                             \
+            cudaFuncSetAttribute(mf_sub_kernel<kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMfSmem);      \
             smem_set = true;                                                                                         \
         }                                                                                                            \
-        PS_LAUNCH_SMEM(ps, mf_fused_kernel<kCh>, blocks, 256, reduce_smem(kCh), s, FUSED_ARGS);                      \
+        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, all_blocks - col_first, 256, kMfSmem, s,                               \
+                       SUB_ARGS(n_cells, n, col_first, 0));                                                          \
+        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, row_blocks, 256, kMfSmem, s, SUB_ARGS(0, n_cells, 0, 1));              \
     } while (0)
-    if (L4 <= 32) FUSED_LAUNCH(1);
-    else if (L4 <= 64) FUSED_LAUNCH(2);
-    else if (L4 <= 96) FUSED_LAUNCH(3);
-    else FUSED_LAUNCH(4);
-#undef FUSED_LAUNCH
-#undef FUSED_ARGS
-    launch_fixup(ps, sk, n, d_loss_accum, d_loss_accum ? blocks : 0, true, s);
+    if (L4 <= 8) SUB_LAUNCH(1);
+    else if (L4 <= 16) SUB_LAUNCH(2);
+    else if (L4 <= 24) SUB_LAUNCH(3);
+    else SUB_LAUNCH(4);
+#undef SUB_LAUNCH
+#undef SUB_ARGS
+    launch_fixup(ps, sk, n, d_loss_accum, d_loss_accum ? row_blocks : 0, true, kMfTile, n_cells, s);
 }
 
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
@@ -948,7 +1024,7 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     }
 #undef REDUCE_LAUNCH
 #undef REDUCE_ARGS
-    launch_fixup(ps, sk, n, d_loss_accum, loss_blocks, false, s);
+    launch_fixup(ps, sk, n, d_loss_accum, loss_blocks, false, kReduceTile, 0, s);
 }
 
 void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_loss_accum, uint32_t loss_blocks,

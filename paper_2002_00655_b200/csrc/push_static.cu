@@ -99,6 +99,7 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     int bits = 0;
     while (bits < 32 && (num_keys >> bits) != 0) ++bits;
     tmp.key_bits = bits < 1 ? 1 : bits;
+    tmp.sort_blocks_cap = (uint32_t)((kStaticMaxKeys + kSortTile - 1) / kSortTile);
     tmp.store = (float*)d_store;
     tmp.table = (uint2*)const_cast<void*>(d_table);
     tmp.status = (DevStatus*)(dev.scratch + kOffStatus);
@@ -119,6 +120,8 @@ extern "C" ps_status_t ps_push_static(void* d_store, const void* d_table, uint64
     cudaStream_t s = (cudaStream_t)stream;
     // The array keeps whatever the previous call left: the status words must start at zero.
     if (cudaMemsetAsync(tmp.status, 0, sizeof(DevStatus), s) != cudaSuccess) return PS_ERR_CUDA;
+    // ... and so must the two words of the sort's grid barrier, should an earlier call have given up inside it
+    if (cudaMemsetAsync(tmp.sort_ctl, 0, 2 * sizeof(uint32_t), s) != cudaSuccess) return PS_ERR_CUDA;
     launch_prepare_keys(&tmp, d_keys, n, s);
     run_push_pipeline(&tmp, (uint32_t)n, d_updates, nullptr, 0, s);
     if (cudaGetLastError() != cudaSuccess) return PS_ERR_CUDA;

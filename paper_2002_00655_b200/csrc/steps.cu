@@ -191,18 +191,6 @@ mf_step_small_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict
     block_loss_out(loss, loss_partial);
 }
 
-// keys of the occurrences of a batch of cells: [2t] = row factor, [2t+1] = column factor
-__global__ void __launch_bounds__(256)
-mf_keys_kernel(const uint32_t* __restrict__ ci, const uint32_t* __restrict__ cj, uint64_t n, uint64_t col_base,
-               uint64_t K, uint32_t* __restrict__ keys_out, DevStatus* st, unsigned int epoch) {
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= n) return;
-    const uint64_t kw = ci[t], kh = col_base + cj[t];
-    const bool bad = kw >= col_base || kh >= K;
-    if (bad) latch_error(st, epoch, PS_ERR_KEY_RANGE);
-    reinterpret_cast<uint2*>(keys_out)[t] = bad ? make_uint2((uint32_t)K, (uint32_t)K) : make_uint2((uint32_t)kw, (uint32_t)kh);
-}
-
 uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
                         uint64_t col_key_base, float lr, float lambda, cudaStream_t s) {
     const uint32_t L4 = ps->cfg.row_len / 4;
@@ -216,12 +204,6 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
     else PS_LAUNCH(ps, mf_step_kernel<0>, grid, 256, s, MF_ARGS);
 #undef MF_ARGS
     return grid;
-}
-
-void launch_keys_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, uint64_t n, uint64_t col_key_base,
-                    cudaStream_t s) {
-    PS_LAUNCH(ps, mf_keys_kernel, div_up_u32(n, 256), 256, s, d_i, d_j, n, col_key_base, ps->cfg.num_keys, ps->keysA,
-              ps->status, ps->epoch);
 }
 
 // ------------------------------------------------------------- ComplEx ----
