@@ -122,11 +122,18 @@ def n_unique(*tensors) -> int:
     return int(torch.unique(torch.cat([t.reshape(-1).to(torch.int64) for t in tensors])).numel())
 
 
-def kernel_bytes_of_step(batch_bytes, occ, u, rb, keys_prefix, step_prefix):
+def sort_bytes(occ, key_bits, extra=0):
+    """The one-launch key sort: per pass keys and values in and out (the first pass reads no values)."""
+    passes = (key_bits + 7) // 8
+    return occ * (16 * passes - 4) + extra
+
+
+def kernel_bytes_of_step(batch_bytes, occ, u, rb, keys_prefix, step_prefix, key_bits):
     """Bytes per LAUNCH that each kernel of a step call must move, by kernel-name prefix: what it reads of the
     batch, the table and the store, and what it has to write for the next kernel (keys, update rows)."""
     return {
         keys_prefix: batch_bytes + occ * 4,                      # batch arrays in, one 32-bit key per occurrence out
+        "sort_all_kernel": sort_bytes(occ, key_bits),
         step_prefix: batch_bytes + occ * (8 + rb) + occ * rb,    # table entry + row per occurrence in, update row out
         "push_reduce_kernel": occ * (8 + rb) + u * (8 + 2 * rb), # sorted pair + update row in; row read-modify-write
     }
@@ -201,7 +208,19 @@ class MFWorkload:
         c, b = self.cfg, self.cfg.batch
         sl = slice(k * b, (k + 1) * b)
         u = n_unique(self.i[sl]) + n_unique(self.j[sl])
-        return kernel_bytes_of_step(b * 12, 2 * b, u, self.row_bytes, "mf_keys", "mf_step")
+        occ, rb = 2 * b, self.row_bytes
+        bits = int(c.num_keys).bit_length()
+        if c.rank > 128:                                        # unfused path: update rows are materialised
+            return kernel_bytes_of_step(b * 12, occ, u, rb, "mf_keys", "mf_step", bits)
+        return {
+            # batch arrays in (twice: keys, then records), two table entries per occurrence, keys and records out
+            "sort_all_kernel": sort_bytes(occ, bits, extra=2 * b * 12 + occ * (16 + 4 + 16)),
+            # per launch (two per step, one per side): a record and the partner row per occurrence, the own row
+            # once per distinct key, the new row out (to the store or to the staging rows)
+            "mf_sub_kernel": (occ * (16 + rb) + u * 2 * rb) / 2,
+            # staged column rows moved into the store (read + write); border-crossing segments are not counted
+            "push_fixup_kernel": n_unique(self.j[sl]) * 2 * rb,
+        }
 
     # --- oracle leg ---
     def oracle_setup(self, device):
@@ -295,7 +314,8 @@ class KGEWorkload:
     def kernel_bytes(self, k):
         c, sl, b = self.cfg, self._sl(k), self.cfg.batch
         u = n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl])
-        return kernel_bytes_of_step(b * (12 + c.n_neg * 5), (3 + c.n_neg) * b, u, self.row_bytes, "kge_keys", "kge_step")
+        return kernel_bytes_of_step(b * (12 + c.n_neg * 5), (3 + c.n_neg) * b, u, self.row_bytes, "kge_keys", "kge_step",
+                                    int(c.num_keys).bit_length())
 
     def oracle_setup(self, device):
         from oracle import OracleStore
@@ -396,7 +416,7 @@ class SGNSWorkload:
         c = self.cfg
         pairs, occ, u = self._occ_u(k)
         kb = kernel_bytes_of_step(c.batch * 4 + pairs * (1 + c.n_neg) * 4, occ, u, self.row_bytes,
-                                  "sgns_keys", "sgns_step")
+                                  "sgns_keys", "sgns_step", int(c.num_keys).bit_length())
         # the step kernel writes two source rows per center and one factor per occurrence, not a row per occurrence
         kb["sgns_step"] += c.batch * 2 * self.row_bytes + occ * 4 - occ * self.row_bytes
         # ... and the reduction reads a factor per occurrence and those 2 x centers source rows (from L2 after the first touch)

@@ -128,7 +128,7 @@ static SortSet* next_set(ps_store* ps) {
 // Ordered mode: the side stream starts after everything already enqueued on the caller's stream.
 // Pipelined mode: it starts as soon as the buffer set's previous user is done, i.e. beside the previous
 // step's kernels; the batch arrays must then be complete when the call is made.
-static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
+static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_table = false) {
     // When the caller's stream enters or leaves a CUDA-graph capture, events recorded on the other side of
     // that border cannot be waited on, and the side stream has to join (or leave) the capture: the first
     // call after such a change forks in ordered mode and forgets the older events.
@@ -138,12 +138,19 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s) {
     if (cs != cudaStreamCaptureStatusActive) id = 0;
     const bool crossed = id != ps->capture_id;
     ps->capture_id = id;
-    if (crossed)
+    if (crossed) {
         for (int b = 0; b < kSortSets; ++b) ps->sets[b].used = false;
+        ps->mid_valid = false;
+    }
     // a sort that reads the location table (the matrix-factorization records) must come after a call that rewrote it
-    const bool ordered = crossed || ps->table_dirty;
-    ps->table_dirty = false;
-    if (ps->pipelined && !ordered) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
+    const bool ordered = crossed || (reads_table && ps->table_dirty);
+    if (ordered) ps->table_dirty = false;
+    if (ps->pipelined && !ordered) {
+        // not before the previous step's first kernel is through: the sort's blocks wait at grid barriers most of
+        // the time and would hold registers that kernel's blocks need (see run_mf_fused)
+        if (ps->mid_valid && cudaStreamWaitEvent(ps->side, ps->ev_mid, 0) != cudaSuccess) return false;
+        return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
+    }
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
@@ -250,7 +257,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
     if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_mid, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
     }
@@ -270,6 +278,7 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
+    cudaEventDestroy(ps->ev_mid);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
     cudaStreamDestroy(ps->side);
     delete ps;
@@ -341,7 +350,7 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
     SortSet* ss = next_set(ps);
-    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
+    if (!fork_side(ps, ss, s, true)) return PS_ERR_CUDA;
     // rows short enough to be staged whole, and row numbers that fit the 32-bit fields of the sort's records
     const bool fused = ps->cfg.row_len <= 128 && (uint64_t)ps->cfg.num_workers * ps->cfg.slots_per_part < (1ull << 32);
     const int which = radix_sort_mf(ps, d_i, d_j, d_v, (uint32_t)n, col_key_base, fused, ps->side, ps->starter_count,

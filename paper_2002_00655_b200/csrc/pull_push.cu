@@ -977,6 +977,7 @@ void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_ba
         }                                                                                                            \
         PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, all_blocks - col_first, 256, kMfSmem, s,                               \
                        SUB_ARGS(n_cells, n, col_first, 0));                                                          \
+        ps->mid_valid = cudaEventRecord(ps->ev_mid, s) == cudaSuccess;                                               \
         PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, row_blocks, 256, kMfSmem, s, SUB_ARGS(0, n_cells, 0, 1));              \
     } while (0)
     if (L4 <= 8) SUB_LAUNCH(1);
