@@ -511,7 +511,7 @@ class StressWorkload:
     def kernel_bytes(self, k):
         n, rb = self.cfg.batch, self.row_bytes
         u = n_unique(self.keys[k])
-        return {"pull_kernel": n * (16 + 2 * rb), "push_reduce_kernel": n * (8 + rb) + u * (8 + 2 * rb)}
+        return {"pull_bulk_kernel": n * (16 + 2 * rb), "pull_kernel": n * (16 + 2 * rb), "push_reduce_kernel": n * (8 + rb) + u * (8 + 2 * rb)}
 
     def oracle_setup(self, device):
         return None

@@ -63,9 +63,131 @@ void launch_set_rows(ps_store* ps, const uint64_t* d_keys, uint64_t n, const flo
               ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, ps->epoch);
 }
 
+// ---- bulk asynchronous copies global -> shared, reporting to a barrier word in shared memory ----
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
+// one arrival that also announces `bytes` of copies
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// 16-byte aligned source and destination, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
+                     smem_addr(smem)),
+                 "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.
+constexpr unsigned kBarPollLimit = 1u << 22;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
+    const unsigned a = smem_addr(bar);
+    for (unsigned i = 0; i < kBarPollLimit; ++i) {
+        unsigned done;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(done)
+            : "r"(a), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// shared -> global, tracked in the issuing thread's bulk groups
+__device__ __forceinline__ void bulk_s2g(void* gmem, const void* smem, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem), "r"(smem_addr(smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+// until at most kPending of this thread's bulk groups still have to READ their source
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(kPending) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+
 // ---------------------------------------------------------------- pull ----
+// Rows travel store -> shared memory -> caller's buffer as bulk asynchronous copies of whole rows, without
+// passing through registers: a lane looks its key up, asks for the row, and once the round's rows have
+// landed asks for them to be written out.  A warp works on rounds of kPullStageBytes / row_bytes keys, two
+// rounds in flight (the loads of one beside the stores of the one before).
+constexpr uint32_t kPullStageBytes = 4096;          // per warp and stage
+constexpr size_t kPullSmem = (size_t)8 * 2 * kPullStageBytes;
+
+__global__ void __launch_bounds__(256)
+pull_bulk_kernel(const uint64_t* __restrict__ keys, uint64_t n, char* __restrict__ out, const char* __restrict__ store,
+                 const uint2* __restrict__ table, uint64_t S, uint64_t K, uint32_t row_bytes, uint32_t per_round,
+                 DevStatus* st, unsigned int epoch) {
+    __shared__ __align__(8) uint64_t bars[8][2];
+    extern __shared__ __align__(128) char pull_stage[];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    char* my = pull_stage + (size_t)w * 2 * kPullStageBytes;
+    if (lane < 2) mbar_init(&bars[w][lane], 1);
+    mbar_init_fence();
+    __syncwarp();
+    uint32_t uses = 0;
+    int stage = 0;
+    // the round whose loads are in flight: its first key, how many rows were asked for, whether this lane has one
+    uint64_t prev_t0 = 0;
+    uint32_t prev_rows = 0;
+    bool prev_mine = false, have_prev = false;
+    auto finish = [&](int sg) -> bool {             // waits for a round's rows and sends them on their way
+        if (prev_rows) {
+            const uint32_t parity = (uses >> sg) & 1u;
+            if (!mbar_wait(&bars[w][sg], parity) && !mbar_wait(&bars[w][sg], parity)) {
+                if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
+                return false;
+            }
+            uses ^= 1u << sg;
+            fence_async_smem();
+        }
+        if (prev_mine)
+            bulk_s2g(out + (prev_t0 + lane) * row_bytes, my + (size_t)sg * kPullStageBytes + (size_t)lane * row_bytes,
+                     row_bytes);
+        bulk_commit();
+        return true;
+    };
+    for (uint64_t t0 = warp * per_round; t0 < n; t0 += n_warps * per_round) {
+        const uint64_t t = t0 + lane;
+        const bool mine = (uint32_t)lane < per_round && t < n;
+        uint64_t row = 0;
+        bool ok = false;
+        if (mine) {
+            const uint64_t key = keys[t];
+            if (key < K) {
+                row = phys_row(table[key], S);
+                ok = true;
+            } else {
+                latch_error(st, epoch, PS_ERR_KEY_RANGE);
+                float4* o = (float4*)(out + t * row_bytes);         // a key out of range reads as a row of zeros
+                for (uint32_t f = 0; f < row_bytes / 16; ++f) o[f] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        const uint32_t rows = __popc(__ballot_sync(0xffffffffu, ok));
+        bulk_wait_read<0>();                        // the stores that last read this stage (the round before last) are done with it
+        __syncwarp();
+        if (rows) {
+            if (lane == 0) mbar_expect_tx(&bars[w][stage], rows * row_bytes);
+            __syncwarp();
+            if (ok)
+                bulk_g2s(my + (size_t)stage * kPullStageBytes + (size_t)lane * row_bytes, store + row * row_bytes,
+                         row_bytes, &bars[w][stage]);
+        }
+        if (have_prev && !finish(stage ^ 1)) return;
+        prev_t0 = t0; prev_rows = rows; prev_mine = ok; have_prev = true;
+        stage ^= 1;
+    }
+    if (have_prev && !finish(stage ^ 1)) return;
+    bulk_wait_read<0>();
+}
+
 // One warp gathers kRows rows at a time so that several independent 128-bit
-// loads are in flight per lane.
+// loads are in flight per lane (rows too long for the staged kernel above).
 template <int kRows>
 __global__ void __launch_bounds__(256)
 pull_kernel(const uint64_t* __restrict__ keys, uint64_t n, float4* __restrict__ out,
@@ -104,6 +226,20 @@ pull_kernel(const uint64_t* __restrict__ keys, uint64_t n, float4* __restrict__ 
 }
 
 void launch_pull(ps_store* ps, const uint64_t* d_keys, uint64_t n, float* d_out, cudaStream_t s) {
+    const uint32_t row_bytes = ps->cfg.row_len * 4;
+    if (row_bytes <= kPullStageBytes) {
+        static bool smem_set = false;
+        if (!smem_set) {
+            cudaFuncSetAttribute(pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPullSmem);
+            smem_set = true;
+        }
+        const uint32_t per_round = tmin<uint32_t>(32u, kPullStageBytes / row_bytes);
+        const uint64_t rounds = (n + per_round - 1) / per_round;
+        const uint32_t grid = (uint32_t)tmin<uint64_t>((rounds + 7) / 8, (uint64_t)ps->sm_count * 3);
+        PS_LAUNCH_SMEM(ps, pull_bulk_kernel, grid, 256, kPullSmem, s, d_keys, n, (char*)d_out, (const char*)ps->store,
+                       ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, row_bytes, per_round, ps->status, ps->epoch);
+        return;
+    }
     const uint32_t grid = (uint32_t)tmin<uint64_t>((n + 31) / 32, (uint64_t)ps->sm_count * 8);
     PS_LAUNCH(ps, pull_kernel<4>, grid, 256, s, d_keys, n, (float4*)d_out, (const float4*)ps->store, ps->table,
               ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, ps->epoch);
@@ -173,39 +309,6 @@ void launch_prepare_keys(ps_store* ps, const uint64_t* d_keys, uint64_t n, cudaS
 struct d4 {
     double x, y, z, w;
 };
-
-// ---- bulk asynchronous copies global -> shared, reporting to a barrier word in shared memory ----
-__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
-// one arrival that also announces `bytes` of copies
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-// 16-byte aligned source and destination, size a multiple of 16 bytes
-__device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
-                     smem_addr(smem)),
-                 "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.
-constexpr unsigned kBarPollLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
-    const unsigned a = smem_addr(bar);
-    for (unsigned i = 0; i < kBarPollLimit; ++i) {
-        unsigned done;
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(done)
-            : "r"(a), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
 
 // Staging of the reduction kernel for rows of up to kCh column blocks (32 float4 each): positions whose
 // copies are asked for together, and groups in flight per warp.  A position takes 2 x kCh x 512 bytes (update
