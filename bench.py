@@ -115,7 +115,11 @@ def smi_clocks():
 # ----------------------------------------------------------------------------------------
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/,
 # keyed by (workload, kernel).  An entry is removed when its kernel changes after the capture.
-TRAFFIC = {}
+TRAFFIC = {
+    ("mf_large", "mf_sub_kernel<4>"): 41.5e6,                   # profiles/mf_step_kernels_ncu_full.md (same-batch twin)
+    ("kge", "kge_step_kernel<10>"): 305.4e6,                    # profiles/kge_step_kernels_ncu_full.md
+    ("sgns", "push_reduce_kernel<3,true>"): 1520.6e6,           # profiles/sgns_step_kernels_ncu_full.md
+}
 
 
 def n_unique(*tensors) -> int:
@@ -522,7 +526,8 @@ def make_workload(name):
              "mf_medium": lambda: MFWorkload(W.MF_MEDIUM),
              "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
              "sgns": lambda: SGNSWorkload(W.SGNS), "sgns_tiny": lambda: SGNSWorkload(W.SGNS_TINY),
-             "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY)}
+             "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY),
+             "stress_medium": lambda: StressWorkload(W.STRESS_MEDIUM)}
     return table[name]()
 
 
@@ -779,7 +784,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mf_large",
-                    choices=["mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny"])
+                    choices=["mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny",
+                             "stress_medium"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host")

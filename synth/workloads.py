@@ -361,6 +361,9 @@ class StressConfig:
 
 STRESS = StressConfig("stress", 100_000_000, 128, 64, 1_000_000, 1_000, 0.9, 100_000)
 STRESS_TINY = StressConfig("stress_tiny", 50_000, 128, 8, 6_000, 12, 0.9, 600)
+# the stress batch (1M keys, 100k of them localized) on a store of 3 GB: for profiler captures.  Fewer workers and
+# more spare slots than the full configuration, so that a partition can take 100k keys at a time.
+STRESS_MEDIUM = StressConfig("stress_medium", 4_000_000, 128, 16, 1_000_000, 200, 0.9, 100_000, slack=1.5)
 
 
 def stress_init_rows(cfg: StressConfig, key_start: int, count: int, device) -> torch.Tensor:
