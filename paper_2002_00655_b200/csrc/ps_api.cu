@@ -38,6 +38,7 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.tile_state[b] = take((size_t)kMaxSortPasses * sort_tiles * kRadix * 4);
         l.sort_ctl[b] = take(((size_t)kSortCtlWords + groups) * 4);
         l.rec[b] = take(mk * 16);
+        l.cellpos[b] = take(mk * 4);
         l.starters[b] = take(reduce_tiles * 16);
         l.starter_count[b] = take(4);
     }
@@ -119,7 +120,7 @@ static SortSet* next_set(ps_store* ps) {
     SortSet* ss = &ps->sets[ps->cur_set];
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
     ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
-    ps->starters = ss->starters; ps->starter_count = ss->starter_count; ps->rec = ss->rec;
+    ps->starters = ss->starters; ps->starter_count = ss->starter_count; ps->rec = ss->rec; ps->cellpos = ss->cellpos;
     return ss;
 }
 
@@ -223,6 +224,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.sort_ctl = (uint32_t*)(ps->ws + l.sort_ctl[b]);
         ss.group_done = ss.sort_ctl + kSortCtlWords;
         ss.rec = (uint4*)(ps->ws + l.rec[b]);
+        ss.cellpos = (uint32_t*)(ps->ws + l.cellpos[b]);
         ss.starters = (uint4*)(ps->ws + l.starters[b]);
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;

@@ -45,6 +45,7 @@ struct SortSet {
     uint32_t* sort_ctl;
     unsigned int* group_done;
     uint4* rec;
+    uint32_t* cellpos;
     uint4* starters;
     unsigned int* starter_count;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
@@ -71,7 +72,8 @@ struct ps_store {
     uint32_t *keysA, *keysB, *valsA, *valsB;
     uint32_t* tile_state;           // kMaxSortPasses x sort blocks x kRadix digit counters
     uint32_t* sort_ctl;             // the sort's grid barrier (two words) in kSortCtlWords, followed by group_done
-    uint4* rec;                     // MF: {key, cell value, row of the key, row of the other factor} per sorted position
+    uint4* rec;                     // MF: {cell, cell value, row of the key, row of the other factor} per sorted position
+    uint32_t* cellpos;              // MF: sorted position of each cell's row-factor occurrence
     unsigned int* group_done;       // per group of 64 reduction tiles: reduction blocks that have finished
     double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
@@ -102,7 +104,7 @@ namespace psb {
 
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
-        sort_ctl[kSortSets], rec[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
         loss_partial, apply_rows, staging, total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);

@@ -553,7 +553,7 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
 
 // ------------------------------------------------- MF: gradient inside the reduction ----
 // One minibatch of matrix factorization without update rows.  The occurrences (2t: row factor of cell t,
-// 2t + 1: its column factor) arrive sorted by key, as for a push, each with a record {key, value of the
+// 2t + 1: its column factor) arrive sorted by key, as for a push, each with a record {cell, value of the
 // cell, row of the key, row of the cell's other factor} written by the sort.  For every sorted position
 // the PARTNER row (the other factor) is fetched and, where a segment's part in a tile begins, the key's
 // own row; e = v - <own, partner> is formed on the spot and lr (e partner - lambda own) is added to the
@@ -569,25 +569,29 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
 // A segment of exactly one position needs no fp64 sum: own + update is formed in fp32, which rounds the
 // same exact sum once.
 //
-// Column-factor keys sort after row-factor keys, so the two sides are two ranges of positions, and the
-// step runs this kernel twice.  First the column side: it reads row factors as partners and leaves its new
-// rows in `staged` (the fix-up launch moves them into the store).  Then the row side: its partners are
-// column factors, which nothing has overwritten, and nobody reads a row factor any more except the group
-// that owns its segment, so new rows go straight into the store.  The loss of a cell is taken at its
-// row-factor occurrence.
+// Nothing may overwrite a row that another position still reads, so new rows are left in `staged` (indexed by
+// the sorted position where the segment ends) with the row's address in `apply_row`, and the fix-up launch,
+// which runs after every read of this kernel, moves them into the store.  One case needs neither staging nor a
+// segment: a row factor whose key occurs ONCE in the batch (nearly all of them, rows being drawn uniformly) is
+// read by exactly one position, the column-factor occurrence of its cell, as the partner.  That position has
+// both rows in hand; it forms the row factor's new row too and writes it in place, and the row factor's own
+// position is skipped together with its two row fetches.  The loss of a cell is taken where its row factor
+// is updated.
 constexpr int kMfTile = 8;
 constexpr int kMfStages = 3;
 constexpr size_t kMfSmem = (size_t)8 * kMfStages * 4 * 64 * sizeof(float4);     // warp x stage x group x {partner, own}
 
-enum : uint32_t { kFUsable = 1, kFBegin = 2, kFEnd = 4, kFParked = 8, kFFromPrev = 16, kFSide0 = 32, kFSingle = 64 };
+enum : uint32_t { kFUsable = 1, kFBegin = 2, kFEnd = 4, kFParked = 8, kFFromPrev = 16, kFBoth = 32, kFSingle = 64,
+                  kFColumn = 128 };
 
 template <int kC>
 __global__ void __launch_bounds__(256, 2)
-mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, uint32_t n, uint32_t lo, uint32_t hi,
-              uint32_t first_block, int in_place, uint32_t col_base, float lr, float lam, float4* store, uint32_t K,
+mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, const uint32_t* __restrict__ cellpos,
+              uint32_t n,
+              uint32_t col_base, float lr, float lam, float4* store, uint32_t K,
               uint32_t L4, float4* __restrict__ staged, uint64_t* __restrict__ apply_row, double* __restrict__ carry,
               uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
-              unsigned int* __restrict__ group_done, double* __restrict__ group_sum, uint32_t extra_group,
+              unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
               double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
     __shared__ unsigned int s_ticket;
     __shared__ __align__(8) uint64_t bars[8][kMfStages];
@@ -597,14 +601,14 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int sg = lane >> 3, l8 = lane & 7;
-    const uint32_t gb = first_block + blockIdx.x;                   // block number over all sorted positions
+    const uint32_t gb = blockIdx.x;
     const uint32_t tile32 = gb * 8 + w;
     const uint64_t base = (uint64_t)tile32 * 32;
     const uint64_t pos = base + lane;
-    const bool inside = pos >= lo && pos < hi;                      // hi <= n
-    const uint4 me = inside ? rec[pos] : make_uint4(kSentinelPad, 0u, 0u, 0u);
-    const uint32_t key = me.x;
-    const bool usable = key < K;
+    const bool inside = pos < n;
+    // {cell, value of the cell, row of the key, row of the cell's other factor}, written by the sort's last pass
+    const uint4 me = inside ? rec[pos] : make_uint4(0u, 0u, 0u, 0u);
+    const uint32_t key = inside ? sk[pos] : kSentinelPad;
     const float val = __uint_as_float(me.y);
     const uint32_t row = me.z, prow = me.w;
     uint32_t prev = __shfl_up_sync(full, key, 1);
@@ -612,6 +616,20 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
     uint32_t next = __shfl_down_sync(full, key, 1);
     if (lane == 31) next = (base + 32 < n) ? sk[base + 32] : kSentinelPad;
     const bool head = key != prev;
+    // A row factor whose key occurs once in the batch is read by exactly one position of the column side (its
+    // cell's), as the partner.  That position has both rows in hand, so it also forms the row factor's new row and
+    // writes it in place; the row side then skips the position, and its two row fetches.
+    bool both = false;                              // column side: this position also updates its partner
+    bool usable = key < K;
+    const bool row_side = key < col_base;
+    if (row_side) {
+        if (usable && head && key != next) usable = false;
+    } else if (usable) {
+        const uint32_t pp = cellpos[me.x];          // sorted position of the cell's row-factor occurrence
+        const uint32_t kp = sk[pp];
+        const uint32_t kl = pp > 0 ? sk[pp - 1] : kSentinelPad, kr = pp + 1 < n ? sk[pp + 1] : kSentinelPad;
+        both = kl != kp && kr != kp;
+    }
     const unsigned head_mask = __ballot_sync(full, head);
     const unsigned usable_mask = __ballot_sync(full, usable);
     // the head of this position's segment, if it lies in the warp's 32 positions
@@ -625,13 +643,12 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
     const bool stage_me = end_me && !parked;                        // a whole segment ends here: new row
     const uint32_t tile8 = tile32 * 4 + sg;
     if (runs_on && !from_prev) starters[atomicAdd(starter_count, 1u)] = make_uint4(tile8, key, row, 0u);
-    if (!in_place && inside) apply_row[pos] = stage_me ? (uint64_t)row : ~0ull;
+    if (inside) apply_row[pos] = stage_me ? (uint64_t)row : ~0ull;
     const unsigned begin_mask = __ballot_sync(full, begin_me);
     const uint32_t flags = (usable ? kFUsable : 0u) | (begin_me ? kFBegin : 0u) | (end_me ? kFEnd : 0u) |
                            (parked ? kFParked : 0u) | (from_prev ? kFFromPrev : 0u) |
-                           ((usable && key < col_base) ? kFSide0 : 0u) | ((begin_me && stage_me) ? kFSingle : 0u);
-    // where a finished row goes: the store row (row side) or the staging row of the position (column side)
-    const uint64_t dst_row = in_place ? (uint64_t)row : pos;
+                           (((usable && row_side) || both) ? kFBoth : 0u) | ((begin_me && stage_me) ? kFSingle : 0u) |
+                           ((usable && !row_side) ? kFColumn : 0u);
     // does a long segment enter this block's group of 64 tiles from the group before?
     constexpr uint32_t kTilesPerBlock = 8 * 4;
     const uint32_t group = gb / (kGroupTiles / kTilesPerBlock);
@@ -677,8 +694,9 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
     float nw = 0.f, loss_f = 0.f;                   // this lane's share of |own|^2 and of the tile's loss
     uint32_t uses = 0;
     int st_use = 0, st_fill = kMfStages - 1;
+    const int n_steps = usable_mask ? kMfTile : 0;  // (a warp of skipped positions has nothing to walk)
 #pragma unroll 1
-    for (int s2 = 0; s2 < kMfTile; ++s2) {
+    for (int s2 = 0; s2 < n_steps; ++s2) {
         __syncwarp();                               // every lane is done reading the stage to be refilled
         issue(s2 + kMfStages - 1, st_fill);
         const unsigned sm = 0x01010101u << s2;
@@ -696,7 +714,8 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
         const int src = 8 * sg + s2;
         const uint32_t f = __shfl_sync(full, flags, src);
         const float v = __shfl_sync(full, val, src);
-        const uint64_t drow = __shfl_sync(full, dst_row, src);
+        const uint64_t drow = base + src;           // a finished row goes to the staging row of its position
+        const uint32_t prow_s = __shfl_sync(full, prow, src);
         const bool live = f & kFUsable;
         if (f & kFBegin) {
             nw = 0.f;
@@ -720,7 +739,21 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
         dot += __shfl_xor_sync(full, dot, 4);
         const float e = v - dot;
         // the cell's loss: the lanes keep their shares of the two squared norms, one lane adds the squared error
-        if (f & kFSide0) loss_f += 0.5f * lam * (nw + nh) + (l8 == 0 ? 0.5f * e * e : 0.f);
+        // (taken where the cell's row factor is updated: on the row side, or here for a row key that occurs once)
+        if (f & kFBoth) loss_f += 0.5f * lam * (nw + nh) + (l8 == 0 ? 0.5f * e * e : 0.f);
+        if ((f & kFBoth) && (f & kFColumn)) {        // the partner's new row: it is a segment of this one position
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                if ((uint32_t)(l8 + 8 * c) < L4) {
+                    float4 r;
+                    r.x = h[c].x + lr * (e * own[c].x - lam * h[c].x);
+                    r.y = h[c].y + lr * (e * own[c].y - lam * h[c].y);
+                    r.z = h[c].z + lr * (e * own[c].z - lam * h[c].z);
+                    r.w = h[c].w + lr * (e * own[c].w - lam * h[c].w);
+                    store[(uint64_t)prow_s * L4 + l8 + 8 * c] = r;
+                }
+            }
+        }
         if (f & kFSingle) {
 #pragma unroll
             for (int c = 0; c < kC; ++c) {
@@ -730,8 +763,7 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
                     r.y = own[c].y + lr * (e * h[c].y - lam * own[c].y);
                     r.z = own[c].z + lr * (e * h[c].z - lam * own[c].z);
                     r.w = own[c].w + lr * (e * h[c].w - lam * own[c].w);
-                    if (in_place) store[drow * L4 + l8 + 8 * c] = r;
-                    else staged[drow * L4 + l8 + 8 * c] = r;
+                    staged[drow * L4 + l8 + 8 * c] = r;
                 }
             }
         } else if (live) {
@@ -755,30 +787,26 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, ui
                         float4 r = own[c];
                         r.x = (float)((double)r.x + acc[c].x); r.y = (float)((double)r.y + acc[c].y);
                         r.z = (float)((double)r.z + acc[c].z); r.w = (float)((double)r.w + acc[c].w);
-                        if (in_place) store[drow * L4 + fi] = r;
-                        else staged[drow * L4 + fi] = r;
+                        staged[drow * L4 + fi] = r;
                     }
                 }
             }
         }
     }
     __syncthreads();                                // the staging memory is scratch from here on
-    // per-block loss partial, fixed order (only the row side has loss terms)
-    if (in_place) {
+    // per-block loss partial, fixed order
+    {
         const double lw = warp_sum_d((double)loss_f);
         if (lane == 0) wl[w] = lw;
         __syncthreads();
         if (threadIdx.x == 0) {
             double t = 0;
             for (int i = 0; i < 8; ++i) t += wl[i];
-            loss_partial[gb] = t;
+            loss_partial[blockIdx.x] = t;
         }
     }
     if (!(kg < K && kg_prev == kg && kg_far == kg)) return;
-    // blocks that work on the group's tiles: those of the launch, plus one if a block runs in both launches
-    const uint32_t n_blocks_all = (uint32_t)(((uint64_t)n + 255) / 256);
-    const uint32_t arrivals = tmin<uint32_t>(kGroupTiles / kTilesPerBlock, n_blocks_all - group * (kGroupTiles / kTilesPerBlock)) +
-                              (group == extra_group ? 1u : 0u);
+    const uint32_t arrivals = tmin<uint32_t>(kGroupTiles / kTilesPerBlock, gridDim.x - group * (kGroupTiles / kTilesPerBlock));
     group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
                  &s_ticket, kMfTile, arrivals);
 }
@@ -1054,23 +1082,18 @@ static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d
 }
 
 // The MF step on sorted occurrences (which: buffer that holds the sorted keys; the records are in ps->rec); rows
-// of at most 128 values.  Column side first (new rows staged), then the row side (new rows written in place),
-// then the fix-up launch, which also moves the staged column rows into the store.
+// of at most 128 values.  One launch over all positions, then the fix-up launch, which also moves the staged rows
+// into the store.
 void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
                   double* d_loss_accum, cudaStream_t s) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     const uint32_t n = 2 * n_cells;
     const uint32_t L4 = ps->cfg.row_len / 4;
-    const uint32_t all_blocks = div_up_u32(n, 256);
-    const uint32_t row_blocks = div_up_u32(n_cells, 256);               // blocks 0 .. row_blocks work on the row side
-    const uint32_t col_first = n_cells / 256;                           // blocks col_first .. all_blocks on the column side
-    // a block that holds positions of both sides runs in both launches: one more arrival for its group of tiles
-    const uint32_t extra_group = (n_cells % 256) ? col_first / (kGroupTiles / 32) : 0xFFFFFFFFu;
-#define SUB_ARGS(lo, hi, first, in_place)                                                                            \
-    sk, ps->rec, n, (uint32_t)(lo), (uint32_t)(hi), (uint32_t)(first), (int)(in_place), (uint32_t)col_key_base, lr,  \
-        lambda, (float4*)ps->store, (uint32_t)ps->cfg.num_keys, L4, (float4*)ps->upd, ps->apply_rows, ps->carry,     \
-        ps->starters, ps->starter_count, ps->group_done, ps->group_sum, extra_group, ps->loss_partial, ps->status,  \
-        ps->epoch
+    const uint32_t blocks = div_up_u32(n, 256);
+#define SUB_ARGS                                                                                                     \
+    sk, ps->rec, ps->cellpos, n, (uint32_t)col_key_base, lr, lambda, (float4*)ps->store, (uint32_t)ps->cfg.num_keys, \
+        L4, (float4*)ps->upd, ps->apply_rows, ps->carry, ps->starters, ps->starter_count, ps->group_done,            \
+        ps->group_sum, ps->loss_partial, ps->status, ps->epoch
 #define SUB_LAUNCH(kC)                                                                                               \
     do {                                                                                                             \
         static bool smem_set = false;                                                                                \
@@ -1078,10 +1101,7 @@ void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_ba
             cudaFuncSetAttribute(mf_sub_kernel<kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMfSmem);      \
             smem_set = true;                                                                                         \
         }                                                                                                            \
-        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, all_blocks - col_first, 256, kMfSmem, s,                               \
-                       SUB_ARGS(n_cells, n, col_first, 0));                                                          \
-        ps->mid_valid = cudaEventRecord(ps->ev_mid, s) == cudaSuccess;                                               \
-        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, row_blocks, 256, kMfSmem, s, SUB_ARGS(0, n_cells, 0, 1));              \
+        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, blocks, 256, kMfSmem, s, SUB_ARGS);                                    \
     } while (0)
     if (L4 <= 8) SUB_LAUNCH(1);
     else if (L4 <= 16) SUB_LAUNCH(2);
@@ -1089,7 +1109,7 @@ void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_ba
     else SUB_LAUNCH(4);
 #undef SUB_LAUNCH
 #undef SUB_ARGS
-    launch_fixup(ps, sk, n, d_loss_accum, d_loss_accum ? row_blocks : 0, true, kMfTile, n_cells, s);
+    launch_fixup(ps, sk, n, d_loss_accum, d_loss_accum ? blocks : 0, true, kMfTile, 0, s);
 }
 
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,

@@ -113,7 +113,7 @@ struct SinkPairs {
 };
 // Matrix factorization: besides the sorted key, one record per sorted position with everything the gradient
 // kernel would otherwise have to chase through three dependent loads: {key, value of the cell, physical
-// row of the key, physical row of the cell's other factor}.
+// row of the key, physical row of the cell's other factor}.  (It says {cell, ...}: the key is in the sorted key array.)
 struct SinkMF {
     static constexpr bool kPairs = false;
     const uint32_t *ci, *cj;
@@ -122,6 +122,7 @@ struct SinkMF {
     const uint2* table;
     uint64_t S;
     uint4* rec;
+    uint32_t* cellpos;                  // sorted position of each cell's row-factor occurrence
 };
 
 // Exclusive scan of one value per digit held by threads 0..255 of a block of kThreads; every thread calls.
@@ -400,7 +401,8 @@ sort_all_kernel(Src src, Sink sink, SortParams P) {
                         const int it = i0 + i;
                         if (it * kThreads + tid < in_tile) {
                             kout[pos[it]] = key[it];
-                            sink.rec[pos[it]] = make_uint4(key[it], __float_as_uint(cval[i]),
+                            if (!(val[it] & 1u)) sink.cellpos[val[it] >> 1] = pos[it];
+                            sink.rec[pos[it]] = make_uint4(val[it] >> 1, __float_as_uint(cval[i]),
                                                            (uint32_t)phys_row(e_own[i], sink.S),
                                                            (uint32_t)phys_row(e_par[i], sink.S));
                         }
@@ -498,7 +500,7 @@ int radix_sort_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const 
     if (!records)
         return sort_launch(ps, src, SinkPairs{}, 2 * n_cells, nullptr, ps->key_bits, stream, 0, zero_me, zero_groups);
     SinkMF sink{d_i, d_j, d_v, (uint32_t)col_key_base, (uint32_t)ps->cfg.num_keys, ps->table,
-                ps->cfg.slots_per_part, ps->rec};
+                ps->cfg.slots_per_part, ps->rec, ps->cellpos};
     return sort_launch(ps, src, sink, 2 * n_cells, nullptr, ps->key_bits, stream, 0, zero_me, zero_groups);
 }
 
