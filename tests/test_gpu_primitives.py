@@ -156,3 +156,36 @@ def test_stress_twin_pull_push_localize_loop():
         o.localize(cfg.requester(b), keys[:cfg.localize_count])
         g.sync()
         compare_state(g, o, what=f"stress batch {b}")
+
+
+def test_push_of_a_batch_that_gives_every_sort_block_several_tiles():
+    """700k occurrences: more than one tile per block of the one-launch sort on any GPU, hot and cold keys."""
+    K, L, n = 300_000, 4, 700_001
+    g, o = make_pair(K, L, 5, K, rows=f_row(np.arange(K), L), max_batch_keys=n)      # any partition can hold every key
+    rng = np.random.default_rng(7)
+    keys = rng.integers(0, K, size=n)
+    keys[rng.random(n) < 0.2] = 123_456                          # one key a fifth of the batch
+    keys[rng.random(n) < 0.01] = K - 1
+    upd = rng.integers(-3, 4, size=(n, L)).astype(np.float32)    # integer-valued: sums are exact in any order
+    g.push(dev(keys), dev(upd))
+    g.sync()
+    o.push(keys, upd)
+    compare_state(g, o, exact_rows=True, what="large push")
+    g.localize(3, dev(keys[:250_000]))                           # a large localize sorts the same way
+    g.sync()
+    o.localize(3, keys[:250_000])
+    compare_state(g, o, exact_rows=True, what="large localize")
+
+
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 255, 256, 257, 2047, 2048, 2049, 4095, 4097, 6145])
+def test_push_sizes_around_the_sort_and_reduction_tile_borders(n):
+    K, L = 777, 8
+    g, o = make_pair(K, L, 2, rows=f_row(np.arange(K), L), max_batch_keys=8192)
+    rng = np.random.default_rng(n)
+    keys = rng.integers(0, K, size=n)
+    keys[::3] = 5                                                # a segment through every tile
+    upd = rng.integers(-3, 4, size=(n, L)).astype(np.float32)
+    g.push(dev(keys), dev(upd))
+    g.sync()
+    o.push(keys, upd)
+    compare_state(g, o, exact_rows=True, what=f"push of {n}")

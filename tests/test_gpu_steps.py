@@ -239,3 +239,30 @@ def test_pipelined_mode_gives_identical_results():
         out.append((g.export()[0].numpy(), loss_of(g)))
     assert (out[0][0] == out[1][0]).all() and out[0][1] == out[1][1]
     assert np.isfinite(out[0][1])
+
+
+def test_mf_pipelined_steps_with_relocations_in_between():
+    """In pipelined mode the key sort of a step starts early and reads the location table (it writes the row
+    addresses the gradient kernel uses): a localize between two steps must still be seen by the next step."""
+    cfg = W.MFConfig("t", 2000, 300, 100, 6 * 1500, 1500, 0.002, 0.05, 0.1, 0.5, 1.1)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    g, o = make_pair(cfg.num_keys, cfg.rank, 6, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
+    ps.ps_set_pipelining(g.h, True)
+    di, dj, dv = i.cuda(), j.cuda(), v.cuda()
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(3)
+    for b in range(cfg.n_batches):
+        s, c = cfg.batch_range(b)
+        ps.ps_step_mf(g.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+        o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+        # the keys of the NEXT batch move to another partition before it runs
+        nxt = np.concatenate([i[s + c:s + 2 * c].numpy().astype(np.int64),
+                              cfg.col_key_base + j[s + c:s + 2 * c].numpy().astype(np.int64)])
+        if len(nxt):
+            w = int(rng.integers(0, 6))
+            g.localize(w, dev(nxt))
+            o.localize(w, nxt)
+    g.sync()
+    compare_state(g, o, what="pipelined mf with relocations")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
