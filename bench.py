@@ -218,11 +218,10 @@ class MFWorkload:
         return {
             # batch arrays in (twice: keys, then records), two table entries per occurrence, keys and records out
             "sort_all_kernel": sort_bytes(occ, bits, extra=2 * b * 12 + occ * (16 + 4 + 16)),
-            # the step's pull, gradient and push except the last write of the column rows: the algorithmic bytes of
-            # the step (a table entry and a row per occurrence, read + write of every distinct row) less those writes
-            "mf_sub_kernel": b * 12 + occ * (8 + rb) + u * 2 * rb - n_unique(self.j[sl]) * rb,
-            # new column rows written into the store (they are read from staging rows: scratch, not counted)
-            "push_fixup_kernel": n_unique(self.j[sl]) * rb,
+            # the step's pull, gradient and push: the algorithmic bytes of the step (a table entry and a row per
+            # occurrence, read + write of every distinct row); the fix-up launch only finishes segments that cross
+            # tile borders and moves the few rows that had to be staged
+            "mf_sub_kernel": b * 12 + occ * (8 + rb) + u * 2 * rb,
         }
 
     # --- oracle leg ---

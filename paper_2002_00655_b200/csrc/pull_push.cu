@@ -692,6 +692,10 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
         own[c] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     float nw = 0.f, loss_f = 0.f;                   // this lane's share of |own|^2 and of the tile's loss
+    // A column factor's new row may go straight into the store if nobody else reads the row: its readers are the
+    // positions of its own segment and, as a partner, the row-factor positions of its cells, and those are all
+    // skipped if every position of the segment also updates its partner.
+    bool direct = false;
     uint32_t uses = 0;
     int st_use = 0, st_fill = kMfStages - 1;
     const int n_steps = usable_mask ? kMfTile : 0;  // (a warp of skipped positions has nothing to walk)
@@ -715,8 +719,11 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
         const uint32_t f = __shfl_sync(full, flags, src);
         const float v = __shfl_sync(full, val, src);
         const uint64_t drow = base + src;           // a finished row goes to the staging row of its position
-        const uint32_t prow_s = __shfl_sync(full, prow, src);
+        const uint32_t prow_s = __shfl_sync(full, prow, src), row_s = __shfl_sync(full, row, src);
         const bool live = f & kFUsable;
+        constexpr uint32_t kFDirect = kFBoth | kFColumn;
+        if (f & kFBegin) direct = true;
+        if (live) direct = direct && (f & kFDirect) == kFDirect;
         if (f & kFBegin) {
             nw = 0.f;
 #pragma unroll
@@ -763,9 +770,11 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
                     r.y = own[c].y + lr * (e * h[c].y - lam * own[c].y);
                     r.z = own[c].z + lr * (e * h[c].z - lam * own[c].z);
                     r.w = own[c].w + lr * (e * h[c].w - lam * own[c].w);
-                    staged[drow * L4 + l8 + 8 * c] = r;
+                    if (direct) store[(uint64_t)row_s * L4 + l8 + 8 * c] = r;
+                    else staged[drow * L4 + l8 + 8 * c] = r;
                 }
             }
+            if (direct && l8 == 0) apply_row[drow] = ~0ull;     // nothing to move later
         } else if (live) {
 #pragma unroll
             for (int c = 0; c < kC; ++c) {
@@ -787,9 +796,11 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
                         float4 r = own[c];
                         r.x = (float)((double)r.x + acc[c].x); r.y = (float)((double)r.y + acc[c].y);
                         r.z = (float)((double)r.z + acc[c].z); r.w = (float)((double)r.w + acc[c].w);
-                        staged[drow * L4 + fi] = r;
+                        if (direct) store[(uint64_t)row_s * L4 + fi] = r;
+                        else staged[drow * L4 + fi] = r;
                     }
                 }
+                if (direct && !(f & kFParked) && l8 == 0) apply_row[drow] = ~0ull;
             }
         }
     }
