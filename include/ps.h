@@ -238,6 +238,21 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream);
  * handle's earlier work has completed. */
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
 
+/* Overlap of host batches with the steps before them (the same latency hiding of
+ * Section 2.2, one level further out: the next batch travels while the current
+ * one is processed).  It concerns the ps_step_*_host calls.
+ * Off (default): such a call copies its batch on `stream`, runs the step, copies
+ * the loss back and waits for the stream.
+ * On: the batch is copied on an internal stream into one of three staging areas
+ * as soon as the step that last used the area is through, the step's kernels
+ * wait for that copy, and the call returns WITHOUT waiting: the h_* arrays must
+ * stay unchanged, and *h_loss is not valid, until ps_sync (or another wait for
+ * `stream`) has returned.  Give every call in flight its own h_loss word.  With
+ * ps_set_pipelining on, the key sort of the next batch also starts as soon as its
+ * copy has landed.  Results are identical in both modes.  The switch itself waits
+ * for the device.  Do not capture ps_step_*_host calls into a CUDA graph. */
+ps_status_t ps_set_host_overlap(ps_store_t* ps, int on);
+
 /* Number of kernels this handle has launched so far. */
 uint64_t ps_launch_count(const ps_store_t* ps);
 

@@ -65,6 +65,7 @@ SIGNATURES = {
     "ps_export_freelists": (C.c_int, [_vp, _vp, _vp]),
     "ps_sync": (C.c_int, [_vp, _vp]),
     "ps_set_pipelining": (C.c_int, [_vp, C.c_int]),
+    "ps_set_host_overlap": (C.c_int, [_vp, C.c_int]),
     "ps_launch_count": (C.c_uint64, [_vp]),
     "ps_rows_moved": (C.c_int, [_vp, C.POINTER(_u64)]),
     "ps_profile_start": (C.c_int, [_vp, _u32]),
@@ -238,6 +239,10 @@ def ps_export_freelists(ps, h_stacks=None, h_tops=None):
 def ps_sync(ps) -> int:
     """Waits for the current stream; returns (and clears) the first error latched on the device."""
     return load_library().ps_sync(ps, _stream())
+
+
+def ps_set_host_overlap(ps, on: bool) -> None:
+    _check(load_library().ps_set_host_overlap(ps, 1 if on else 0), "ps_set_host_overlap")
 
 
 def ps_set_pipelining(ps, on: bool) -> None:

@@ -48,7 +48,7 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     l.group_sum = take(groups * (size_t)cfg.row_len * 8);
     l.loss_partial = take(tmax<size_t>(kMaxLossBlocks, mk / 256 + 1) * 8);
     l.apply_rows = take(mk * 8);
-    l.staging = take(mk * 8 + 256);
+    for (int b = 0; b < kHostStages; ++b) l.staging[b] = take(mk * 8 + 256);
     l.total = off;
     return l;
 }
@@ -133,6 +133,11 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_tabl
     // When the caller's stream enters or leaves a CUDA-graph capture, events recorded on the other side of
     // that border cannot be waited on, and the side stream has to join (or leave) the capture: the first
     // call after such a change forks in ordered mode and forgets the older events.
+    if (ps->batch_ready) {                  // the call's batch is still being copied from the host on the copy stream
+        const cudaEvent_t ev = ps->batch_ready;
+        ps->batch_ready = nullptr;
+        if (cudaStreamWaitEvent(ps->side, ev, 0) != cudaSuccess) return false;
+    }
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
     unsigned long long id = 0;
     if (cudaStreamGetCaptureInfo(s, &cs, &id) != cudaSuccess) return false;
@@ -237,7 +242,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->group_sum = (double*)(ps->ws + l.group_sum);
     ps->loss_partial = (double*)(ps->ws + l.loss_partial);
     ps->apply_rows = (uint64_t*)(ps->ws + l.apply_rows);
-    ps->staging = ps->ws + l.staging;
+    for (int b = 0; b < kHostStages; ++b) ps->stagings[b] = ps->ws + l.staging[b];
+    ps->staging = ps->stagings[0];
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0) {
         delete ps;
@@ -269,6 +275,16 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
             delete ps;
             return PS_ERR_CUDA;
         }
+    if (cudaStreamCreateWithFlags(&ps->copy, cudaStreamNonBlocking) != cudaSuccess) {
+        delete ps;
+        return PS_ERR_CUDA;
+    }
+    for (int b = 0; b < kHostStages; ++b)
+        if (cudaEventCreateWithFlags(&ps->ev_copied[b], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ps->ev_consumed[b], cudaEventDisableTiming) != cudaSuccess) {
+            delete ps;
+            return PS_ERR_CUDA;
+        }
     *out = ps;
     return PS_OK;
 }
@@ -283,6 +299,11 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     cudaEventDestroy(ps->ev_mid);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
     cudaStreamDestroy(ps->side);
+    cudaStreamDestroy(ps->copy);
+    for (int b = 0; b < kHostStages; ++b) {
+        cudaEventDestroy(ps->ev_copied[b]);
+        cudaEventDestroy(ps->ev_consumed[b]);
+    }
     delete ps;
     return PS_OK;
 }
@@ -425,10 +446,46 @@ ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t firs
 }
 
 // ---- host-batch variants ----
-static ps_status_t finish_host_step(double* d_loss_accum, double* h_loss, cudaStream_t s) {
+// Where a host batch is copied to and on which stream.  Plain mode: the one staging area, the caller's stream.
+// Overlapped mode (ps_set_host_overlap): the next of kHostStages areas, on the handle's copy stream, as soon as
+// the step that last read that area is through; the step's kernels then wait for the copy, not the other way round.
+struct HostBatch {
+    char* buf;
+    cudaStream_t cs;
+    int slot;               // -1 in plain mode
+};
+static bool host_batch_begin(ps_store* ps, cudaStream_t s, HostBatch* hb) {
+    if (!ps->host_overlap) {
+        hb->buf = ps->stagings[0];
+        hb->cs = s;
+        hb->slot = -1;
+        return true;
+    }
+    ps->host_slot = (ps->host_slot + 1) % kHostStages;
+    hb->slot = ps->host_slot;
+    hb->buf = ps->stagings[hb->slot];
+    hb->cs = ps->copy;
+    return !ps->consumed_valid[hb->slot] || cudaStreamWaitEvent(ps->copy, ps->ev_consumed[hb->slot], 0) == cudaSuccess;
+}
+// after the copies have been enqueued: every stream that reads the batch waits for them
+static bool host_batch_copied(ps_store* ps, cudaStream_t s, const HostBatch& hb) {
+    if (hb.slot < 0) return true;
+    if (cudaEventRecord(ps->ev_copied[hb.slot], ps->copy) != cudaSuccess ||
+        cudaStreamWaitEvent(s, ps->ev_copied[hb.slot], 0) != cudaSuccess)
+        return false;
+    ps->batch_ready = ps->ev_copied[hb.slot];       // picked up by the step's fork of the side stream
+    return true;
+}
+static ps_status_t finish_host_step(ps_store* ps, const HostBatch& hb, double* d_loss_accum, double* h_loss,
+                                    cudaStream_t s) {
     if (d_loss_accum && h_loss &&
         cudaMemcpyAsync(h_loss, d_loss_accum, sizeof(double), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return PS_ERR_CUDA;
+    if (hb.slot >= 0) {                              // overlapped mode: nothing waits; the area is free once s gets here
+        if (cudaEventRecord(ps->ev_consumed[hb.slot], s) != cudaSuccess) return PS_ERR_CUDA;
+        ps->consumed_valid[hb.slot] = true;
+        return PS_OK;
+    }
     if (cudaStreamSynchronize(s) != cudaSuccess) return PS_ERR_CUDA;
     return PS_OK;
 }
@@ -441,19 +498,22 @@ ps_status_t ps_step_mf_host(ps_store_t* ps, const uint32_t* h_i, const uint32_t*
     if (!h_i || !h_j || !h_v) return PS_ERR_INVALID_ARG;
     if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
-    uint32_t* d_i = (uint32_t*)ps->staging;
+    HostBatch hb;
+    if (!host_batch_begin(ps, s, &hb)) return PS_ERR_CUDA;
+    uint32_t* d_i = (uint32_t*)hb.buf;
     uint32_t* d_j = d_i + n;
     float* d_v = (float*)(d_j + n);
-    if (cudaMemcpyAsync(d_i, h_i, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_j, h_j, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_v, h_v, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    if (cudaMemcpyAsync(d_i, h_i, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess ||
+        cudaMemcpyAsync(d_j, h_j, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess ||
+        cudaMemcpyAsync(d_v, h_v, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess)
         return PS_ERR_CUDA;
-    const bool was = ps->pipelined;         // the batch arrives on the caller's stream: order the side stream after it
-    ps->pipelined = false;
+    if (!host_batch_copied(ps, s, hb)) return PS_ERR_CUDA;
+    const bool was = ps->pipelined;         // plain mode: the batch arrives on the caller's stream, order the side stream after it
+    if (hb.slot < 0) ps->pipelined = false;
     const ps_status_t c = ps_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, d_loss_accum, stream);
     ps->pipelined = was;
     if (c != PS_OK) return c;
-    return finish_host_step(d_loss_accum, h_loss, s);
+    return finish_host_step(ps, hb, d_loss_accum, h_loss, s);
 }
 
 ps_status_t ps_step_kge_host(ps_store_t* ps, const uint32_t* h_s, const uint32_t* h_r, const uint32_t* h_o,
@@ -465,25 +525,28 @@ ps_status_t ps_step_kge_host(ps_store_t* ps, const uint32_t* h_s, const uint32_t
     if (!h_s || !h_r || !h_o || (n_neg && (!h_neg_ent || !h_neg_side))) return PS_ERR_INVALID_ARG;
     if ((3 + (uint64_t)n_neg) * n > ps->max_keys) return PS_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
-    uint32_t* d_s = (uint32_t*)ps->staging;
+    HostBatch hb;
+    if (!host_batch_begin(ps, s, &hb)) return PS_ERR_CUDA;
+    uint32_t* d_s = (uint32_t*)hb.buf;
     uint32_t* d_r = d_s + n;
     uint32_t* d_o = d_r + n;
     uint32_t* d_ne = d_o + n;
     uint8_t* d_ns = (uint8_t*)(d_ne + n * n_neg);
-    if (cudaMemcpyAsync(d_s, h_s, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_r, h_r, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_o, h_o, n * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    if (cudaMemcpyAsync(d_s, h_s, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess ||
+        cudaMemcpyAsync(d_r, h_r, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess ||
+        cudaMemcpyAsync(d_o, h_o, n * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess)
         return PS_ERR_CUDA;
-    if (n_neg && (cudaMemcpyAsync(d_ne, h_neg_ent, n * n_neg * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-                  cudaMemcpyAsync(d_ns, h_neg_side, n * n_neg, cudaMemcpyHostToDevice, s) != cudaSuccess))
+    if (n_neg && (cudaMemcpyAsync(d_ne, h_neg_ent, n * n_neg * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess ||
+                  cudaMemcpyAsync(d_ns, h_neg_side, n * n_neg, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess))
         return PS_ERR_CUDA;
-    const bool was = ps->pipelined;         // the batch arrives on the caller's stream: order the side stream after it
-    ps->pipelined = false;
+    if (!host_batch_copied(ps, s, hb)) return PS_ERR_CUDA;
+    const bool was = ps->pipelined;         // plain mode: the batch arrives on the caller's stream, order the side stream after it
+    if (hb.slot < 0) ps->pipelined = false;
     const ps_status_t c = ps_step_kge(ps, d_s, d_r, d_o, d_ne, d_ns, n, n_neg, rel_key_base, dim_complex, lr, eps,
                                       d_loss_accum, stream);
     ps->pipelined = was;
     if (c != PS_OK) return c;
-    return finish_host_step(d_loss_accum, h_loss, s);
+    return finish_host_step(ps, hb, d_loss_accum, h_loss, s);
 }
 
 ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t tok_first, uint64_t tok_count,
@@ -504,15 +567,20 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     if ((tok_count + n_negs) * 4 > ps->max_keys * 8) return PS_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
     next_epoch(ps);
-    uint32_t* d_tok = (uint32_t*)ps->staging;
+    HostBatch hb;
+    if (!host_batch_begin(ps, s, &hb)) return PS_ERR_CUDA;
+    uint32_t* d_tok = (uint32_t*)hb.buf;
     uint32_t* d_negs = d_tok + tok_count;
-    if (cudaMemcpyAsync(d_tok, h_tokens, tok_count * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return PS_ERR_CUDA;
-    if (n_negs && cudaMemcpyAsync(d_negs, h_negs, n_negs * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    if (cudaMemcpyAsync(d_tok, h_tokens, tok_count * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess) return PS_ERR_CUDA;
+    if (n_negs && cudaMemcpyAsync(d_negs, h_negs, n_negs * 4, cudaMemcpyHostToDevice, hb.cs) != cudaSuccess)
         return PS_ERR_CUDA;
+    if (!host_batch_copied(ps, s, hb)) return PS_ERR_CUDA;
     SortSet* ss = next_set(ps);
-    // the batch was just copied on the caller's stream: the side stream has to wait for that
-    if (cudaEventRecord(ps->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) != cudaSuccess)
-        return PS_ERR_CUDA;
+    if (hb.slot >= 0) {
+        if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;      // waits for the copy; pipelined or ordered as the handle is set
+    } else if (cudaEventRecord(ps->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) != cudaSuccess) {
+        return PS_ERR_CUDA;                                  // the batch was just copied on the caller's stream
+    }
     launch_keys_sgns(ps, d_tok, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base,
                      ps->side);
     const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
@@ -523,7 +591,7 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
                     sgns_scales(ps, n_centers), (uint32_t)(occ / n_centers));
     c = release_set(ss, s);
     if (c != PS_OK) return c;
-    return finish_host_step(d_loss_accum, h_loss, s);
+    return finish_host_step(ps, hb, d_loss_accum, h_loss, s);
 }
 
 ps_status_t ps_get_location(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner, uint32_t* d_slot,
@@ -588,6 +656,15 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream) {
             if (cudaMemset(ps->sets[b].sort_ctl, 0, kSortCtlWords * sizeof(uint32_t)) != cudaSuccess) return PS_ERR_CUDA;
     }
     return (ps_status_t)code;
+}
+
+ps_status_t ps_set_host_overlap(ps_store_t* ps, int on) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;     // no host batch in flight across the switch
+    ps->host_overlap = on != 0;
+    for (int b = 0; b < kHostStages; ++b) ps->consumed_valid[b] = false;
+    ps->batch_ready = nullptr;
+    return PS_OK;
 }
 
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on) {

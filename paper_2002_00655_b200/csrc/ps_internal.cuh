@@ -20,6 +20,7 @@ constexpr int kSortCtlWords = kMaxSortPasses * kRadix + kMaxSortPasses;   // dig
 constexpr int kReduceTile = 32;                  // sorted occurrences per warp in the segmented reduction
 constexpr int kGroupSpan = 64 * kReduceTile;      // sorted positions whose parked parts are pre-added together
 constexpr int kMaxLossBlocks = 4096;
+constexpr int kHostStages = 3;                   // staging areas for batches that arrive from host memory
 constexpr int kSortSets = 3;                     // calls whose key sort may be in flight at once (see SortSet)
 
 // Device-resident status words.  An error is latched per call with the call's
@@ -83,7 +84,8 @@ struct ps_store {
     unsigned int* starter_count;
     double* loss_partial;           // max(kMaxLossBlocks, one per 256 key occurrences)
     uint64_t* apply_rows;           // per sorted position: address of the row staged there, or all ones
-    char* staging;                  // host-batch staging, max_keys x 8 bytes
+    char* staging;                  // host-batch staging, max_keys x 8 bytes (the first of `stagings`)
+    char* stagings[psb::kHostStages];
     // host state
     uint32_t epoch;
     uint64_t launches;
@@ -95,6 +97,12 @@ struct ps_store {
     bool mid_valid;
     psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
+    cudaStream_t copy;              // host batches are copied here in overlapped mode (ps_set_host_overlap)
+    cudaEvent_t ev_copied[psb::kHostStages], ev_consumed[psb::kHostStages];
+    bool consumed_valid[psb::kHostStages];
+    int host_slot;
+    bool host_overlap;
+    cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
     bool table_dirty;               // the location table was rewritten since the side stream last waited for the caller's
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
@@ -105,7 +113,7 @@ namespace psb {
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
         sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
-        loss_partial, apply_rows, staging, total;
+        loss_partial, apply_rows, staging[kHostStages], total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
 

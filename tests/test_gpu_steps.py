@@ -266,3 +266,36 @@ def test_mf_pipelined_steps_with_relocations_in_between():
     g.sync()
     compare_state(g, o, what="pipelined mf with relocations")
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
+def test_overlapped_host_batches_give_identical_results():
+    """ps_set_host_overlap: batches are copied on the library's copy stream while earlier steps run and the
+    calls do not wait; parameters and every step's loss must equal those of the device-batch calls."""
+    cfg = W.scaled(W.MF_TINY, rows=3000, cols=400, rank=100, n_cells=24 * 2048, batch=2048, col_zipf=1.1, lr=0.0005)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    hi, hj, hv = i.pin_memory(), j.pin_memory(), v.pin_memory()
+    a, _ = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
+    losses = []
+    for b in range(cfg.n_batches):
+        s, c = cfg.batch_range(b)
+        ps.ps_step_mf(a.h, i[s:s + c].cuda(), j[s:s + c].cuda(), v[s:s + c].cuda(), cfg.col_key_base, cfg.lr, cfg.lam, a.loss)
+        a.sync()
+        losses.append(loss_of(a))
+    want = a.export(table=False)[0]
+    for pipelined in (False, True):
+        g, _ = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
+        ps.ps_set_pipelining(g.h, pipelined)
+        ps.ps_set_host_overlap(g.h, True)
+        h_loss = torch.zeros(cfg.n_batches, dtype=torch.float64).pin_memory()
+        for b in range(cfg.n_batches):
+            s, c = cfg.batch_range(b)
+            ps.ps_step_mf_host(g.h, hi[s:s + c], hj[s:s + c], hv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss,
+                               h_loss[b:b + 1])
+        g.sync()
+        assert (h_loss.numpy() == np.array(losses)).all()
+        assert (g.export(table=False)[0] == want).all()
+        ps.ps_set_host_overlap(g.h, False)                      # back to calls that wait
+        s, c = cfg.batch_range(0)
+        ps.ps_step_mf_host(g.h, hi[s:s + c], hj[s:s + c], hv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss, h_loss[0:1])
+        assert h_loss[0] == loss_of(g)
