@@ -356,6 +356,7 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     if (n == 0) return PS_OK;
     if (!d_keys) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    if (n > (1u << 20)) return PS_ERR_UNSUPPORTED;          // one block scans the call's per-chunk counts in shared memory
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, nullptr, 0);

@@ -26,36 +26,6 @@
 
 namespace psb {
 
-constexpr unsigned kBarrierSpins = 1u << 21;     // x ~100 ns: gives up after about a fifth of a second
-
-// Barrier over all blocks of a cooperative launch.  bar[0] counts arrivals and only grows while the kernel
-// runs: the k-th barrier is passed once it reaches k times the number of blocks.  bar[1] counts the blocks that
-// have left the kernel; the last one to leave puts both words back to zero, so a launch always starts from
-// zero without a clearing step in between.
-__device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int target, int* s_ok) {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;\n" ::"l"(bar) : "memory");
-        unsigned int seen = 0, spins = 0;
-        for (;;) {
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(seen) : "l"(bar) : "memory");
-            if (seen >= target || spins >= kBarrierSpins) break;
-            __nanosleep(spins < 256 ? 20 : 100);
-            ++spins;
-        }
-        *s_ok = seen >= target;
-    }
-    __syncthreads();
-    return *s_ok != 0;
-}
-__device__ __forceinline__ void grid_leave(unsigned int* bar, unsigned int n_blocks) {
-    if (threadIdx.x == 0 && atomicAdd(bar + 1, 1u) == n_blocks - 1) {
-        // every other block has left, so nobody is waiting on the arrival count any more
-        atomicExch(bar, 0u);
-        atomicExch(bar + 1, 0u);
-    }
-}
-
 struct SortParams {
     uint32_t *kA, *vA, *kB, *vB;        // pass p reads (kA, vA) if (start + p) is even, else (kB, vB)
     int start;
