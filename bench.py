@@ -735,7 +735,7 @@ def run_ours(args):
     }
     if want_cpu:
         try:
-            out["cpu_baseline"] = cpu_baseline(wl, device, min(64, total))
+            out["cpu_baseline"] = cpu_baseline(wl, device, min(256, total))
         except MemoryError as e:
             out["cpu_baseline"] = {"unavailable": f"host memory: {e}"}
     if rank == 0:
