@@ -220,16 +220,21 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
 // expression is evaluated in fp32 on the rounded gradient.
 // kMaxNeg bounds n_neg at compile time so that a data point's values live in registers: for every block
 // of 32 complex dimensions the Re and Im of all its rows are requested together, before any is used.
-template <int kMaxNeg>
+// kDim / kExactNeg: the complex dimension and "n_neg equals kMaxNeg" known at compile time (0 / false: taken from
+// the arguments).  With both fixed the offsets of the four quarters of a row become immediates and the tests on
+// the number of negatives fold away; the kernel spends more issue slots on integer bookkeeping than on fp64.
+template <int kMaxNeg, int kDim, bool kExactNeg>
 __global__ void __launch_bounds__(256, kMaxNeg <= 10 ? 2 : 1)
 kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                 const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
-                uint32_t n_neg, uint64_t rel_base, uint32_t d, float lr, float eps, const float* __restrict__ store,
+                uint32_t n_neg_arg, uint64_t rel_base, uint32_t d_arg, float lr, float eps, const float* __restrict__ store,
                 const uint2* __restrict__ table, uint64_t S, uint64_t K, float* __restrict__ upd,
                 double* __restrict__ loss_partial, DevStatus* st, unsigned int epoch) {
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t d = kDim ? (uint32_t)kDim : d_arg;
+    const uint32_t n_neg = kExactNeg ? (uint32_t)kMaxNeg : n_neg_arg;
     const int n_slots = 3 + (int)n_neg;
     const uint32_t L = 4 * d;
     const unsigned full = 0xffffffffu;
@@ -440,9 +445,27 @@ uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r,
 #define KGE_ARGS d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, lr, eps,                     \
                  (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->upd,         \
                  ps->loss_partial, ps->status, ps->epoch
-    if (n_neg <= 4) PS_LAUNCH(ps, kge_step_kernel<4>, grid, 256, s, KGE_ARGS);
-    else if (n_neg <= 10) PS_LAUNCH(ps, kge_step_kernel<10>, grid, 256, s, KGE_ARGS);
-    else PS_LAUNCH(ps, kge_step_kernel<29>, grid, 256, s, KGE_ARGS);
+    if (n_neg == 10 && dim == 100) {
+        if (ps->prof) prof_before(ps, "kge_step_kernel<10>", s);
+        kge_step_kernel<10, 100, true><<<grid, 256, 0, s>>>(KGE_ARGS);
+        if (ps->prof) prof_after(ps, s);
+        ps->launches++;
+    } else if (n_neg <= 4) {
+        if (ps->prof) prof_before(ps, "kge_step_kernel<4>", s);
+        kge_step_kernel<4, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
+        if (ps->prof) prof_after(ps, s);
+        ps->launches++;
+    } else if (n_neg <= 10) {
+        if (ps->prof) prof_before(ps, "kge_step_kernel<10>", s);
+        kge_step_kernel<10, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
+        if (ps->prof) prof_after(ps, s);
+        ps->launches++;
+    } else {
+        if (ps->prof) prof_before(ps, "kge_step_kernel<29>", s);
+        kge_step_kernel<29, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
+        if (ps->prof) prof_after(ps, s);
+        ps->launches++;
+    }
 #undef KGE_ARGS
     return grid;
 }
