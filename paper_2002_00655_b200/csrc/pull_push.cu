@@ -386,17 +386,22 @@ __device__ __noinline__ void group_preadd(const uint32_t* __restrict__ sk, uint3
 // kScaled: occurrence o does not have an update row of its own.  Its update is scales[o] times a source
 // row shared with other occurrences: the occurrences come in runs of `slots` per example, example e owning
 // source rows 2e (used, by its slot 0) and 2e + 1 (used by all its other slots) of `upd`.
-template <int kCh, bool kScaled>
+//
+// kL4 / kSlots: the row length in float4 and the slots per example if known at compile time (0: taken from the
+// arguments); row offsets, the copy size and the division by the slots then fold.
+template <int kCh, bool kScaled, int kL4, int kSlots>
 __global__ void __launch_bounds__(256)
 push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
-                   const float4* __restrict__ upd, const float* __restrict__ scales, uint32_t slots,
+                   const float4* __restrict__ upd, const float* __restrict__ scales, uint32_t slots_arg,
                    float4* __restrict__ store, const uint2* __restrict__ table,
-                   uint64_t S, uint32_t K, uint32_t L4, double* __restrict__ carry,
+                   uint64_t S, uint32_t K, uint32_t L4_arg, double* __restrict__ carry,
                    uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
                    unsigned int* __restrict__ group_done, double* __restrict__ group_sum,
                    DevStatus* st, unsigned int epoch) {
     __shared__ unsigned int s_ticket;
     __shared__ __align__(8) uint64_t bars[8][3];    // per warp and stage: the barrier word its copies report to
+    const uint32_t L4 = kL4 ? (uint32_t)kL4 : L4_arg;
+    const uint32_t slots = kSlots ? (uint32_t)kSlots : slots_arg;
     if (call_failed(st, epoch)) return;
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -1133,29 +1138,33 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
 #define REDUCE_ARGS sk, sv, n, (const float4*)d_upd, d_scales, slots, (float4*)ps->store, ps->table,                 \
                     ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4, ps->carry, ps->starters,                \
                     ps->starter_count, ps->group_done, ps->group_sum, ps->status, ps->epoch
-#define REDUCE_LAUNCH(kCh, kScaled)                                                                                  \
+#define REDUCE_LAUNCH(kCh, kScaled, kL4, kSlots)                                                                     \
     do {                                                                                                             \
         static bool smem_set = false;                                                                                \
         if (!smem_set) {                                                                                             \
-            cudaFuncSetAttribute(push_reduce_kernel<kCh, kScaled>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
-                                 (int)reduce_smem(kCh));                                                             \
+            cudaFuncSetAttribute(push_reduce_kernel<kCh, kScaled, kL4, kSlots>,                                      \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kCh));                \
             smem_set = true;                                                                                         \
         }                                                                                                            \
         if (ps->prof) prof_before(ps, "push_reduce_kernel<" #kCh "," #kScaled ">", s);                               \
-        push_reduce_kernel<kCh, kScaled><<<blocks, 256, reduce_smem(kCh), s>>>(REDUCE_ARGS);                         \
+        push_reduce_kernel<kCh, kScaled, kL4, kSlots><<<blocks, 256, reduce_smem(kCh), s>>>(REDUCE_ARGS);            \
         if (ps->prof) prof_after(ps, s);                                                                             \
         ps->launches++;                                                                                              \
     } while (0)
+    // the row lengths of the paper's workloads get kernels of their own: 128, 300 (41 slots per center) and 400 values
     if (d_scales) {
-        if (L4 <= 32) REDUCE_LAUNCH(1, true);
-        else if (L4 <= 64) REDUCE_LAUNCH(2, true);
-        else if (L4 <= 96) REDUCE_LAUNCH(3, true);
-        else REDUCE_LAUNCH(4, true);
+        if (L4 == 75 && slots == 41) REDUCE_LAUNCH(3, true, 75, 41);
+        else if (L4 <= 32) REDUCE_LAUNCH(1, true, 0, 0);
+        else if (L4 <= 64) REDUCE_LAUNCH(2, true, 0, 0);
+        else if (L4 <= 96) REDUCE_LAUNCH(3, true, 0, 0);
+        else REDUCE_LAUNCH(4, true, 0, 0);
     } else {
-        if (L4 <= 32) REDUCE_LAUNCH(1, false);
-        else if (L4 <= 64) REDUCE_LAUNCH(2, false);
-        else if (L4 <= 96) REDUCE_LAUNCH(3, false);
-        else REDUCE_LAUNCH(4, false);
+        if (L4 == 32) REDUCE_LAUNCH(1, false, 32, 0);
+        else if (L4 == 100) REDUCE_LAUNCH(4, false, 100, 0);
+        else if (L4 <= 32) REDUCE_LAUNCH(1, false, 0, 0);
+        else if (L4 <= 64) REDUCE_LAUNCH(2, false, 0, 0);
+        else if (L4 <= 96) REDUCE_LAUNCH(3, false, 0, 0);
+        else REDUCE_LAUNCH(4, false, 0, 0);
     }
 #undef REDUCE_LAUNCH
 #undef REDUCE_ARGS

@@ -499,17 +499,22 @@ __device__ __forceinline__ uint64_t sgns_pairs_before(uint64_t p, uint64_t T, ui
 // A warp takes one center at a time.  The output-vector slots are handled 32 at a time: every lane first
 // resolves one slot (word -> key -> table entry -> row address), so those lookups are in flight together;
 // the rows are then read four slots at a time, all loads of the four before the first dot product.
-template <int kCh>
+// kL4, kWindow, kNeg: row length (float4), window and negatives per context if known at compile time (0: taken
+// from the arguments; kNeg < 0: from the argument); divisions by the slots per context and row offsets then fold.
+template <int kCh, int kL4, int kWindow, int kNeg>
 __global__ void __launch_bounds__(256, 2)
 sgns_step_kernel(const uint32_t* __restrict__ tokens, uint64_t tok_first, uint64_t first_pos, uint64_t n_centers,
-                 uint64_t T, uint32_t window, const uint32_t* __restrict__ negs, uint32_t n_neg, uint64_t out_base,
+                 uint64_t T, uint32_t window_arg, const uint32_t* __restrict__ negs, uint32_t n_neg_arg, uint64_t out_base,
                  float lr, const float4* __restrict__ store, const uint2* __restrict__ table, uint64_t S, uint64_t K,
-                 uint32_t L4, float4* __restrict__ upd, float* __restrict__ scales, double* __restrict__ loss_partial,
+                 uint32_t L4_arg, float4* __restrict__ upd, float* __restrict__ scales, double* __restrict__ loss_partial,
                  DevStatus* st, unsigned int epoch) {
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = kL4 ? (uint32_t)kL4 : L4_arg;
+    const uint32_t window = kWindow ? (uint32_t)kWindow : window_arg;
+    const uint32_t n_neg = kNeg >= 0 ? (uint32_t)kNeg : n_neg_arg;
     const uint32_t per_ctx = 1 + n_neg;
     const uint64_t slots = 1 + (uint64_t)2 * window * per_ctx;
     const uint64_t pairs0 = sgns_pairs_before(first_pos, T, window);
@@ -673,10 +678,19 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
 #define SG_ARGS d_tokens, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, lr,   \
                 (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4,              \
                 (float4*)ps->upd, sgns_scales(ps, n_centers), ps->loss_partial, ps->status, ps->epoch
-    if (L4 <= 32) PS_LAUNCH(ps, sgns_step_kernel<1>, grid, 256, s, SG_ARGS);
-    else if (L4 <= 64) PS_LAUNCH(ps, sgns_step_kernel<2>, grid, 256, s, SG_ARGS);
-    else if (L4 <= 96) PS_LAUNCH(ps, sgns_step_kernel<3>, grid, 256, s, SG_ARGS);
-    else PS_LAUNCH(ps, sgns_step_kernel<4>, grid, 256, s, SG_ARGS);
+#define SG_LAUNCH(kCh, kL4, kW, kN)                                                                                  \
+    do {                                                                                                             \
+        if (ps->prof) prof_before(ps, "sgns_step_kernel<" #kCh ">", s);                                              \
+        sgns_step_kernel<kCh, kL4, kW, kN><<<grid, 256, 0, s>>>(SG_ARGS);                                            \
+        if (ps->prof) prof_after(ps, s);                                                                             \
+        ps->launches++;                                                                                              \
+    } while (0)
+    if (L4 == 75 && window == 5 && n_neg == 3) SG_LAUNCH(3, 75, 5, 3);     // 300 values, window 5, 3 negatives
+    else if (L4 <= 32) SG_LAUNCH(1, 0, 0, -1);
+    else if (L4 <= 64) SG_LAUNCH(2, 0, 0, -1);
+    else if (L4 <= 96) SG_LAUNCH(3, 0, 0, -1);
+    else SG_LAUNCH(4, 0, 0, -1);
+#undef SG_LAUNCH
 #undef SG_ARGS
     return grid;
 }
