@@ -80,16 +80,19 @@ __device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned 
                  "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
 }
-// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.
-constexpr unsigned kBarPollLimit = 1u << 22;
+// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.  Each poll
+// may stay suspended in hardware for up to kBarSuspendNs (it returns as soon as the phase completes), so that a
+// waiting warp does not spend issue slots on polling: about a quarter of a second per call at most.
+constexpr unsigned kBarPollLimit = 1u << 17;
+constexpr unsigned kBarSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
     const unsigned a = smem_addr(bar);
     for (unsigned i = 0; i < kBarPollLimit; ++i) {
         unsigned done;
         asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
             : "=r"(done)
-            : "r"(a), "r"(parity)
+            : "r"(a), "r"(parity), "r"(kBarSuspendNs)
             : "memory");
         if (done) return true;
     }
