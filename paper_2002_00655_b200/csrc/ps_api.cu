@@ -144,19 +144,12 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_tabl
     if (cs != cudaStreamCaptureStatusActive) id = 0;
     const bool crossed = id != ps->capture_id;
     ps->capture_id = id;
-    if (crossed) {
+    if (crossed)
         for (int b = 0; b < kSortSets; ++b) ps->sets[b].used = false;
-        ps->mid_valid = false;
-    }
     // a sort that reads the location table (the matrix-factorization records) must come after a call that rewrote it
     const bool ordered = crossed || (reads_table && ps->table_dirty);
     if (ordered) ps->table_dirty = false;
-    if (ps->pipelined && !ordered) {
-        // not before the previous step's first kernel is through: the sort's blocks wait at grid barriers most of
-        // the time and would hold registers that kernel's blocks need (see run_mf_fused)
-        if (ps->mid_valid && cudaStreamWaitEvent(ps->side, ps->ev_mid, 0) != cudaSuccess) return false;
-        return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
-    }
+    if (ps->pipelined && !ordered) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
@@ -265,8 +258,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
     if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_mid, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
     }
@@ -296,7 +288,6 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
-    cudaEventDestroy(ps->ev_mid);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
     cudaStreamDestroy(ps->side);
     cudaStreamDestroy(ps->copy);

@@ -93,8 +93,6 @@ struct ps_store {
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
     cudaStream_t side;              // key extraction and sort of a step run here, beside the gradient kernel
     cudaEvent_t ev_fork, ev_join;
-    cudaEvent_t ev_mid;             // recorded after the first of a step's kernels on the caller's stream
-    bool mid_valid;
     psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
     cudaStream_t copy;              // host batches are copied here in overlapped mode (ps_set_host_overlap)

@@ -20,8 +20,6 @@
 //
 // The only waiting is the grid barrier; it is bounded, and a block that gives
 // up latches an error and returns.
-#include <cooperative_groups.h>
-
 #include "ps_internal.cuh"
 
 namespace psb {
