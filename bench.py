@@ -117,7 +117,6 @@ def smi_clocks():
 # keyed by (workload, kernel).  An entry is removed when its kernel changes after the capture.
 TRAFFIC = {
     ("mf_large", "mf_sub_kernel<4>"): 46.4e6,                   # profiles/mf_step_kernels_ncu_full.md (same-batch twin)
-    ("kge", "kge_step_kernel<10>"): 296.2e6,                    # profiles/kge_step_kernels_ncu_full.md
     ("sgns", "push_reduce_kernel<3,true>"): 1557.5e6,           # profiles/sgns_step_kernels_ncu_full.md
 }
 
@@ -317,8 +316,14 @@ class KGEWorkload:
     def kernel_bytes(self, k):
         c, sl, b = self.cfg, self._sl(k), self.cfg.batch
         u = n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl])
-        return kernel_bytes_of_step(b * (12 + c.n_neg * 5), (3 + c.n_neg) * b, u, self.row_bytes, "kge_keys", "kge_step",
-                                    int(c.num_keys).bit_length())
+        kb = kernel_bytes_of_step(b * (12 + c.n_neg * 5), (3 + c.n_neg) * b, u, self.row_bytes, "kge_keys", "kge_step",
+                                  int(c.num_keys).bit_length())
+        occ, rb = (3 + c.n_neg) * b, self.row_bytes
+        # the step kernel reads the embedding half of every row and writes a gradient row of the same size; the
+        # reduction reads those and read-modify-writes every distinct row
+        kb["kge_step"] = b * (12 + c.n_neg * 5) + occ * (8 + rb // 2) + occ * (rb // 2)
+        kb["kge_reduce_kernel"] = occ * (8 + rb // 2) + u * (8 + 2 * rb)
+        return kb
 
     def oracle_setup(self, device):
         from oracle import OracleStore

@@ -398,10 +398,13 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_kge(ps, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base, ps->side);
     const int which = run_push_sort(ps, occ, ps->side);
-    const uint32_t lb =
-        launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex, lr, eps, s);
+    // gradient rows + AdaGrad inside the reduction where a gradient row is whole float4s and fits the reduction's staging
+    const bool grad_only = dim_complex % 2 == 0 && dim_complex <= 128;
+    const uint32_t lb = launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex,
+                                        lr, eps, grad_only, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
-    run_push_reduce(ps, occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
+    if (grad_only) run_kge_reduce(ps, occ, which, dim_complex, lr, eps, d_loss_accum, d_loss_accum ? lb : 0, s);
+    else run_push_reduce(ps, occ, which, ps->upd, d_loss_accum, d_loss_accum ? lb : 0, s);
     return release_set(ss, s);
 }
 

@@ -181,6 +181,9 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
 // then the fix-up launch that also moves the staged rows into the store
 void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
                   double* d_loss_accum, cudaStream_t s);
+// ComplEx: reduce GRADIENT rows (2 dim values per occurrence, in ps->upd) into AdaGrad steps per key; dim even, <= 128
+void run_kge_reduce(ps_store* ps, uint32_t n, int which, uint32_t dim, float lr, float eps, double* d_loss_accum,
+                    uint32_t loss_blocks, cudaStream_t s);
 
 // ---- localize.cu ----
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
@@ -197,9 +200,10 @@ void launch_keys_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first
                       uint64_t out_key_base, cudaStream_t s);
 uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
                         uint64_t col_key_base, float lr, float lambda, cudaStream_t s);
+// grad_only: the update rows hold gradients (2 dim values each), to be reduced with run_kge_reduce
 uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                          const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
-                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s);
+                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, bool grad_only, cudaStream_t s);
 float* sgns_scales(ps_store* ps, uint64_t n_centers);     // where launch_step_sgns puts the per-slot factors
 uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
                           uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
@@ -225,6 +229,12 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 __device__ __forceinline__ uint64_t phys_row(uint2 e, uint64_t S) { return (uint64_t)e.x * S + e.y; }
+// AdaGrad's step -lr g / (sqrt(x) + eps), x = accumulator + g^2, with the hardware reciprocal square root and
+// reciprocal (each within 2 ulp, far inside the fp32 tolerance of the result); x = 0 is kept away from 0 * inf
+__device__ __forceinline__ float adagrad_step(float g, float x, float lr, float eps) {
+    const float root = x > 0.f ? x * rsqrtf(x) : 0.f;
+    return __fdividef(-lr * g, root + eps);
+}
 
 constexpr unsigned kBarrierSpins = 1u << 21;     // x ~100 ns: gives up after about a fifth of a second
 

@@ -559,6 +559,159 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
                  &s_ticket, kReduceTile, tmin<uint32_t>(kGroupTiles / 8, gridDim.x - group * (kGroupTiles / 8)));
 }
 
+// ------------------------------------------------- ComplEx: AdaGrad inside the reduction ----
+// The reduction of a ComplEx step whose update rows are GRADIENTS (2 d values per occurrence, Re then Im,
+// written by kge_step_kernel<.., kGradOnly>), not finished steps.  AdaGrad is taken per data point from the
+// accumulators as they were before the batch (Appendix A of the paper stores them in the PS, next to the
+// embedding): an occurrence with gradient g adds (-lr g / (sqrt(G + g^2) + eps), g^2) to its key's row
+// [Re | Im | G_Re | G_Im].  So where a part of a segment begins the warp fetches the key's row and keeps embedding
+// and accumulators in registers; every position then needs only its gradient row, half the bytes of a finished
+// update row, and the step kernel neither loads accumulators nor evaluates square roots.  The sums, the
+// parked partials of parts that cross tile borders (laid out like the row: steps, then squared gradients) and
+// the fix-up launch are those of push_reduce_kernel; the arithmetic per occurrence is the same fp32 expression
+// the step kernel used, so results do not change.  kC: float4 of a gradient row per lane (d <= 64 kC).
+template <int kC>
+__global__ void __launch_bounds__(256)
+kge_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
+                  const float4* __restrict__ grad, float4* __restrict__ store, const uint2* __restrict__ table,
+                  uint64_t S, uint32_t K, uint32_t G4, float lr, float eps, double* __restrict__ carry,
+                  uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
+                  unsigned int* __restrict__ group_done, double* __restrict__ group_sum, DevStatus* st,
+                  unsigned int epoch) {
+    __shared__ unsigned int s_ticket;
+    __shared__ __align__(8) uint64_t bars[8][2];
+    extern __shared__ float4 stage_mem[];
+    if (call_failed(st, epoch)) return;
+    constexpr int kST = 2;
+    constexpr int kSlotF4 = 3 * kC * 32;            // one position: gradient row, then the key's whole row
+    const uint32_t L4 = 2 * G4;                     // float4 of a row: embedding (G4), accumulators (G4)
+    const uint32_t L = L4 * 4;
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const uint32_t tile = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t base = (uint64_t)tile * kReduceTile;
+    const uint32_t n_valid = base < n ? (uint32_t)tmin<uint64_t>((uint64_t)kReduceTile, n - base) : 0u;
+    const uint32_t key = lane < n_valid ? sk[base + lane] : kSentinelPad;
+    const uint32_t occ = lane < n_valid ? sv[base + lane] : 0u;
+    const bool usable = key < K;
+    uint64_t row = 0;
+    if (usable) row = phys_row(table[key], S);
+    uint32_t prev = __shfl_up_sync(full, key, 1);
+    if (lane == 0) prev = (base > 0 && base - 1 < n) ? sk[base - 1] : kSentinelPad;
+    const uint32_t next_after = (base + kReduceTile < n) ? sk[base + kReduceTile] : kSentinelPad;
+    uint32_t next = __shfl_down_sync(full, key, 1);
+    if (lane == 31) next = next_after;
+    const unsigned head_mask = __ballot_sync(full, key != prev);
+    const unsigned usable_mask = __ballot_sync(full, usable);
+    const unsigned end_mask = __ballot_sync(full, usable && (key != next || lane == 31));
+    const int first_head = head_mask ? (__ffs(head_mask) - 1) : 32;
+    const uint32_t key31 = __shfl_sync(full, key, 31);
+    const bool runs_on = key31 < K && next_after == key31;
+    if (runs_on && head_mask != 0u && lane == 31)
+        starters[atomicAdd(starter_count, 1u)] = make_uint4(tile, key, (uint32_t)row, (uint32_t)(row >> 32));
+    const bool begin_me = usable && (lane == 0 || key != prev);     // the key's row is fetched here
+    const unsigned begin_mask = __ballot_sync(full, begin_me);
+    const uint32_t group = blockIdx.x / (kGroupTiles / 8);
+    const uint64_t gpos = (uint64_t)group * kGroupTiles * kReduceTile;
+    uint32_t kg = kSentinelPad, kg_prev = kSentinelPad - 1, kg_far = kSentinelPad - 2;
+    if (gpos > 0 && gpos + kGroupMinSpan - 1 < n) {
+        kg = sk[gpos];
+        kg_prev = sk[gpos - 1];
+        kg_far = sk[gpos + kGroupMinSpan - 1];
+    }
+    float4* my_stage = stage_mem + (size_t)w * (kST * kSlotF4);
+    if (lane < kST) mbar_init(&bars[w][lane], 1);
+    mbar_init_fence();
+    __syncwarp();
+    const uint32_t grad_bytes = G4 * 16u, row_bytes = L4 * 16u;
+    auto issue = [&](int p, int stage) {
+        if (p >= (int)n_valid || !((usable_mask >> p) & 1u)) return;
+        const bool b = (begin_mask >> p) & 1u;
+        if (lane == p) {
+            mbar_expect_tx(&bars[w][stage], grad_bytes + (b ? row_bytes : 0u));
+            float4* dst = my_stage + (size_t)stage * kSlotF4;
+            bulk_g2s(dst, grad + (uint64_t)occ * G4, grad_bytes, &bars[w][stage]);
+            if (b) bulk_g2s(dst + kC * 32, store + row * L4, row_bytes, &bars[w][stage]);
+        }
+    };
+    issue(0, 0);
+    d4 acc_t[kC], acc_g[kC];
+    float4 th[kC], Gv[kC];
+#pragma unroll
+    for (int c = 0; c < kC; ++c) {
+        acc_t[c] = acc_g[c] = d4{0.0, 0.0, 0.0, 0.0};
+        th[c] = Gv[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    uint32_t uses = 0;
+    for (int p = 0; p < (int)n_valid; ++p) {
+        const int stg = p & 1;
+        __syncwarp();                               // every lane is done reading the stage to be refilled
+        issue(p + 1, stg ^ 1);
+        if (!((usable_mask >> p) & 1u)) continue;
+        const uint32_t parity = (uses >> stg) & 1u;
+        if (!mbar_wait(&bars[w][stg], parity) && !mbar_wait(&bars[w][stg], parity)) {
+            if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
+            break;                                  // a copy that does not arrive: give the call up
+        }
+        uses ^= 1u << stg;
+        const float4* slot = my_stage + (size_t)stg * kSlotF4;
+        if ((begin_mask >> p) & 1u) {
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                const uint32_t f = lane + 32 * c;
+                if (f < G4) {
+                    th[c] = slot[kC * 32 + f];
+                    Gv[c] = slot[kC * 32 + G4 + f];
+                }
+                acc_t[c] = acc_g[c] = d4{0.0, 0.0, 0.0, 0.0};
+            }
+        }
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            const uint32_t f = lane + 32 * c;
+            if (f >= G4) continue;
+            const float4 g = slot[f];
+            const float qx = g.x * g.x, qy = g.y * g.y, qz = g.z * g.z, qw = g.w * g.w;
+            acc_t[c].x += (double)adagrad_step(g.x, Gv[c].x + qx, lr, eps);
+            acc_t[c].y += (double)adagrad_step(g.y, Gv[c].y + qy, lr, eps);
+            acc_t[c].z += (double)adagrad_step(g.z, Gv[c].z + qz, lr, eps);
+            acc_t[c].w += (double)adagrad_step(g.w, Gv[c].w + qw, lr, eps);
+            acc_g[c].x += (double)qx; acc_g[c].y += (double)qy; acc_g[c].z += (double)qz; acc_g[c].w += (double)qw;
+        }
+        if (!((end_mask >> p) & 1u)) continue;
+        const uint64_t rw = __shfl_sync(full, row, p);
+        const bool from_prev = p < first_head;
+        const bool parked = from_prev || (p == 31 && runs_on);
+#pragma unroll
+        for (int c = 0; c < kC; ++c) {
+            const uint32_t f = lane + 32 * c;
+            if (f >= G4) continue;
+            if (!parked) {
+                float4 t = th[c], a = Gv[c];
+                t.x = (float)((double)t.x + acc_t[c].x); t.y = (float)((double)t.y + acc_t[c].y);
+                t.z = (float)((double)t.z + acc_t[c].z); t.w = (float)((double)t.w + acc_t[c].w);
+                a.x = (float)((double)a.x + acc_g[c].x); a.y = (float)((double)a.y + acc_g[c].y);
+                a.z = (float)((double)a.z + acc_g[c].z); a.w = (float)((double)a.w + acc_g[c].w);
+                store[rw * L4 + f] = t;
+                store[rw * L4 + G4 + f] = a;
+            } else {
+                double* cs = carry + ((uint64_t)tile * 2 + (from_prev ? 0 : 1)) * L;
+                double* ct = cs + (uint64_t)f * 4;
+                double* cg = cs + (uint64_t)(G4 + f) * 4;
+                *(double2*)ct = make_double2(acc_t[c].x, acc_t[c].y);
+                *(double2*)(ct + 2) = make_double2(acc_t[c].z, acc_t[c].w);
+                *(double2*)cg = make_double2(acc_g[c].x, acc_g[c].y);
+                *(double2*)(cg + 2) = make_double2(acc_g[c].z, acc_g[c].w);
+            }
+        }
+    }
+    __syncwarp();
+    if (!(kg < K && kg_prev == kg && kg_far == kg)) return;     // nothing to pre-add for this group
+    __syncthreads();                                // the staging memory serves as scratch from here on
+    group_preadd(sk, n, L4, carry, group_done, group_sum, group, gpos, kg, reinterpret_cast<d4 (*)[32]>(stage_mem),
+                 &s_ticket, kReduceTile, tmin<uint32_t>(kGroupTiles / 8, gridDim.x - group * (kGroupTiles / 8)));
+}
+
 // ------------------------------------------------- MF: gradient inside the reduction ----
 // One minibatch of matrix factorization without update rows.  The occurrences (2t: row factor of cell t,
 // 2t + 1: its column factor) arrive sorted by key, as for a push, each with a record {cell, value of the
@@ -1171,6 +1324,35 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
     }
 #undef REDUCE_LAUNCH
 #undef REDUCE_ARGS
+    launch_fixup(ps, sk, n, d_loss_accum, loss_blocks, false, kReduceTile, 0, s);
+}
+
+void run_kge_reduce(ps_store* ps, uint32_t n, int which, uint32_t dim, float lr, float eps, double* d_loss_accum,
+                    uint32_t loss_blocks, cudaStream_t s) {
+    const uint32_t* sk = which ? ps->keysB : ps->keysA;
+    const uint32_t* sv = which ? ps->valsB : ps->valsA;
+    const uint32_t blocks = div_up_u32(div_up_u32(n, kReduceTile), 8);
+    const uint32_t G4 = dim / 2;                     // float4 of a gradient row (2 dim values)
+#define KR_ARGS sk, sv, n, (const float4*)ps->upd, (float4*)ps->store, ps->table, ps->cfg.slots_per_part,            \
+                (uint32_t)ps->cfg.num_keys, G4, lr, eps, ps->carry, ps->starters, ps->starter_count, ps->group_done, \
+                ps->group_sum, ps->status, ps->epoch
+#define KR_LAUNCH(kC)                                                                                                \
+    do {                                                                                                             \
+        static bool smem_set = false;                                                                                \
+        const size_t smem = (size_t)8 * 2 * 3 * kC * 32 * sizeof(float4);                                            \
+        if (!smem_set) {                                                                                             \
+            cudaFuncSetAttribute(kge_reduce_kernel<kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
+            smem_set = true;                                                                                         \
+        }                                                                                                            \
+        if (ps->prof) prof_before(ps, "kge_reduce_kernel<" #kC ">", s);                                              \
+        kge_reduce_kernel<kC><<<blocks, 256, smem, s>>>(KR_ARGS);                                                    \
+        if (ps->prof) prof_after(ps, s);                                                                             \
+        ps->launches++;                                                                                              \
+    } while (0)
+    if (G4 <= 32) KR_LAUNCH(1);
+    else KR_LAUNCH(2);
+#undef KR_LAUNCH
+#undef KR_ARGS
     launch_fixup(ps, sk, n, d_loss_accum, loss_blocks, false, kReduceTile, 0, s);
 }
 

@@ -223,7 +223,10 @@ uint32_t launch_step_mf(ps_store* ps, const uint32_t* d_i, const uint32_t* d_j, 
 // kDim / kExactNeg: the complex dimension and "n_neg equals kMaxNeg" known at compile time (0 / false: taken from
 // the arguments).  With both fixed the offsets of the four quarters of a row become immediates and the tests on
 // the number of negatives fold away; the kernel spends more issue slots on integer bookkeeping than on fp64.
-template <int kMaxNeg, int kDim, bool kExactNeg>
+// kGradOnly: the update row of a slot is the GRADIENT of the data point's loss with respect to the slot's key
+// (2 d values, Re then Im), and the reduction turns it into the AdaGrad step from the accumulators it finds in the
+// target row (kge_reduce_kernel); otherwise the row is the finished pair (step, squared gradient) of 4 d values.
+template <int kMaxNeg, int kDim, bool kExactNeg, bool kGradOnly>
 __global__ void __launch_bounds__(256, kMaxNeg <= 10 ? 2 : 1)
 kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                 const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
@@ -337,18 +340,20 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
         const double wS2 = __shfl_sync(full, wS, 2), wO2 = __shfl_sync(full, wO, 2);
 
         // ---- pass B: gradients per block of 32 complex dimensions, AdaGrad, update rows ----
-        float* U = upd + (t * n_slots) * L;
+        const uint32_t LU = kGradOnly ? 2 * d : L;        // values per update row
+        float* U = upd + (t * n_slots) * LU;
         // -lr g / (sqrt(G + g^2) + eps) with the hardware reciprocal square root and reciprocal (each within
         // 2 ulp, far inside the fp32 tolerance of the result); x = 0 is kept away from 0 * inf
-        auto adagrad_step = [&](float g, float x) {
-            const float root = x > 0.f ? x * rsqrtf(x) : 0.f;
-            return __fdividef(-lr * g, root + eps);
-        };
         auto adagrad_out = [&](float* Uu, uint32_t c, double gd_re, double gd_im, float G_re, float G_im) {
             const float g_re = (float)gd_re, g_im = (float)gd_im;
+            if (kGradOnly) {
+                Uu[c] = g_re;
+                Uu[d + c] = g_im;
+                return;
+            }
             const float g2_re = g_re * g_re, g2_im = g_im * g_im;
-            Uu[c] = adagrad_step(g_re, G_re + g2_re);
-            Uu[d + c] = adagrad_step(g_im, G_im + g2_im);
+            Uu[c] = adagrad_step(g_re, G_re + g2_re, lr, eps);
+            Uu[d + c] = adagrad_step(g_im, G_im + g2_im, lr, eps);
             Uu[2 * d + c] = g2_re;
             Uu[3 * d + c] = g2_im;
         };
@@ -359,17 +364,20 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
             // every value this block of dimensions needs, requested before the first use
             const float a_f = Srow[cl], b_f = Srow[d + cl], cr_f = Rrow[cl], ci_f = Rrow[d + cl];
             const float e_f = Orow[cl], f_f = Orow[d + cl];
-            const float GS_re = Srow[2 * d + cl], GS_im = Srow[3 * d + cl];
-            const float GR_re = Rrow[2 * d + cl], GR_im = Rrow[3 * d + cl];
-            const float GO_re = Orow[2 * d + cl], GO_im = Orow[3 * d + cl];
+            float GS_re = 0.f, GS_im = 0.f, GR_re = 0.f, GR_im = 0.f, GO_re = 0.f, GO_im = 0.f;
+            if (!kGradOnly) {
+                GS_re = Srow[2 * d + cl]; GS_im = Srow[3 * d + cl];
+                GR_re = Rrow[2 * d + cl]; GR_im = Rrow[3 * d + cl];
+                GO_re = Orow[2 * d + cl]; GO_im = Orow[3 * d + cl];
+            }
             float na_f[kMaxNeg], nb_f[kMaxNeg], GN_re[kMaxNeg], GN_im[kMaxNeg];
 #pragma unroll
             for (int q = 0; q < kMaxNeg; ++q) {
                 const bool live = q < (int)n_neg;
                 na_f[q] = live ? Nrow[q][cl] : 0.f;
                 nb_f[q] = live ? Nrow[q][d + cl] : 0.f;
-                GN_re[q] = ((nrep_mask >> q) & 1u) ? Nrow[q][2 * d + cl] : 0.f;
-                GN_im[q] = ((nrep_mask >> q) & 1u) ? Nrow[q][3 * d + cl] : 0.f;
+                GN_re[q] = (!kGradOnly && ((nrep_mask >> q) & 1u)) ? Nrow[q][2 * d + cl] : 0.f;
+                GN_im[q] = (!kGradOnly && ((nrep_mask >> q) & 1u)) ? Nrow[q][3 * d + cl] : 0.f;
             }
             const double a = a_f, b = b_f, cr = cr_f, ci = ci_f, e = e_f, f = f_f;
             // directions that do not depend on the negative
@@ -396,14 +404,14 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
             if (rep_o == 0) { gs_re += go_re; gs_im += go_im; }
             if (act) {
                 adagrad_out(U, c, gs_re, gs_im, GS_re, GS_im);
-                adagrad_out(U + L, c, gr_re, gr_im, GR_re, GR_im);
-                if (rep_o == 2) adagrad_out(U + 2 * (uint64_t)L, c, go_re, go_im, GO_re, GO_im);
+                adagrad_out(U + LU, c, gr_re, gr_im, GR_re, GR_im);
+                if (rep_o == 2) adagrad_out(U + 2 * (uint64_t)LU, c, go_re, go_im, GO_re, GO_im);
             }
 #pragma unroll
             for (int q = 0; q < kMaxNeg; ++q) {
                 const double wSq = __shfl_sync(full, wS, (3 + q) & 31), wOq = __shfl_sync(full, wO, (3 + q) & 31);
                 if (act && ((nrep_mask >> q) & 1u))
-                    adagrad_out(U + (uint64_t)(3 + q) * L, c, wSq * dS_re + wOq * dO_re, wSq * dS_im + wOq * dO_im,
+                    adagrad_out(U + (uint64_t)(3 + q) * LU, c, wSq * dS_re + wOq * dO_re, wSq * dS_im + wOq * dO_im,
                                 GN_re[q], GN_im[q]);
             }
         }
@@ -440,32 +448,29 @@ kge_keys_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
 
 uint32_t launch_step_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                          const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
-                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, cudaStream_t s) {
+                         uint64_t rel_key_base, uint32_t dim, float lr, float eps, bool grad_only, cudaStream_t s) {
     const uint32_t grid = step_grid(ps, n);
 #define KGE_ARGS d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, lr, eps,                     \
                  (const float*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, ps->upd,         \
                  ps->loss_partial, ps->status, ps->epoch
-    if (n_neg == 10 && dim == 100) {
-        if (ps->prof) prof_before(ps, "kge_step_kernel<10>", s);
-        kge_step_kernel<10, 100, true><<<grid, 256, 0, s>>>(KGE_ARGS);
-        if (ps->prof) prof_after(ps, s);
-        ps->launches++;
-    } else if (n_neg <= 4) {
-        if (ps->prof) prof_before(ps, "kge_step_kernel<4>", s);
-        kge_step_kernel<4, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
-        if (ps->prof) prof_after(ps, s);
-        ps->launches++;
-    } else if (n_neg <= 10) {
-        if (ps->prof) prof_before(ps, "kge_step_kernel<10>", s);
-        kge_step_kernel<10, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
-        if (ps->prof) prof_after(ps, s);
-        ps->launches++;
+#define KGE_LAUNCH(kMaxNeg, kDim, kExact, kGrad)                                                                 \
+    do {                                                                                                         \
+        if (ps->prof) prof_before(ps, "kge_step_kernel<" #kMaxNeg ">", s);                                       \
+        kge_step_kernel<kMaxNeg, kDim, kExact, kGrad><<<grid, 256, 0, s>>>(KGE_ARGS);                            \
+        if (ps->prof) prof_after(ps, s);                                                                         \
+        ps->launches++;                                                                                          \
+    } while (0)
+    if (grad_only) {
+        if (n_neg == 10 && dim == 100) KGE_LAUNCH(10, 100, true, true);
+        else if (n_neg <= 4) KGE_LAUNCH(4, 0, false, true);
+        else if (n_neg <= 10) KGE_LAUNCH(10, 0, false, true);
+        else KGE_LAUNCH(29, 0, false, true);
     } else {
-        if (ps->prof) prof_before(ps, "kge_step_kernel<29>", s);
-        kge_step_kernel<29, 0, false><<<grid, 256, 0, s>>>(KGE_ARGS);
-        if (ps->prof) prof_after(ps, s);
-        ps->launches++;
+        if (n_neg <= 4) KGE_LAUNCH(4, 0, false, false);
+        else if (n_neg <= 10) KGE_LAUNCH(10, 0, false, false);
+        else KGE_LAUNCH(29, 0, false, false);
     }
+#undef KGE_LAUNCH
 #undef KGE_ARGS
     return grid;
 }
