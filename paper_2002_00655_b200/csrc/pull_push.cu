@@ -571,7 +571,7 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
 // the fix-up launch are those of push_reduce_kernel; the arithmetic per occurrence is the same fp32 expression
 // the step kernel used, so results do not change.  kC: float4 of a gradient row per lane (d <= 64 kC).
 template <int kC>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 kge_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ sv, uint32_t n,
                   const float4* __restrict__ grad, float4* __restrict__ store, const uint2* __restrict__ table,
                   uint64_t S, uint32_t K, uint32_t G4, float lr, float eps, double* __restrict__ carry,
