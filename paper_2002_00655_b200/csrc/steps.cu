@@ -37,9 +37,12 @@ __device__ __forceinline__ void block_loss_out(double loss, double* __restrict__
     }
 }
 
-static uint32_t step_grid(ps_store* ps, uint64_t n_examples) {
+// blocks_per_sm: how many blocks of the kernel an SM holds.  With exactly the resident number of blocks every warp
+// loops over its share of the examples, and the shares differ by at most one example; with more blocks than fit, the
+// last wave is partly empty.
+static uint32_t step_grid(ps_store* ps, uint64_t n_examples, uint32_t blocks_per_sm = 8) {
     uint64_t g = (n_examples + 7) / 8;
-    const uint64_t cap = (uint64_t)ps->sm_count * 8;
+    const uint64_t cap = (uint64_t)ps->sm_count * blocks_per_sm;
     if (g > cap) g = cap;
     if (g > kMaxLossBlocks) g = kMaxLossBlocks;
     return g ? (uint32_t)g : 1u;
@@ -679,7 +682,7 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
                           uint64_t n_centers, uint64_t corpus_len, uint32_t window, const uint32_t* d_negs,
                           uint32_t n_neg, uint64_t out_key_base, float lr, cudaStream_t s) {
     const uint32_t L4 = ps->cfg.row_len / 4;
-    const uint32_t grid = step_grid(ps, n_centers);
+    const uint32_t grid = step_grid(ps, n_centers, 2);      // the kernels are bounded to two blocks per SM
 #define SG_ARGS d_tokens, tok_first, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, lr,   \
                 (const float4*)ps->store, ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, L4,              \
                 (float4*)ps->upd, sgns_scales(ps, n_centers), ps->loss_partial, ps->status, ps->epoch
