@@ -14,7 +14,8 @@ def f_row(keys, L):
 
 
 @pytest.mark.parametrize("K,L,N,n", [(5000, 100, 1, 4099), (3001, 128, 7, 10007), (640, 8, 3, 33), (900, 300, 2, 1),
-                                      (2000, 400, 5, 2500), (700, 516, 1, 777)])
+                                      (2000, 400, 5, 2500), (700, 516, 1, 777), (300, 1028, 2, 500),
+                                      (40, 16000, 2, 100)])     # the last: a ComplEx-4000 row (Table 3: 8000 values + AdaGrad)
 def test_pull_is_bit_exact(K, L, N, n):
     g, o = make_pair(K, L, N, rows=f_row(np.arange(K), L))
     keys = np.random.default_rng(n).integers(0, K, size=n)
@@ -26,7 +27,7 @@ def test_pull_is_bit_exact(K, L, N, n):
     assert g.pull(dev(np.zeros(0, np.int64))).shape == (0, L)
 
 
-@pytest.mark.parametrize("L", [4, 100, 128, 300])
+@pytest.mark.parametrize("L", [4, 100, 128, 300, 1028])
 def test_push_integer_updates_are_exact_and_order_free(L):
     K, n = 3000, 20011
     g, o = make_pair(K, L, 4, rows=f_row(np.arange(K), L), max_batch_keys=n)
@@ -47,7 +48,8 @@ def test_push_integer_updates_are_exact_and_order_free(L):
 
 
 @pytest.mark.parametrize("K,L,n,hot", [(4000, 100, 9001, 0.2), (1000, 128, 65, 0.0), (50000, 128, 60000, 0.1),
-                                         (300, 400, 4000, 0.5), (64, 8, 31, 0.9), (64, 8, 32, 1.0)])
+                                         (300, 400, 4000, 0.5), (64, 8, 31, 0.9), (64, 8, 32, 1.0),
+                                         (60, 16000, 300, 0.3)])
 def test_push_matches_oracle(K, L, n, hot):
     g, o = make_pair(K, L, 3, max_batch_keys=n)
     rng = np.random.default_rng(n)
@@ -82,7 +84,8 @@ def test_push_and_pull_reject_bad_keys_without_touching_the_store():
 
 
 @pytest.mark.parametrize("K,L,N,slack,n,seed", [(5000, 16, 4, 1.5, 700, 0), (20000, 128, 8, 1.25, 6000, 1),
-                                                 (1000, 4, 64, 2.0, 300, 2), (3000, 100, 3, 1.3, 2048, 3)])
+                                                 (1000, 4, 64, 2.0, 300, 2), (3000, 100, 3, 1.3, 2048, 3),
+                                                 (120, 16000, 3, 1.5, 90, 4)])
 def test_localize_sequences_are_bit_exact(K, L, N, slack, n, seed):
     S = int(np.ceil(slack * -(-K // N)))
     g, o = make_pair(K, L, N, S, max_batch_keys=n)

@@ -123,7 +123,7 @@ def test_kge_free_running():
 
 # (33 and 130: an odd dimension and one above 128 take the path with finished update rows, the others gradient rows)
 @pytest.mark.parametrize("dim,n_neg,batch,ents", [(100, 10, 700, 5000), (32, 1, 333, 40), (36, 29, 64, 9), (4, 0, 100, 30),
-                                                  (33, 3, 200, 50), (130, 2, 90, 25)])
+                                                  (33, 3, 200, 50), (130, 2, 90, 25), (4000, 2, 24, 20)])
 def test_kge_shapes_and_heavy_key_collisions(dim, n_neg, batch, ents):
     cfg = W.scaled(W.KGE_TINY, entities=ents, relations=5, dim=dim, n_neg=n_neg, batch=batch, n_triples=3 * batch - 11)
     kge_run(cfg, cfg.n_batches, single_step=True)
