@@ -1,0 +1,256 @@
+"""GPU parity at the full sizes of the four timed workloads, in the launch configuration that is timed
+(pipelined steps, one logical worker for the three training tasks, 64 workers for the primitives loop).
+
+The three training stores fit the host, so the oracle holds all of their rows: three steps run back to
+back on both sides without re-synchronising, every row a batch touched is compared, a sample of the
+other rows must be bit-identical to the initial values, and then the ragged last batch of the epoch runs
+as a single step.  The 51 GB store of the primitives loop does not fit an oracle on the host; there the
+location table and the free-slot stacks (which do not depend on what the rows hold) are compared bit by
+bit against an oracle store with the same keys and narrow rows, and the rows of a sample of keys (the hot
+head of the Zipf distribution and ranges further out) are compared against an oracle store that holds
+just those keys and is given the batch's occurrences of them in call order.
+"""
+import numpy as np
+import psutil
+import pytest
+import torch
+
+import paper_2002_00655_b200 as ps
+from oracle import OracleStore
+from synth import workloads as W
+from tests.util import assert_close, close, dev
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def need(host_gb, dev_gb):
+    if psutil.virtual_memory().available < host_gb * 2**30:
+        pytest.skip(f"needs {host_gb} GB of free host memory for the oracle")
+    if torch.cuda.mem_get_info()[0] < dev_gb * 2**30:
+        pytest.skip(f"needs {dev_gb} GB of free device memory")
+
+
+def fill_both(g, o, gen, K, chunk=1 << 20):
+    for s in range(0, K, chunk):
+        c = min(chunk, K - s)
+        rows = gen(s, c)
+        g.set_rows(torch.arange(s, s + c, dtype=torch.int64, device=DEV), rows)
+        o.set_rows(np.arange(s, s + c), rows.cpu().numpy())
+    torch.cuda.synchronize()
+
+
+CHUNK = 1 << 16                             # keys per pull or set call: within every store's batch limit
+
+
+def pull_host(g, keys):
+    out = np.empty((len(keys), g.L), dtype=np.float32)
+    for s in range(0, len(keys), CHUNK):
+        out[s:s + CHUNK] = g.pull(dev(keys[s:s + CHUNK])).cpu().numpy()
+    g.sync()
+    return out
+
+
+def check_rows(g, o, keys, what, loose=False):
+    """Rows of `keys` on the GPU against the oracle's."""
+    keys = np.unique(np.asarray(keys, dtype=np.int64))
+    got = pull_host(g, keys)
+    want = o.rows[keys]
+    if not loose:
+        assert_close(got, want, what)
+    else:
+        # Several AdaGrad steps in a row.  The first step on a component with accumulator 0 is -lr g / (|g| + eps):
+        # where g is within rounding of zero the two sides may step by lr in opposite directions, so a few values
+        # in ten thousand leave the single-step tolerance; none may differ by more than such a pair of steps.
+        ok = close(got, want)
+        assert (~ok).mean() <= 1e-4, (what, int((~ok).sum()))
+        assert np.abs(got.astype(np.float64) - want).max() <= 0.2, what
+    return keys
+
+
+def check_untouched(g, o, touched, K, what, n=20000):
+    rest = np.setdiff1d(np.random.default_rng(5).integers(0, K, size=n), touched)
+    assert (pull_host(g, rest) == o.rows[rest]).all(), f"{what}: a row no batch touched has changed"
+
+
+def resync(g, o, keys):
+    for s in range(0, len(keys), CHUNK):
+        part = keys[s:s + CHUNK]
+        g.set_rows(dev(part), torch.from_numpy(o.rows[part]).cuda())
+    g.loss.zero_()
+    o.loss[0] = 0
+
+
+def loss_of(g):
+    return float(g.loss.cpu()[0])
+
+
+def test_mf_large_steps():
+    c = W.MF_LARGE
+    need(12, 12)
+    g = ps.Store(c.num_keys, c.rank, 1, max_batch_keys=2 * c.batch)
+    o = OracleStore(c.num_keys, c.rank, 1)
+    fill_both(g, o, lambda s, n: W.mf_init_rows(c, s, n, DEV), c.num_keys)
+    ps.ps_set_pipelining(g.h, True)
+    planted = W.mf_planted(c, DEV)
+    i, j, v = W.mf_cells(c, planted, 0, 3 * c.batch, DEV)
+    last, n_last = c.batch_range(c.n_batches - 1)
+    li, lj, lv = W.mf_cells(c, planted, last, n_last, DEV)
+    del planted
+    for b in range(3):
+        sl = slice(b * c.batch, (b + 1) * c.batch)
+        ps.ps_step_mf(g.h, i[sl], j[sl], v[sl], c.col_key_base, c.lr, c.lam, g.loss)
+    hi, hj, hv = i.cpu().numpy(), j.cpu().numpy(), v.cpu().numpy()
+    for b in range(3):
+        sl = slice(b * c.batch, (b + 1) * c.batch)
+        o.step_mf(hi[sl], hj[sl], hv[sl], c.col_key_base, c.lr, c.lam)
+    g.sync()
+    touched = check_rows(g, o, np.concatenate([hi, hj.astype(np.int64) + c.col_key_base]), "mf_large, three steps")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    check_untouched(g, o, touched, c.num_keys, "mf_large")
+    resync(g, o, touched)
+    assert 0 < n_last < c.batch
+    ps.ps_step_mf(g.h, li, lj, lv, c.col_key_base, c.lr, c.lam, g.loss)
+    hi, hj, hv = li.cpu().numpy(), lj.cpu().numpy(), lv.cpu().numpy()
+    o.step_mf(hi, hj, hv, c.col_key_base, c.lr, c.lam)
+    g.sync()
+    check_rows(g, o, np.concatenate([hi, hj.astype(np.int64) + c.col_key_base]), "mf_large, last batch")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
+def test_kge_steps():
+    c = W.KGE
+    need(4, 12)
+    g = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(3 + c.n_neg) * c.batch)
+    o = OracleStore(c.num_keys, c.row_len, 1)
+    fill_both(g, o, lambda s, n: W.kge_init_rows(c, s, n, DEV), c.num_keys, chunk=1 << 18)
+    ps.ps_set_pipelining(g.h, True)
+
+    def run(first, n, steps):
+        d = W.kge_triples(c, first, n, DEV)
+        h = [t.cpu().numpy() for t in d]
+        for b in range(steps):
+            sl = slice(b * c.batch, min((b + 1) * c.batch, n))
+            ps.ps_step_kge(g.h, *(t[sl] for t in d), c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps, g.loss)
+        for b in range(steps):
+            sl = slice(b * c.batch, min((b + 1) * c.batch, n))
+            o.step_kge(*(t[sl] for t in h), c.rel_key_base, c.dim, c.lr, c.eps)
+        g.sync()
+        s, r, t, neg, _ = h
+        return np.concatenate([s, t, neg.ravel(), r.astype(np.int64) + c.rel_key_base])
+
+    for b in range(2):                                      # single steps (the second one with accumulators > 0)
+        touched = check_rows(g, o, run(b * c.batch, c.batch, 1), f"kge, step {b}")
+        assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+        resync(g, o, touched)
+    # three steps back to back, the sort of one beside the reduction of the one before
+    touched = check_rows(g, o, run(2 * c.batch, 3 * c.batch, 3), "kge, three steps in a row", loose=True)
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    check_untouched(g, o, touched, c.num_keys, "kge")
+    resync(g, o, touched)
+    last, n_last = c.batch_range(c.n_batches - 1)
+    assert 0 < n_last < c.batch
+    check_rows(g, o, run(last, n_last, 1), "kge, last batch")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
+def test_sgns_steps():
+    c = W.SGNS
+    need(8, 16)
+    occ = c.batch * (1 + 2 * c.window * (1 + c.n_neg))
+    g = ps.Store(c.num_keys, c.dim, 1, max_batch_keys=occ)
+    o = OracleStore(c.num_keys, c.dim, 1)
+    fill_both(g, o, lambda s, n: W.sgns_init_rows(c, s, n, DEV), c.num_keys, chunk=1 << 18)
+    ps.ps_set_pipelining(g.h, True)
+    tokens = W.sgns_tokens(c, 0, c.n_tokens, DEV)
+    h_tok = tokens.cpu().numpy()
+
+    def run(batches):
+        keys = []
+        negs = [W.sgns_negatives(c, *c.batch_range(b), DEV) for b in batches]
+        for b, ng in zip(batches, negs):
+            first, n = c.batch_range(b)
+            ps.ps_step_sgns(g.h, tokens, first, n, c.window, ng, c.n_neg, c.out_key_base, c.lr, g.loss)
+        for b, ng in zip(batches, negs):
+            first, n = c.batch_range(b)
+            h_ng = ng.cpu().numpy()
+            o.step_sgns(h_tok, first, n, c.window, h_ng, c.n_neg, c.out_key_base, c.lr)
+            lo, hi = max(first - c.window, 0), min(first + n + c.window, c.n_tokens)
+            keys += [h_tok[first:first + n].astype(np.int64), h_tok[lo:hi].astype(np.int64) + c.out_key_base,
+                     h_ng.astype(np.int64).ravel() + c.out_key_base]
+        g.sync()
+        return np.concatenate(keys)
+
+    touched = check_rows(g, o, run([0, 1, 2]), "sgns, three steps")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    check_untouched(g, o, touched, c.num_keys, "sgns")
+    resync(g, o, touched)
+    assert 0 < c.batch_range(c.n_batches - 1)[1] < c.batch
+    check_rows(g, o, run([c.n_batches - 1]), "sgns, last batch (the end of the token stream)")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
+def test_stress_batches():
+    c = W.STRESS
+    need(12, 80)
+    K, L, N, S = c.num_keys, c.row_len, c.workers, c.slots_per_part
+    g = ps.Store(K, L, N, S, max_batch_keys=c.batch)
+    chunk = 1 << 21
+    for s in range(0, K, chunk):
+        n = min(chunk, K - s)
+        g.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=DEV), W.stress_init_rows(c, s, n, DEV))
+    # sampled keys: the head of the Zipf distribution (hundreds of occurrences of one key in a batch) and
+    # ranges further out; their initial rows come from the generator, not from the store
+    rng = np.random.default_rng(11)
+    starts = [0] + sorted(int(x) for x in rng.integers(4096, K - 512, size=8))
+    ranges = [(0, 2048)] + [(s, 512) for s in starts[1:]]
+    sample = np.concatenate([np.arange(s, s + n) for s, n in ranges])
+    assert (np.diff(sample) > 0).all()
+    o_rows = OracleStore(len(sample), L, 1)                 # holds the sampled keys only, renumbered 0, 1, ...
+    o_rows.set_rows(np.arange(len(sample)), np.concatenate([W.stress_init_rows(c, s, n, DEV).cpu().numpy() for s, n in ranges]))
+    o_tab = OracleStore(K, 4, N, S)                         # all keys, narrow rows: location table and free stacks
+    assert (pull_host(g, sample) == o_rows.rows).all(), "initial rows"
+
+    steps = 3
+    keys = [W.stress_keys(c, k, DEV) for k in range(steps)]
+    upd = [W.stress_updates(c, k, DEV) for k in range(steps)]
+    outs = [torch.empty((c.batch, L), dtype=torch.float32, device=DEV) for _ in range(steps)]
+    for k in range(steps):                                  # the timed loop: no synchronisation in between
+        ps.ps_pull(g.h, keys[k], outs[k])
+        ps.ps_push(g.h, keys[k], upd[k])
+        ps.ps_localize(g.h, c.requester(k), keys[k][:c.localize_count])
+    g.sync()
+
+    for k in range(steps):
+        hk = keys[k].cpu().numpy()
+        pos = np.flatnonzero(np.isin(hk, sample))           # occurrences of sampled keys, in call order
+        ids = np.searchsorted(sample, hk[pos])
+        assert len(pos) > 10000 and np.bincount(ids).max() > 200
+        d_pos = dev(pos)
+        pulled = outs[k][d_pos].cpu().numpy()
+        want = o_rows.pull(ids)
+        if k == 0:
+            assert (pulled == want).all(), "pull of batch 0"
+        else:
+            assert_close(pulled, want, f"pull of batch {k}")
+        o_rows.push(ids, upd[k][d_pos].cpu().numpy())
+        o_tab.localize(c.requester(k), hk[:c.localize_count])
+    assert_close(pull_host(g, sample), o_rows.rows, "rows of the sampled keys after three batches")
+
+    _, owner, slot = g.export(rows=False)
+    assert (owner.numpy().view(np.uint32) == o_tab.owner).all(), "owner table"
+    assert (slot.numpy().view(np.uint32) == o_tab.slot).all(), "slot table"
+    stacks, tops = g.export_freelists()
+    assert (tops.numpy().view(np.uint64) == o_tab.top).all(), "stack heights"
+    st = stacks.numpy().view(np.uint32)
+    for p in range(N):
+        assert (st[p, :o_tab.top[p]] == o_tab.stack[p, :o_tab.top[p]]).all(), f"free stack {p}"
+    moved = int((o_tab.owner != np.arange(K, dtype=np.uint64) // c.part_size).sum())
+    assert moved > 100000 and ps.ps_rows_moved(g.h) >= moved
+    # rows that only moved keep their bits: keys of the localize calls that no push touched do not exist (every
+    # localized key was pushed to), so take untouched keys and the sampled ones through the new locations above
+    rest = np.setdiff1d(rng.integers(0, K, size=20000), np.concatenate([t.cpu().numpy() for t in keys]))
+    base = rest[:64]
+    got = pull_host(g, base)
+    for x, key in enumerate(base):
+        assert (got[x] == W.stress_init_rows(c, int(key), 1, DEV).cpu().numpy()[0]).all(), "an untouched row changed"
