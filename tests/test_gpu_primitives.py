@@ -192,3 +192,22 @@ def test_push_sizes_around_the_sort_and_reduction_tile_borders(n):
     g.sync()
     o.push(keys, upd)
     compare_state(g, o, exact_rows=True, what=f"push of {n}")
+
+
+def test_localize_at_its_largest_call_and_one_key_above():
+    """2^20 keys in one call (every 256-position chunk of the in-kernel scan in use), mostly distinct."""
+    import paper_2002_00655_b200 as ps
+    K, L, N, n = 2_500_000, 4, 2, 1 << 20
+    g, o = make_pair(K, L, N, K, rows=f_row(np.arange(K), L), max_batch_keys=n + 1)
+    rng = np.random.default_rng(21)
+    keys = rng.integers(0, K, size=n)
+    keys[:1000] = K - 1
+    g.localize(1, dev(keys))
+    g.sync()
+    o.localize(1, keys)
+    compare_state(g, o, exact_rows=True, what="localize of 2^20 keys")
+    assert ps.ps_rows_moved(g.h) > 300_000
+    with pytest.raises(ps.PSError) as e:
+        g.localize(0, dev(np.concatenate([keys, keys[:1]])))
+    assert e.value.code == ps.PS_ERR_UNSUPPORTED
+    compare_state(g, o, exact_rows=True, what="refused call")
