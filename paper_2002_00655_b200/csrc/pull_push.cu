@@ -1057,7 +1057,10 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     const uint32_t L = L4 * 4;
     const uint32_t n_tiles = (uint32_t)(((uint64_t)n + tile_len - 1) / tile_len);
     const uint32_t min_span = 8 * tile_len;                 // shortest entering segment a group pre-adds
-    const uint32_t n_warps = fix_blocks * kFixupWarps;
+    // blocks that share the list: a warp per entry in one round if there are enough blocks; the others are done
+    const uint32_t list_blocks = tmin<uint32_t>(fix_blocks, (count + kFixupWarps - 1) / kFixupWarps);
+    if (blockIdx.x >= list_blocks) return;
+    const uint32_t n_warps = list_blocks * kFixupWarps;
     // what a warp found out about its segment, for the block to share the work of a long one
     struct Walk {
         uint32_t tile, last_tile, group0, n_groups, rem_first, rem_cnt, is_long;
@@ -1114,8 +1117,11 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
             }
         }
     };
-    for (uint32_t s0 = blockIdx.x * kFixupWarps; s0 < count; s0 += n_warps) {      // same trip count for all warps
-        const uint32_t si = s0 + w;
+    // The list is roughly in position order, so the most frequent keys (neighbours in key order for Zipf inputs,
+    // each with a long walk that occupies a whole block) stand next to each other: consecutive entries go to
+    // different blocks.
+    for (uint32_t s0 = 0; s0 < count; s0 += n_warps) {      // same trip count for all warps of a block
+        const uint32_t si = s0 + w * list_blocks + blockIdx.x;
         Walk k = {0, 0, 0, 0, 0, 0, 0, 0};
         if (si < count) {
             const uint4 rec = starters[si];                 // {tile, key, row} as the reduction saw them
