@@ -194,13 +194,15 @@ class MFWorkload:
         self.hi_, self.hj_, self.hv_ = (t[lo:lo + n].cpu().pin_memory() for t in (self.i, self.j, self.v))
         self.h_lo = steps[0]
         self.h_loss = torch.zeros(len(steps), dtype=torch.float64).pin_memory()      # one word per step in flight
+        # the batches as the caller would hold them: one view per array and step, made before the timed region
+        self.h_batches = [(self.hi_[x * b:(x + 1) * b], self.hj_[x * b:(x + 1) * b], self.hv_[x * b:(x + 1) * b],
+                           self.h_loss[x:x + 1]) for x in range(len(steps))]
         return b * 12, 8
 
     def step_host(self, k):
-        c, b = self.cfg, self.cfg.batch
-        sl = slice((k - self.h_lo) * b, (k - self.h_lo + 1) * b)
-        self.ps.ps_step_mf_host(self.store.h, self.hi_[sl], self.hj_[sl], self.hv_[sl], c.col_key_base, c.lr, c.lam,
-                                self.store.loss, self.h_loss[k - self.h_lo:k - self.h_lo + 1])
+        c = self.cfg
+        hi, hj, hv, h_loss = self.h_batches[k - self.h_lo]
+        self.ps.ps_step_mf_host(self.store.h, hi, hj, hv, c.col_key_base, c.lr, c.lam, self.store.loss, h_loss)
 
     def alg_bytes(self, k):
         c, b = self.cfg, self.cfg.batch
@@ -299,14 +301,14 @@ class KGEWorkload:
         self.h = [t[lo:lo + n].cpu().contiguous().pin_memory() for t in (self.s, self.r, self.o, self.neg, self.side)]
         self.h_lo = steps[0]
         self.h_loss = torch.zeros(len(steps), dtype=torch.float64).pin_memory()
+        self.h_batches = [tuple(t[x * b:(x + 1) * b] for t in self.h) + (self.h_loss[x:x + 1],) for x in range(len(steps))]
         return b * (12 + self.cfg.n_neg * 5), 8
 
     def step_host(self, k):
-        c, b = self.cfg, self.cfg.batch
-        sl = slice((k - self.h_lo) * b, (k - self.h_lo + 1) * b)
-        s, r, o, neg, side = (t[sl] for t in self.h)
+        c = self.cfg
+        s, r, o, neg, side, h_loss = self.h_batches[k - self.h_lo]
         self.ps.ps_step_kge_host(self.store.h, s, r, o, neg, side, c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps,
-                                 self.store.loss, self.h_loss[k - self.h_lo:k - self.h_lo + 1])
+                                 self.store.loss, h_loss)
 
     def alg_bytes(self, k):
         c, sl, b = self.cfg, self._sl(k), self.cfg.batch
