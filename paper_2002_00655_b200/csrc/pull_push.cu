@@ -991,7 +991,7 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
 // The shape of every sum depends only on the sorted positions.  The last block adds the call's loss
 // partials, in index order.
 template <int kCh>
-__global__ void __launch_bounds__(32 * kFixupWarps, 2)
+__global__ void __launch_bounds__(32 * kFixupWarps, kCh == 3 ? 3 : 2)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
                   const double* __restrict__ carry, const double* __restrict__ group_sum,
