@@ -121,7 +121,17 @@ static SortSet* next_set(ps_store* ps) {
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
     ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
     ps->starters = ss->starters; ps->starter_count = ss->starter_count; ps->rec = ss->rec; ps->cellpos = ss->cellpos;
+    ps->side_idx = 0;
+    ps->side = ps->sides[0];
     return ss;
+}
+// For a call whose sort takes about as long as the rest of the step: successive calls take the two side streams in
+// turn, so that the sort of the step after next can run beside the sort of the next one (each has its own buffer set).
+static void alternate_side(ps_store* ps) {
+    static_assert(kSortSets >= 3, "two sorts in flight and one set being read");
+    ps->side_alt ^= 1;
+    ps->side_idx = ps->side_alt;
+    ps->side = ps->sides[ps->side_idx];
 }
 
 // The keys of a step's occurrences depend on the batch alone, so their extraction and sort run on the
@@ -142,10 +152,12 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_tabl
     unsigned long long id = 0;
     if (cudaStreamGetCaptureInfo(s, &cs, &id) != cudaSuccess) return false;
     if (cs != cudaStreamCaptureStatusActive) id = 0;
-    const bool crossed = id != ps->capture_id;
-    ps->capture_id = id;
-    if (crossed)
+    if (id != ps->capture_id) {
+        ps->capture_id = id;
         for (int b = 0; b < kSortSets; ++b) ps->sets[b].used = false;
+    }
+    const bool crossed = id != ps->side_capture_id[ps->side_idx];       // this side stream is still on the other side
+    ps->side_capture_id[ps->side_idx] = id;
     // a sort that reads the location table (the matrix-factorization records) must come after a call that rewrote it
     const bool ordered = crossed || (reads_table && ps->table_dirty);
     if (ordered) ps->table_dirty = false;
@@ -256,7 +268,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     // the side stream's small kernels should not queue behind the gradient kernel's waves of blocks
     int prio_lo = 0, prio_hi = 0;
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-    if (cudaStreamCreateWithPriority(&ps->side, cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+    if (cudaStreamCreateWithPriority(&ps->sides[0], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&ps->sides[1], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
@@ -289,7 +302,8 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
-    cudaStreamDestroy(ps->side);
+    cudaStreamDestroy(ps->sides[0]);
+    cudaStreamDestroy(ps->sides[1]);
     cudaStreamDestroy(ps->copy);
     for (int b = 0; b < kHostStages; ++b) {
         cudaEventDestroy(ps->ev_copied[b]);
@@ -365,6 +379,7 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (2 * n > ps->max_keys) return PS_ERR_WORKSPACE;
     if (col_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
     SortSet* ss = next_set(ps);
+    alternate_side(ps);
     if (!fork_side(ps, ss, s, true)) return PS_ERR_CUDA;
     // rows short enough to be staged whole, and row numbers that fit the 32-bit fields of the sort's records
     const bool fused = ps->cfg.row_len <= 128 && (uint64_t)ps->cfg.num_workers * ps->cfg.slots_per_part < (1ull << 32);

@@ -91,7 +91,10 @@ struct ps_store {
     uint64_t launches;
     int sm_count;
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
-    cudaStream_t side;              // key extraction and sort of a step run here, beside the gradient kernel
+    cudaStream_t side;              // key extraction and sort of the current call run here, beside the gradient kernel:
+    cudaStream_t sides[2];          // one of these two; calls whose sort is longer than the rest of the step take them
+    int side_idx, side_alt;         // in turn, so that the sorts of two later steps run beside each other
+    unsigned long long side_capture_id[2];  // graph capture each of them was last forked into (0 = none)
     cudaEvent_t ev_fork, ev_join;
     psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;

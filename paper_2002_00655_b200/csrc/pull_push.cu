@@ -762,7 +762,11 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
     const unsigned full = 0xffffffffu;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int sg = lane >> 3, l8 = lane & 7;
-    const uint32_t gb = blockIdx.x;
+    // The row side comes first in key order (one occurrence per cell: the first half of the positions) and its
+    // blocks find almost only positions that the column side handles.  The blocks are taken from the middle on, so
+    // that the column side is placed first, its most frequent keys (whose groups need a pre-added value) before
+    // the rest, and the short blocks of the row side fill in as places come free.
+    const uint32_t gb = (blockIdx.x + (n / 2) / 256) % gridDim.x;
     const uint32_t tile32 = gb * 8 + w;
     const uint64_t base = (uint64_t)tile32 * 32;
     const uint64_t pos = base + lane;
