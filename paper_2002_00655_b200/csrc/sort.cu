@@ -120,7 +120,7 @@ __device__ __forceinline__ uint32_t scan_digits(uint32_t v, uint32_t* sm8, uint3
 // A tile is kThreads x kItems keys.  Small sorts use many threads with few keys each (every phase of a pass is a
 // short chain of dependent steps, and all SMs get a tile); large sorts use 256 threads with 8 keys each.
 template <class Src, class Sink, int kThreads, int kItems>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, kThreads == 256 ? 3 : 2)
 sort_all_kernel(Src src, Sink sink, SortParams P) {
     constexpr int kTile = kThreads * kItems;
     constexpr int kWarps = kThreads / 32;
