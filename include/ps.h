@@ -234,8 +234,10 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream);
  * call time (no writes to them still pending on `stream`).
  * Results are identical in both modes.
  * The ps_step_* calls (device-batch variants) may be captured into a CUDA graph
- * on `stream`; the internal stream joins the capture at the first captured call
- * and is joined back before each call returns.  Begin a capture only when the
+ * on `stream`; an internal stream (the handle has two: ps_step_mf calls use
+ * them in turn so that the sorts of two later steps overlap) joins the capture
+ * at the first captured call that uses it and is joined back before each call
+ * returns.  Begin a capture only when the
  * handle's earlier work has completed. */
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
 
