@@ -301,3 +301,73 @@ def test_overlapped_host_batches_give_identical_results():
         s, c = cfg.batch_range(0)
         ps.ps_step_mf_host(g.h, hi[s:s + c], hj[s:s + c], hv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss, h_loss[0:1])
         assert h_loss[0] == loss_of(g)
+
+
+def test_steps_captured_into_a_graph_give_the_same_results_as_eager_calls():
+    """The timed configuration: pipelined steps captured into one CUDA graph (the internal streams join the
+    capture), replayed with one launch.  Eager calls before and after the capture use the same handle."""
+    cfg = W.scaled(W.MF_TINY, rows=3000, cols=400, rank=100, n_cells=24 * 2048, batch=2048, col_zipf=1.1, lr=0.0005)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    di, dj, dv = i.cuda(), j.cuda(), v.cuda()
+    loc_keys = dev(np.random.default_rng(2).integers(0, cfg.num_keys, size=400))
+
+    def run(g, b):
+        s, c = cfg.batch_range(b)
+        ps.ps_step_mf(g.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+        if b % 5 == 2:
+            g.localize(b % 4, loc_keys)                          # rewrites the table the next step's sort reads
+
+    eager, _ = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
+    graphed, o = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
+    for g in (eager, graphed):
+        ps.ps_set_pipelining(g.h, True)
+    for b in range(cfg.n_batches):
+        run(eager, b)
+    eager.sync()
+    for b in range(3):                                           # eager calls, then a capture, then eager calls again
+        run(graphed, b)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for b in range(3, cfg.n_batches - 2):
+            run(graphed, b)
+    graph.replay()
+    torch.cuda.synchronize()
+    for b in range(cfg.n_batches - 2, cfg.n_batches):
+        run(graphed, b)
+    graphed.sync()
+    r_e, r_g = eager.export(), graphed.export()
+    assert all((x == y).all() for x, y in zip(r_e, r_g)), "graph replay differs from eager calls"
+    assert loss_of(eager) == loss_of(graphed)
+    for b in range(cfg.n_batches):                               # and both agree with the oracle
+        s, c = cfg.batch_range(b)
+        o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+        if b % 5 == 2:
+            o.localize(b % 4, loc_keys.cpu().numpy())
+    compare_state(graphed, o, what="graph-captured MF steps")
+    assert close(loss_of(graphed), o.loss[0])
+
+    kc = W.KGE_TINY                                              # a step with a gradient kernel beside the sort
+    rows = W.kge_init_rows(kc, 0, kc.num_keys, "cpu")
+    a, _ = make_pair(kc.num_keys, kc.row_len, rows=rows, max_batch_keys=13 * kc.batch)
+    b2, _ = make_pair(kc.num_keys, kc.row_len, rows=rows, max_batch_keys=13 * kc.batch)
+    d = [t.cuda() for t in W.kge_triples(kc, 0, 6 * kc.batch, "cpu")]
+
+    def krun(g, k):
+        sl = slice(k * kc.batch, (k + 1) * kc.batch)
+        ps.ps_step_kge(g.h, *(t[sl] for t in d), kc.n_neg, kc.rel_key_base, kc.dim, kc.lr, kc.eps, g.loss)
+
+    for g in (a, b2):
+        ps.ps_set_pipelining(g.h, True)
+    for k in range(6):
+        krun(a, k)
+    a.sync()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for k in range(6):
+            krun(b2, k)
+    graph.replay()
+    b2.sync()
+    assert (a.export(table=False)[0] == b2.export(table=False)[0]).all() and loss_of(a) == loss_of(b2)
