@@ -666,6 +666,26 @@ kge_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ 
                 acc_t[c] = acc_g[c] = d4{0.0, 0.0, 0.0, 0.0};
             }
         }
+        // A segment of exactly one occurrence (most keys of a batch) needs no fp64 sum: row + update in fp32 rounds
+        // the same exact sum once, and the conversions, which share a pipe with the square roots and reciprocals
+        // that bounds this kernel, are not issued.
+        if (((begin_mask & end_mask) >> p) & 1u && p >= first_head && !(p == 31 && runs_on)) {
+            const uint64_t rw = __shfl_sync(full, row, p);
+#pragma unroll
+            for (int c = 0; c < kC; ++c) {
+                const uint32_t f = lane + 32 * c;
+                if (f >= G4) continue;
+                const float4 g = slot[f];
+                const float qx = g.x * g.x, qy = g.y * g.y, qz = g.z * g.z, qw = g.w * g.w;
+                float4 t = th[c], a = Gv[c];
+                t.x += adagrad_step(g.x, a.x + qx, lr, eps); t.y += adagrad_step(g.y, a.y + qy, lr, eps);
+                t.z += adagrad_step(g.z, a.z + qz, lr, eps); t.w += adagrad_step(g.w, a.w + qw, lr, eps);
+                a.x += qx; a.y += qy; a.z += qz; a.w += qw;
+                store[rw * L4 + f] = t;
+                store[rw * L4 + G4 + f] = a;
+            }
+            continue;
+        }
 #pragma unroll
         for (int c = 0; c < kC; ++c) {
             const uint32_t f = lane + 32 * c;
