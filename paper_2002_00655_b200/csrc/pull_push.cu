@@ -515,6 +515,26 @@ push_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__
                 const int p = g * G + k;
                 const float sc = kScaled ? __shfl_sync(full, scale, p) : 1.f;
                 if (!((usable_mask >> p) & 1u)) continue;
+                // A segment of exactly one occurrence needs no fp64 sum: row + update (one fused multiply-add if
+                // the update is a factor times a source row) rounds the exact sum once, and the conversions to
+                // and from fp64, which share a pipe with little throughput, are not issued.
+                if ((((head_mask & fetch_mask) >> p) & 1u)) {
+                    const uint64_t rw1 = __shfl_sync(full, row, p);
+#pragma unroll
+                    for (int c = 0; c < kCh; ++c) {
+                        if (fl + 32 * c >= L4) continue;
+                        const float4 u = slot[(k * 2 * kCh + c) * 32];
+                        float4 v = slot[(k * 2 * kCh + kCh + c) * 32];
+                        if (kScaled) {
+                            v.x = fmaf(sc, u.x, v.x); v.y = fmaf(sc, u.y, v.y);
+                            v.z = fmaf(sc, u.z, v.z); v.w = fmaf(sc, u.w, v.w);
+                        } else {
+                            v.x += u.x; v.y += u.y; v.z += u.z; v.w += u.w;
+                        }
+                        store[rw1 * L4 + fl + 32 * c] = v;
+                    }
+                    continue;
+                }
                 const double d = (double)sc;
 #pragma unroll
                 for (int c = 0; c < kCh; ++c) {
