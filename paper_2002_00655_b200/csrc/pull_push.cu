@@ -1035,7 +1035,7 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
 // The shape of every sum depends only on the sorted positions.  The last block adds the call's loss
 // partials, in index order.
 template <int kCh>
-__global__ void __launch_bounds__(32 * kFixupWarps, kCh == 3 ? 3 : 2)
+__global__ void __launch_bounds__(32 * kFixupWarps, (kCh == 3 || kCh == 1) ? 3 : 2)
 push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restrict__ store,
                   const uint2* __restrict__ table, uint64_t S, uint32_t K, uint32_t L4,
                   const double* __restrict__ carry, const double* __restrict__ group_sum,
@@ -1133,7 +1133,7 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     };
     // Adds partials number i0, i0 + stride, ... (below n_parts) to a[], in that order; kB of them are requested
     // together before the first is added, so a walk costs one round trip per kB partials.
-    constexpr int kB = kCh == 1 ? 8 : (kCh == 2 ? 4 : 2);
+    constexpr int kB = kCh == 1 ? 4 : (kCh == 2 ? 4 : 2);
     auto add_range = [&](d4* a, uint32_t f0, const Walk& k, uint32_t i0, uint32_t stride, uint32_t n_parts) {
         for (uint32_t i = i0; i < n_parts; i += kB * stride) {
             double2 x[kB][kCh], y[kB][kCh];
