@@ -119,7 +119,8 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
  * the top of worker's free stack; afterwards each vacated slot is pushed onto
  * its old owner's stack, ascending by key.  If worker has fewer free slots
  * than keys to move: PS_ERR_CAPACITY is latched and nothing changes.
- * At most 2^20 keys per call (PS_ERR_UNSUPPORTED beyond; split the call). */
+ * Stores of more than 1024 partitions take at most 2^20 keys per call
+ * (PS_ERR_UNSUPPORTED beyond; split the call). */
 ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n,
                         void* stream);
 

@@ -145,6 +145,241 @@ loc_apply_kernel(const uint32_t* __restrict__ so, const uint32_t* __restrict__ s
     grid_leave(bar, gridDim.x);
 }
 
+// ------------------------------------------------------------------------------------------------
+// The whole call after the key sort as ONE cooperative launch, for stores of at most kLocFastWorkers
+// partitions.  A block owns a contiguous span of the sorted positions.
+//   phase 1   count the span's first occurrences that must move                          -> grid barrier 1
+//   phase 2a  every block adds up the block counts (its own offset m0 among the moving keys, and the call's
+//             total: the capacity check, the same decision in every block); the m-th moving key takes the m-th
+//             slot from the top of the requester's stack, its old location is noted, its table entry rewritten;
+//             old owners are counted per block                                           -> arrive at barrier 2
+//   phase 2b  the block's rows travel old slot -> shared memory -> new slot as bulk asynchronous copies of
+//             whole rows, several rounds in flight per warp, while the other blocks arrive
+//   phase 3   (after barrier 2) per old owner: keys that leave it in earlier blocks = where this block's
+//             vacated slots go on that owner's stack; one warp ranks the block's keys per owner in key order
+//             (warp match, running counters in shared memory: stable) and pushes the vacated slots; the last
+//             block writes the new stack heights (every block read the old ones before barrier 2).
+// No second sort, no flag array, two grid barriers instead of four launches with four.
+constexpr uint32_t kLocFastWorkers = 1024;          // partitions the per-block owner counters have room for
+constexpr uint32_t kLocMaxGrid = 512;
+constexpr uint32_t kLocStageBytes = 4096;           // row staging per warp and stage
+constexpr int kLocStages = 3;
+constexpr size_t kLocSmem = (size_t)8 * kLocStages * kLocStageBytes;
+
+__global__ void __launch_bounds__(256, 2)
+loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uint2* table, uint32_t worker,
+                 uint32_t N, uint64_t S, uint32_t K, unsigned long long* tops, uint32_t* stacks, char* store,
+                 uint32_t row_bytes, uint32_t* block_counts, uint32_t* owner_counts, LocScratch sc,
+                 unsigned int* bar, DevStatus* st, unsigned int epoch) {
+    __shared__ uint32_t s_hist[kLocFastWorkers];    // phase 2a: keys leaving each owner from this block; phase 3: next stack position
+    __shared__ uint32_t s_top[kLocFastWorkers];     // stack heights before the call (S < 2^32)
+    __shared__ uint32_t s_part[2][256];
+    __shared__ uint32_t sm[8];
+    __shared__ int s_ok;
+    __shared__ __align__(8) uint64_t bars[8][kLocStages];
+    extern __shared__ __align__(128) char loc_stage[];
+    if (call_failed(st, epoch)) return;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const uint32_t b = blockIdx.x, G = gridDim.x;
+    const uint32_t lo = (uint32_t)tmin<uint64_t>((uint64_t)b * span, n), hi = (uint32_t)tmin<uint64_t>((uint64_t)lo + span, n);
+    // does sorted position pos hold the first occurrence of a key that must move?
+    auto must_move = [&](uint32_t pos) -> bool {
+        if (pos >= hi) return false;
+        const uint32_t key = sk[pos];
+        if (key >= K || (pos > 0 && sk[pos - 1] == key)) return false;
+        return table[key].x != worker;
+    };
+    // ---- phase 1 ----
+    uint32_t cnt = 0;
+    for (uint32_t t0 = lo; t0 < hi; t0 += 256) cnt += (uint32_t)__syncthreads_count(must_move(t0 + tid));
+    if (tid == 0) block_counts[b] = cnt;
+    if (!grid_barrier(bar, G, &s_ok)) {
+        if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
+        return;
+    }
+    // ---- phase 2a ----
+    uint32_t before = 0, all = 0;
+    for (uint32_t i = tid; i < G; i += 256) {
+        const uint32_t v = __ldcg(block_counts + i);
+        all += v;
+        if (i < b) before += v;
+    }
+    uint32_t m0, total;
+    block_exclusive_scan_256(before, sm, &m0);
+    block_exclusive_scan_256(all, sm, &total);
+    const unsigned long long top_w = tops[worker];
+    if (b == 0 && tid == 0) st->moved_total = total;
+    if ((unsigned long long)total > top_w) {                    // the same decision in every block: nothing has changed yet
+        if (b == 0 && tid == 0) latch_error(st, epoch, PS_ERR_CAPACITY);
+        grid_leave(bar, G);
+        return;
+    }
+    for (uint32_t i = tid; i < N; i += 256) {
+        s_hist[i] = 0u;
+        s_top[i] = (uint32_t)tops[i];
+    }
+    __syncthreads();
+    uint32_t running = 0;
+    for (uint32_t t0 = lo; t0 < hi; t0 += 256) {
+        const bool f = must_move(t0 + tid);
+        uint32_t tot;
+        const uint32_t ex = block_exclusive_scan_256(f ? 1u : 0u, sm, &tot);
+        if (f) {
+            const uint32_t key = sk[t0 + tid];
+            const uint32_t m = m0 + running + ex;
+            const uint2 e = table[key];
+            const uint32_t new_slot = stacks[(uint64_t)worker * S + (top_w - 1 - m)];
+            sc.mowner[m] = e.x;
+            sc.mslot[m] = e.y;
+            sc.mnew[m] = new_slot;
+            table[key] = make_uint2(worker, new_slot);
+            atomicAdd(&s_hist[e.x], 1u);
+        }
+        running += tot;
+    }
+    __syncthreads();
+    for (uint32_t i = tid; i < N; i += 256) owner_counts[(size_t)b * N + i] = s_hist[i];
+    __threadfence();
+    grid_arrive(bar);                                           // (has a __syncthreads: the block's records are complete)
+    // ---- phase 2b: the block's rows, m0 .. m0 + cnt ----
+    if (row_bytes <= kLocStageBytes) {
+        char* my = loc_stage + (size_t)w * kLocStages * kLocStageBytes;
+        if (lane < kLocStages) mbar_init(&bars[w][lane], 1);
+        mbar_init_fence();
+        __syncwarp();
+        const uint32_t per_round = tmin<uint32_t>(32u, kLocStageBytes / row_bytes);
+        const uint32_t n_rounds = (cnt + per_round - 1) / per_round;
+        uint32_t uses = 0;
+        // rounds w, w + 8, ...; the loads of up to kLocStages - 1 later rounds are in flight while one is written out
+        uint64_t dst_of[kLocStages];
+        bool mine_of[kLocStages];
+        uint32_t rows_of[kLocStages];
+        auto issue = [&](uint32_t r, int stage) {
+            mine_of[stage] = false;
+            rows_of[stage] = 0;
+            if (r >= n_rounds) return;
+            const uint32_t i = r * per_round + lane;
+            const bool mine = (uint32_t)lane < per_round && i < cnt;
+            uint64_t src = 0;
+            if (mine) {
+                const uint32_t m = m0 + i;
+                src = (uint64_t)sc.mowner[m] * S + sc.mslot[m];
+                dst_of[stage] = (uint64_t)worker * S + sc.mnew[m];
+            }
+            const uint32_t rows = tmin<uint32_t>(per_round, cnt - r * per_round);
+            mine_of[stage] = mine;
+            rows_of[stage] = rows;
+            bulk_wait_read<kLocStages - 2>();                   // the stores that last read this stage have let go of it
+            __syncwarp();
+            if (lane == 0) mbar_expect_tx(&bars[w][stage], rows * row_bytes);
+            __syncwarp();
+            if (mine) bulk_g2s(my + (size_t)stage * kLocStageBytes + (size_t)lane * row_bytes, store + src * row_bytes,
+                               row_bytes, &bars[w][stage]);
+        };
+        bool dead = false;
+        int st_fill = 0;
+        uint32_t r_next = w;
+        for (int k = 0; k < kLocStages - 1; ++k) {
+            issue(r_next, st_fill);
+            bulk_commit();                                      // keeps one bulk group per issued round (empty here)
+            r_next += 8;
+            st_fill = st_fill + 1 == kLocStages ? 0 : st_fill + 1;
+        }
+        int st_use = 0;
+        for (uint32_t r = w; r < n_rounds && !dead; r += 8) {
+            const uint32_t parity = (uses >> st_use) & 1u;
+            if (!mbar_wait(&bars[w][st_use], parity) && !mbar_wait(&bars[w][st_use], parity)) {
+                if (lane == 0) latch_error(st, epoch, PS_ERR_CUDA);
+                dead = true;
+                break;
+            }
+            uses ^= 1u << st_use;
+            fence_async_smem();
+            if (mine_of[st_use])
+                bulk_s2g(store + dst_of[st_use] * row_bytes, my + (size_t)st_use * kLocStageBytes + (size_t)lane * row_bytes,
+                         row_bytes);
+            bulk_commit();
+            st_use = st_use + 1 == kLocStages ? 0 : st_use + 1;
+            issue(r_next, st_fill);
+            r_next += 8;
+            st_fill = st_fill + 1 == kLocStages ? 0 : st_fill + 1;
+        }
+        bulk_wait_read<0>();
+    } else {
+        // rows too long for the staging: a warp per row, 128-bit loads and stores
+        const uint32_t L4 = row_bytes / 16;
+        float4* st4 = reinterpret_cast<float4*>(store);
+        for (uint32_t i = w; i < cnt; i += 8) {
+            const uint32_t m = m0 + i;
+            const uint64_t src = (uint64_t)sc.mowner[m] * S + sc.mslot[m], dst = (uint64_t)worker * S + sc.mnew[m];
+            for (uint32_t f = lane; f < L4; f += 32) st4[dst * L4 + f] = st4[src * L4 + f];
+        }
+    }
+    // ---- phase 3 ----
+    if (!grid_wait(bar, 2 * G, &s_ok)) {
+        if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
+        return;
+    }
+    {
+        // owner p's column of the per-block counts, added up by 256 / Np threads (Np = N rounded up to a power of two)
+        uint32_t Np = 1;
+        while (Np < N && Np < 256) Np <<= 1;
+        const uint32_t nq = 256 / Np, q = tid / Np;
+        for (uint32_t p0 = 0; p0 < N; p0 += Np) {
+            const uint32_t p = p0 + (tid % Np);
+            uint32_t base = 0, tot = 0;
+            if (p < N) {
+                for (uint32_t r0 = q; r0 < G; r0 += 4 * nq) {
+                    uint32_t c[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        c[k] = r0 + k * nq < G ? __ldcg(owner_counts + (size_t)(r0 + k * nq) * N + p) : 0u;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        tot += c[k];
+                        if (r0 + k * nq < b) base += c[k];
+                    }
+                }
+            }
+            s_part[0][tid] = base;
+            s_part[1][tid] = tot;
+            __syncthreads();
+            if (q == 0 && p < N) {
+                for (uint32_t i = 1; i < nq; ++i) {
+                    base += s_part[0][tid + i * Np];
+                    tot += s_part[1][tid + i * Np];
+                }
+                s_hist[p] = s_top[p] + base;
+                if (b == G - 1 && tot) tops[p] = (unsigned long long)s_top[p] + tot;    // never the requester's stack
+            }
+            __syncthreads();
+        }
+        if (b == G - 1 && tid == 0) {
+            tops[worker] = top_w - total;
+            st->rows_moved += total;
+        }
+    }
+    if (w == 0) {
+        const unsigned lt = (1u << lane) - 1u;
+        for (uint32_t i0 = 0; i0 < cnt; i0 += 32) {
+            const bool valid = i0 + lane < cnt;
+            const uint32_t m = m0 + i0 + lane;
+            const uint32_t owner = valid ? sc.mowner[m] : 0u;
+            const unsigned peers = __match_any_sync(0xffffffffu, valid ? owner : (0x80000000u + lane));
+            const int leader = __ffs(peers) - 1;
+            uint32_t old = 0;
+            if (valid && lane == leader) {
+                old = s_hist[owner];
+                s_hist[owner] = old + __popc(peers);
+            }
+            old = __shfl_sync(0xffffffffu, old, leader);
+            if (valid) stacks[(uint64_t)owner * S + old + __popc(peers & lt)] = sc.mslot[m];
+            __syncwarp();
+        }
+    }
+    grid_leave(bar, G);
+}
+
 // The call's keys (range-checked) have been sorted already; `which` says into which buffers.
 void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s) {
     LocScratch sc = loc_scratch(ps);
@@ -154,6 +389,33 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
     const uint64_t S = ps->cfg.slots_per_part;
     const uint32_t K = (uint32_t)ps->cfg.num_keys;
     const uint32_t L4 = ps->cfg.row_len / 4;
+    if (ps->cfg.num_workers <= kLocFastWorkers) {
+        static std::atomic<unsigned long long> smem_set{0};
+        opt_in_smem((const void*)loc_fused_kernel, kLocSmem, &smem_set);
+        // two blocks per SM at most (all of them resident: they meet at grid barriers), spans of whole tiles of 256
+        const uint32_t max_grid = tmin<uint32_t>((uint32_t)ps->sm_count * 2, kLocMaxGrid);
+        uint32_t span = div_up_u32(div_up_u32(n, max_grid), 256) * 256;
+        const uint32_t grid_f = div_up_u32(n, span);
+        uint2* table = ps->table;
+        unsigned long long* tops = ps->tops;
+        uint32_t* stacks = ps->stacks;
+        char* store = (char*)ps->store;
+        uint32_t row_bytes = ps->cfg.row_len * 4, N = ps->cfg.num_workers;
+        uint32_t* block_counts = ps->loc_counts;
+        uint32_t* owner_counts = ps->loc_counts + kLocMaxGrid;
+        unsigned int* bar = ps->sort_ctl + 2;                   // words 0 and 1 belong to the sort
+        DevStatus* st = ps->status;
+        unsigned int epoch = ps->epoch;
+        void* args[] = {(void*)&sk, (void*)&n, (void*)&span, (void*)&table, (void*)&worker, (void*)&N, (void*)&S, (void*)&K,
+                        (void*)&tops, (void*)&stacks, (void*)&store, (void*)&row_bytes, (void*)&block_counts,
+                        (void*)&owner_counts, (void*)&sc, (void*)&bar, (void*)&st, (void*)&epoch};
+        if (ps->prof) prof_before(ps, "loc_fused_kernel", s);
+        cudaLaunchCooperativeKernel((const void*)loc_fused_kernel, dim3(grid_f), dim3(256), args, kLocSmem, s);
+        if (ps->prof) prof_after(ps, s);
+        ps->launches++;
+        return;
+    }
+    // more partitions than the fused kernel keeps counters for: plan, sort the moving keys by old owner, apply.
     // cooperative launches (the blocks meet at a grid barrier): as many blocks as are resident at once, at most
     uint32_t grid = tmin<uint32_t>(chunks, (uint32_t)ps->sm_count * 4);
     unsigned int* bar_plan = ps->sort_ctl + 2;               // words 0 and 1 belong to the sort

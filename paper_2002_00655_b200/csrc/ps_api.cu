@@ -43,6 +43,9 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.starter_count[b] = take(4);
     }
     l.scan_sums = take(((mk + 255) / 256) * 4);
+    // localize in one launch: a count per block (at most 512 blocks), then one per block and partition (stores of
+    // at most 1024 partitions; larger ones take the path that sorts by old owner)
+    l.loc_counts = take((size_t)512 * 4 + (size_t)512 * (cfg.num_workers <= 1024 ? cfg.num_workers : 1) * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
     l.group_sum = take(groups * (size_t)cfg.row_len * 8);
@@ -115,7 +118,11 @@ static ps_status_t after_launch() { return cuda_ok(cudaGetLastError()); }
 
 
 // Calls that sort rotate through the handle's sets of sort buffers.
+static void next_epoch(ps_store* ps);
 static SortSet* next_set(ps_store* ps) {
+    // The call's number for the device-side error marks advances with the buffer sets: at most kSortSets such calls
+    // are in flight, so their numbers never collide modulo the marks' slots (calls that sort nothing take no number).
+    next_epoch(ps);
     ps->cur_set = (ps->cur_set + 1) % kSortSets;
     SortSet* ss = &ps->sets[ps->cur_set];
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
@@ -159,8 +166,9 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_tabl
     const bool crossed = id != ps->side_capture_id[ps->side_idx];       // this side stream is still on the other side
     ps->side_capture_id[ps->side_idx] = id;
     // a sort that reads the location table (the matrix-factorization records) must come after a call that rewrote it
-    const bool ordered = crossed || (reads_table && ps->table_dirty);
-    if (ordered) ps->table_dirty = false;
+    // (every side stream on its own: the one that did not fork ordered has still not seen the rewrite)
+    const bool ordered = crossed || (reads_table && ps->table_dirty[ps->side_idx]);
+    if (ordered) ps->table_dirty[ps->side_idx] = false;
     if (ps->pipelined && !ordered) return !ss->used || cudaStreamWaitEvent(ps->side, ss->ev_free, 0) == cudaSuccess;
     return cudaEventRecord(ps->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(ps->side, ps->ev_fork, 0) == cudaSuccess;
 }
@@ -242,6 +250,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     ps->cur_set = kSortSets - 1;
     next_set(ps);
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
+    ps->loc_counts = (uint32_t*)(ps->ws + l.loc_counts);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
     ps->group_sum = (double*)(ps->ws + l.group_sum);
@@ -315,13 +324,12 @@ ps_status_t ps_destroy(ps_store_t* ps) {
 
 #define PS_BEGIN_CALL(ps)                                            \
     if (!(ps)) return PS_ERR_INVALID_ARG;                           \
-    cudaStream_t s = (cudaStream_t)stream;                          \
-    next_epoch(ps);
+    cudaStream_t s = (cudaStream_t)stream;
 
 ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
     PS_BEGIN_CALL(ps);
     launch_init_range_partition(ps, s);
-    ps->table_dirty = true;
+    ps->table_dirty[0] = ps->table_dirty[1] = true;
     return after_launch();
 }
 
@@ -361,13 +369,14 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     if (n == 0) return PS_OK;
     if (!d_keys) return PS_ERR_INVALID_ARG;
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
-    if (n > (1u << 20)) return PS_ERR_UNSUPPORTED;          // one block scans the call's per-chunk counts in shared memory
+    // stores of more than 1024 partitions: one block scans the call's per-chunk counts in shared memory
+    if (n > (1u << 20) && ps->cfg.num_workers > 1024) return PS_ERR_UNSUPPORTED;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, nullptr, 0);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_localize(ps, worker, (uint32_t)n, which, s);
-    ps->table_dirty = true;
+    ps->table_dirty[0] = ps->table_dirty[1] = true;
     return release_set(ss, s);
 }
 
@@ -576,7 +585,6 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     if (tok_first > need_lo || tok_first + tok_count <= need_hi) return PS_ERR_INVALID_ARG;
     if ((tok_count + n_negs) * 4 > ps->max_keys * 8) return PS_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
-    next_epoch(ps);
     HostBatch hb;
     if (!host_batch_begin(ps, s, &hb)) return PS_ERR_CUDA;
     uint32_t* d_tok = (uint32_t*)hb.buf;

@@ -2,6 +2,7 @@
 // Nothing here is part of the public interface (see include/ps.h).
 #pragma once
 
+#include <atomic>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -27,9 +28,9 @@ constexpr int kSortSets = 3;                     // calls whose key sort may be 
 // epoch, so no kernel has to clear anything before a call starts.
 struct DevStatus {
     unsigned int sticky;            // first error code since the last ps_sync
-    unsigned int call_err_epoch[4]; // epoch of the last call with that epoch mod 4 that failed on the device (up
-                                    // to kSortSets calls of one handle are in flight: later ones' sorts beside
-                                    // the current one's kernels)
+    unsigned int call_err_epoch[4]; // number of the last sorting call with that number mod 4 that failed on the device
+                                    // (up to kSortSets such calls of one handle are in flight: later ones' sorts
+                                    // beside the current one's kernels; only calls that take a buffer set are numbered)
     unsigned int moved_total;       // localize: number of keys that move in the current call
     unsigned long long rows_moved;  // rows relocated by all successful localize calls so far
 };
@@ -78,6 +79,7 @@ struct ps_store {
     unsigned int* group_done;       // per group of 64 reduction tiles: reduction blocks that have finished
     double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
+    uint32_t* loc_counts;           // localize: moving keys per block (512 words), then per block and old owner
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
     uint4* starters;                // {tile, key, row} of the tiles that start a border-crossing segment
@@ -105,7 +107,8 @@ struct ps_store {
     bool host_overlap;
     cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
-    bool table_dirty;               // the location table was rewritten since the side stream last waited for the caller's
+    bool table_dirty[2];            // per side stream: the location table was rewritten since that stream last waited
+                                    // for the caller's (a sort that reads the table must not start before the rewrite)
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
 };
 
@@ -113,12 +116,22 @@ namespace psb {
 
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
-        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], scan_sums, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], scan_sums, loc_counts, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
         loss_partial, apply_rows, staging[kHostStages], total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
 
 inline uint32_t div_up_u32(uint64_t a, uint64_t b) { return (uint32_t)((a + b - 1) / b); }
+
+// The opt-in to more than 48 KB of dynamic shared memory is a per-DEVICE attribute of a kernel: `done` keeps one
+// bit per device ordinal (a static of the launch site), so every GPU the process uses gets the attribute once.
+inline void opt_in_smem(const void* fn, size_t bytes, std::atomic<unsigned long long>* done) {
+    int d = -1;
+    const bool known = cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64;
+    if (known && ((done->load(std::memory_order_relaxed) >> d) & 1ull)) return;
+    cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (known) done->fetch_or(1ull << d, std::memory_order_relaxed);
+}
 template <class T> __host__ __device__ inline T tmin(T a, T b) { return a < b ? a : b; }
 template <class T> __host__ __device__ inline T tmax(T a, T b) { return a > b ? a : b; }
 
@@ -214,9 +227,10 @@ uint32_t launch_step_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_f
 
 // ---- device helpers ----
 #ifdef __CUDACC__
+// epoch 0: a call without later kernels to cancel (pull, set rows, get location); only the sticky code is latched
 __device__ __forceinline__ void latch_error(DevStatus* st, unsigned int epoch, unsigned int code) {
     atomicCAS(&st->sticky, 0u, code);
-    atomicExch(&st->call_err_epoch[epoch & 3u], epoch);
+    if (epoch != 0u) atomicExch(&st->call_err_epoch[epoch & 3u], epoch);
 }
 __device__ __forceinline__ bool call_failed(const DevStatus* st, unsigned int epoch) {
     return *((const volatile unsigned int*)&st->call_err_epoch[epoch & 3u]) == epoch;
@@ -261,6 +275,26 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* bar, unsigned int tar
     __syncthreads();
     return *s_ok != 0;
 }
+// The same barrier in two halves, for a block that has work to do between arriving and needing the others' results:
+// everything the block wrote before grid_arrive is visible to a block that has passed grid_wait.
+__device__ __forceinline__ void grid_arrive(unsigned int* bar) {
+    __syncthreads();
+    if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;\n" ::"l"(bar) : "memory");
+}
+__device__ __forceinline__ bool grid_wait(unsigned int* bar, unsigned int target, int* s_ok) {
+    if (threadIdx.x == 0) {
+        unsigned int seen = 0, spins = 0;
+        for (;;) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(seen) : "l"(bar) : "memory");
+            if (seen >= target || spins >= kBarrierSpins) break;
+            __nanosleep(spins < 256 ? 20 : 100);
+            ++spins;
+        }
+        *s_ok = seen >= target;
+    }
+    __syncthreads();
+    return *s_ok != 0;
+}
 __device__ __forceinline__ void grid_leave(unsigned int* bar, unsigned int n_blocks) {
     if (threadIdx.x == 0 && atomicAdd(bar + 1, 1u) == n_blocks - 1) {
         // every other block has left, so nobody is waiting on the arrival count any more
@@ -268,6 +302,55 @@ __device__ __forceinline__ void grid_leave(unsigned int* bar, unsigned int n_blo
         atomicExch(bar + 1, 0u);
     }
 }
+
+// ---- bulk asynchronous copies global -> shared, reporting to a barrier word in shared memory ----
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
+// one arrival that also announces `bytes` of copies
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// 16-byte aligned source and destination, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
+                     smem_addr(smem)),
+                 "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.  Each poll
+// may stay suspended in hardware for up to kBarSuspendNs (it returns as soon as the phase completes), so that a
+// waiting warp does not spend issue slots on polling: about a quarter of a second per call at most.
+constexpr unsigned kBarPollLimit = 1u << 17;
+constexpr unsigned kBarSuspendNs = 2000;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
+    const unsigned a = smem_addr(bar);
+    for (unsigned i = 0; i < kBarPollLimit; ++i) {
+        unsigned done;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+            : "=r"(done)
+            : "r"(a), "r"(parity), "r"(kBarSuspendNs)
+            : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+// shared -> global, tracked in the issuing thread's bulk groups
+__device__ __forceinline__ void bulk_s2g(void* gmem, const void* smem, unsigned bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem), "r"(smem_addr(smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
+// until at most kPending of this thread's bulk groups still have to READ their source
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(kPending) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 
 // Exclusive scan of one value per thread over a block of 256 threads.
 // `smem` must hold 8 uint32.  Returns the exclusive prefix; *total = block sum.

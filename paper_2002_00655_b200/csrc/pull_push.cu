@@ -60,57 +60,8 @@ set_rows_kernel(const uint64_t* __restrict__ keys, uint64_t n, const float4* __r
 void launch_set_rows(ps_store* ps, const uint64_t* d_keys, uint64_t n, const float* d_vals, cudaStream_t s) {
     const uint32_t grid = (uint32_t)tmin<uint64_t>((n + 7) / 8, (uint64_t)ps->sm_count * 8);
     PS_LAUNCH(ps, set_rows_kernel, grid, 256, s, d_keys, n, (const float4*)d_vals, (float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, ps->epoch);
+              ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, 0u);
 }
-
-// ---- bulk asynchronous copies global -> shared, reporting to a barrier word in shared memory ----
-__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory"); }
-// one arrival that also announces `bytes` of copies
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-// 16-byte aligned source and destination, size a multiple of 16 bytes
-__device__ __forceinline__ void bulk_g2s(void* smem, const void* gmem, unsigned bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(
-                     smem_addr(smem)),
-                 "l"(gmem), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-// Waits for the phase of the given parity to complete; gives up (false) after a bounded number of polls.  Each poll
-// may stay suspended in hardware for up to kBarSuspendNs (it returns as soon as the phase completes), so that a
-// waiting warp does not spend issue slots on polling: about a quarter of a second per call at most.
-constexpr unsigned kBarPollLimit = 1u << 17;
-constexpr unsigned kBarSuspendNs = 2000;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
-    const unsigned a = smem_addr(bar);
-    for (unsigned i = 0; i < kBarPollLimit; ++i) {
-        unsigned done;
-        asm volatile(
-            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
-            : "=r"(done)
-            : "r"(a), "r"(parity), "r"(kBarSuspendNs)
-            : "memory");
-        if (done) return true;
-    }
-    return false;
-}
-
-// shared -> global, tracked in the issuing thread's bulk groups
-__device__ __forceinline__ void bulk_s2g(void* gmem, const void* smem, unsigned bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem), "r"(smem_addr(smem)), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
-// until at most kPending of this thread's bulk groups still have to READ their source
-template <int kPending>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;\n" ::"n"(kPending) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 
 // ---------------------------------------------------------------- pull ----
 // Rows travel store -> shared memory -> caller's buffer as bulk asynchronous copies of whole rows, without
@@ -231,21 +182,18 @@ pull_kernel(const uint64_t* __restrict__ keys, uint64_t n, float4* __restrict__ 
 void launch_pull(ps_store* ps, const uint64_t* d_keys, uint64_t n, float* d_out, cudaStream_t s) {
     const uint32_t row_bytes = ps->cfg.row_len * 4;
     if (row_bytes <= kPullStageBytes) {
-        static bool smem_set = false;
-        if (!smem_set) {
-            cudaFuncSetAttribute(pull_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPullSmem);
-            smem_set = true;
-        }
+        static std::atomic<unsigned long long> smem_set{0};
+        opt_in_smem((const void*)pull_bulk_kernel, kPullSmem, &smem_set);
         const uint32_t per_round = tmin<uint32_t>(32u, kPullStageBytes / row_bytes);
         const uint64_t rounds = (n + per_round - 1) / per_round;
         const uint32_t grid = (uint32_t)tmin<uint64_t>((rounds + 7) / 8, (uint64_t)ps->sm_count * 3);
         PS_LAUNCH_SMEM(ps, pull_bulk_kernel, grid, 256, kPullSmem, s, d_keys, n, (char*)d_out, (const char*)ps->store,
-                       ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, row_bytes, per_round, ps->status, ps->epoch);
+                       ps->table, ps->cfg.slots_per_part, ps->cfg.num_keys, row_bytes, per_round, ps->status, 0u);
         return;
     }
     const uint32_t grid = (uint32_t)tmin<uint64_t>((n + 31) / 32, (uint64_t)ps->sm_count * 8);
     PS_LAUNCH(ps, pull_kernel<4>, grid, 256, s, d_keys, n, (float4*)d_out, (const float4*)ps->store, ps->table,
-              ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, ps->epoch);
+              ps->cfg.slots_per_part, ps->cfg.num_keys, ps->cfg.row_len / 4, ps->status, 0u);
 }
 
 // rows of keys first_key .. first_key + n, in key order (export)
@@ -287,7 +235,7 @@ __global__ void get_location_kernel(const uint64_t* __restrict__ keys, uint64_t 
 void launch_get_location(ps_store* ps, const uint64_t* d_keys, uint64_t n, uint32_t* d_owner, uint32_t* d_slot,
                          cudaStream_t s) {
     PS_LAUNCH(ps, get_location_kernel, div_up_u32(n, 256), 256, s, d_keys, n, d_owner, d_slot, ps->table,
-              ps->cfg.num_keys, ps->status, ps->epoch);
+              ps->cfg.num_keys, ps->status, 0u);
 }
 
 // ---------------------------------------------------------------- push ----
@@ -1318,11 +1266,8 @@ void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_ba
         ps->group_sum, ps->loss_partial, ps->status, ps->epoch
 #define SUB_LAUNCH(kC)                                                                                               \
     do {                                                                                                             \
-        static bool smem_set = false;                                                                                \
-        if (!smem_set) {                                                                                             \
-            cudaFuncSetAttribute(mf_sub_kernel<kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMfSmem);      \
-            smem_set = true;                                                                                         \
-        }                                                                                                            \
+        static std::atomic<unsigned long long> smem_set{0};                                                          \
+        opt_in_smem((const void*)mf_sub_kernel<kC>, kMfSmem, &smem_set);                                             \
         PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, blocks, 256, kMfSmem, s, SUB_ARGS);                                    \
     } while (0)
     if (L4 <= 8) SUB_LAUNCH(1);
@@ -1346,12 +1291,8 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
                     ps->starter_count, ps->group_done, ps->group_sum, ps->status, ps->epoch
 #define REDUCE_LAUNCH(kCh, kScaled, kL4, kSlots)                                                                     \
     do {                                                                                                             \
-        static bool smem_set = false;                                                                                \
-        if (!smem_set) {                                                                                             \
-            cudaFuncSetAttribute(push_reduce_kernel<kCh, kScaled, kL4, kSlots>,                                      \
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)reduce_smem(kCh));                \
-            smem_set = true;                                                                                         \
-        }                                                                                                            \
+        static std::atomic<unsigned long long> smem_set{0};                                                          \
+        opt_in_smem((const void*)push_reduce_kernel<kCh, kScaled, kL4, kSlots>, reduce_smem(kCh), &smem_set);        \
         if (ps->prof) prof_before(ps, "push_reduce_kernel<" #kCh "," #kScaled ">", s);                               \
         push_reduce_kernel<kCh, kScaled, kL4, kSlots><<<blocks, 256, reduce_smem(kCh), s>>>(REDUCE_ARGS);            \
         if (ps->prof) prof_after(ps, s);                                                                             \
@@ -1388,12 +1329,9 @@ void run_kge_reduce(ps_store* ps, uint32_t n, int which, uint32_t dim, float lr,
                 ps->group_sum, ps->status, ps->epoch
 #define KR_LAUNCH(kC)                                                                                                \
     do {                                                                                                             \
-        static bool smem_set = false;                                                                                \
+        static std::atomic<unsigned long long> smem_set{0};                                                          \
         const size_t smem = (size_t)8 * 2 * 3 * kC * 32 * sizeof(float4);                                            \
-        if (!smem_set) {                                                                                             \
-            cudaFuncSetAttribute(kge_reduce_kernel<kC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);     \
-            smem_set = true;                                                                                         \
-        }                                                                                                            \
+        opt_in_smem((const void*)kge_reduce_kernel<kC>, smem, &smem_set);                                            \
         if (ps->prof) prof_before(ps, "kge_reduce_kernel<" #kC ">", s);                                              \
         kge_reduce_kernel<kC><<<blocks, 256, smem, s>>>(KR_ARGS);                                                    \
         if (ps->prof) prof_after(ps, s);                                                                             \

@@ -424,22 +424,16 @@ static int sort_launch(ps_store* ps, const Src& src, const Sink& sink, uint32_t 
     void* args[] = {(void*)&src, (void*)&sink, (void*)&P};
     // cooperative: the blocks wait for one another at the grid barrier, so all of them must be resident
     if (small) {
-        static bool attr_set = false;
+        static std::atomic<unsigned long long> attr_set{0};
         const void* fn = (const void*)sort_all_kernel<Src, Sink, kSmallThreads, kSmallItems>;
         const size_t smem = (size_t)2 * kSmallTile * sizeof(uint32_t);
-        if (!attr_set) {
-            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            attr_set = true;
-        }
+        opt_in_smem(fn, smem, &attr_set);
         cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kSmallThreads), args, smem, stream);
     } else {
-        static bool attr_set = false;
+        static std::atomic<unsigned long long> attr_set{0};
         const void* fn = (const void*)sort_all_kernel<Src, Sink, kSortThreads, kSortItems>;
         const size_t smem = (size_t)2 * kSortTile * sizeof(uint32_t);
-        if (!attr_set) {
-            cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            attr_set = true;
-        }
+        opt_in_smem(fn, smem, &attr_set);
         cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kSortThreads), args, smem, stream);
     }
     if (ps->prof) prof_after(ps, stream);

@@ -85,7 +85,8 @@ def test_push_and_pull_reject_bad_keys_without_touching_the_store():
 
 @pytest.mark.parametrize("K,L,N,slack,n,seed", [(5000, 16, 4, 1.5, 700, 0), (20000, 128, 8, 1.25, 6000, 1),
                                                  (1000, 4, 64, 2.0, 300, 2), (3000, 100, 3, 1.3, 2048, 3),
-                                                 (120, 16000, 3, 1.5, 90, 4)])
+                                                 (120, 16000, 3, 1.5, 90, 4), (6000, 8, 1500, 2.0, 900, 5),
+                                                 (4000, 32, 300, 2.0, 1200, 6), (500, 1024, 5, 1.5, 300, 7)])
 def test_localize_sequences_are_bit_exact(K, L, N, slack, n, seed):
     S = int(np.ceil(slack * -(-K // N)))
     g, o = make_pair(K, L, N, S, max_batch_keys=n)
@@ -194,8 +195,9 @@ def test_push_sizes_around_the_sort_and_reduction_tile_borders(n):
     compare_state(g, o, exact_rows=True, what=f"push of {n}")
 
 
-def test_localize_at_its_largest_call_and_one_key_above():
-    """2^20 keys in one call (every 256-position chunk of the in-kernel scan in use), mostly distinct."""
+def test_localize_of_a_million_keys_in_one_call():
+    """2^20 keys in one call, mostly distinct (every block of the one-launch relocation has a span of several
+    tiles), then one key more; a store of more than 1024 partitions refuses calls beyond 2^20 keys."""
     import paper_2002_00655_b200 as ps
     K, L, N, n = 2_500_000, 4, 2, 1 << 20
     g, o = make_pair(K, L, N, K, rows=f_row(np.arange(K), L), max_batch_keys=n + 1)
@@ -207,7 +209,12 @@ def test_localize_at_its_largest_call_and_one_key_above():
     o.localize(1, keys)
     compare_state(g, o, exact_rows=True, what="localize of 2^20 keys")
     assert ps.ps_rows_moved(g.h) > 300_000
+    more = np.concatenate([keys, keys[:1]])
+    g.localize(0, dev(more))
+    g.sync()
+    o.localize(0, more)
+    compare_state(g, o, exact_rows=True, what="localize of 2^20 + 1 keys")
+    wide, _ = make_pair(4000, 4, 2000, 4, max_batch_keys=n + 1)  # the path that sorts by old owner scans in shared memory
     with pytest.raises(ps.PSError) as e:
-        g.localize(0, dev(np.concatenate([keys, keys[:1]])))
+        wide.localize(0, dev(np.concatenate([keys, keys[:1]]) % 4000))
     assert e.value.code == ps.PS_ERR_UNSUPPORTED
-    compare_state(g, o, exact_rows=True, what="refused call")

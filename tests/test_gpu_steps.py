@@ -270,6 +270,47 @@ def test_mf_pipelined_steps_with_relocations_in_between():
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
 
 
+@pytest.mark.parametrize("graph", [False, True])
+def test_two_pipelined_mf_steps_right_after_a_large_localize(graph):
+    """MF steps sort on two internal streams in turn.  After a call that rewrites the location table BOTH streams
+    must wait for it before a sort that reads the table: here a localize of 100,000 keys (long enough to be still
+    running when the second step's sort could start) is followed by two steps whose cells all use moved keys."""
+    cfg = W.MFConfig("t", 120_000, 4_000, 32, 3 * 4096, 4096, 0.002, 0.05, 0.1, 0.5, 1.1)
+    rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+    i, j, v = mf_data(cfg)
+    g, o = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=1 << 17)
+    ps.ps_set_pipelining(g.h, True)
+    di, dj, dv = i.cuda(), j.cuda(), v.cuda()
+    moved = np.concatenate([np.arange(0, 96_000), cfg.col_key_base + np.arange(0, 4_000)]).astype(np.int64)
+    d_moved = dev(moved)
+
+    def steps(lo, hi):
+        for b in range(lo, hi):
+            s, c = cfg.batch_range(b)
+            ps.ps_step_mf(g.h, di[s:s + c], dj[s:s + c], dv[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+
+    steps(0, 1)                                                  # both internal streams have been used before
+    torch.cuda.synchronize()
+    if graph:
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg):
+            g.localize(3, d_moved)
+            steps(1, 3)
+        cg.replay()
+    else:
+        g.localize(3, d_moved)
+        steps(1, 3)
+    g.sync()
+    s, c = cfg.batch_range(0)
+    o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+    o.localize(3, moved)
+    for b in range(1, 3):
+        s, c = cfg.batch_range(b)
+        o.step_mf(i[s:s + c], j[s:s + c], v[s:s + c], cfg.col_key_base, cfg.lr, cfg.lam)
+    compare_state(g, o, what="two pipelined steps after a large localize")
+    assert close(loss_of(g), o.loss[0])
+
+
 def test_overlapped_host_batches_give_identical_results():
     """ps_set_host_overlap: batches are copied on the library's copy stream while earlier steps run and the
     calls do not wait; parameters and every step's loss must equal those of the device-batch calls."""
