@@ -235,7 +235,7 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream);
  * call time (no writes to them still pending on `stream`).
  * Results are identical in both modes.
  * The ps_step_* calls (device-batch variants) may be captured into a CUDA graph
- * on `stream`; an internal stream (the handle has two: ps_step_mf calls use
+ * on `stream`; an internal stream (the handle has three: ps_step_mf calls use
  * them in turn so that the sorts of two later steps overlap) joins the capture
  * at the first captured call that uses it and is joined back before each call
  * returns.  Begin a capture only when the
@@ -256,6 +256,19 @@ ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
  * copy has landed.  Results are identical in both modes.  The switch itself waits
  * for the device.  Do not capture ps_step_*_host calls into a CUDA graph. */
 ps_status_t ps_set_host_overlap(ps_store_t* ps, int on);
+
+/* Which kernels ps_step_mf uses on rows of at most 128 values (results are the same to rounding order; both
+ * sum a key's terms in fp64 in the order of the sorted occurrences and round once).
+ *   PS_MF_BY_COLUMN: one launch that visits the column-factor occurrences only; each forms its cell's terms
+ *     for both factors (the tasks of Section 4.1 draw the rows of a batch from far more rows than the batch has
+ *     cells, so a row factor nearly always has one cell).  Row keys with several cells in a batch are summed by
+ *     the last of their cells to finish; a batch in which few row keys carry most cells is served slowly.
+ *   PS_MF_SYMMETRIC: row and column occurrences are reduced alike, then a second launch finishes the
+ *     segments that cross tile borders.
+ *   PS_MF_AUTO (default): symmetric (the faster of the two on the 10M x 1M matrix of Section 4.1 as measured on
+ *     B200: 45 against 49 microseconds per step of 65,536 cells). */
+enum { PS_MF_AUTO = 0, PS_MF_BY_COLUMN = 1, PS_MF_SYMMETRIC = 2 };
+ps_status_t ps_set_mf_path(ps_store_t* ps, int path);
 
 /* Number of kernels this handle has launched so far. */
 uint64_t ps_launch_count(const ps_store_t* ps);

@@ -39,6 +39,8 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
         l.sort_ctl[b] = take(((size_t)kSortCtlWords + groups) * 4);
         l.rec[b] = take(mk * 16);
         l.cellpos[b] = take(mk * 4);
+        l.mf_dup[b] = take((mk / 2 + 1 + mk / 512 + 2) * 16);      // per column position, then per block of 256 of them
+        l.mf_tickets[b] = take((mk / 2 + 1 + mk / 512 + 4) * 4);
         l.starters[b] = take(reduce_tiles * 16);
         l.starter_count[b] = take(4);
     }
@@ -128,15 +130,16 @@ static SortSet* next_set(ps_store* ps) {
     ps->keysA = ss->keysA; ps->keysB = ss->keysB; ps->valsA = ss->valsA; ps->valsB = ss->valsB;
     ps->tile_state = ss->tile_state; ps->sort_ctl = ss->sort_ctl; ps->group_done = ss->group_done;
     ps->starters = ss->starters; ps->starter_count = ss->starter_count; ps->rec = ss->rec; ps->cellpos = ss->cellpos;
+    ps->mf_dup = ss->mf_dup; ps->mf_tickets = ss->mf_tickets;
     ps->side_idx = 0;
     ps->side = ps->sides[0];
     return ss;
 }
-// For a call whose sort takes about as long as the rest of the step: successive calls take the two side streams in
+// For a call whose sort takes about as long as the rest of the step: successive calls take the side streams in
 // turn, so that the sort of the step after next can run beside the sort of the next one (each has its own buffer set).
 static void alternate_side(ps_store* ps) {
-    static_assert(kSortSets >= 3, "two sorts in flight and one set being read");
-    ps->side_alt ^= 1;
+    static_assert(kSortSets >= kSideStreams + 1, "a sort in flight per internal stream and one set being read");
+    ps->side_alt = (ps->side_alt + 1) % kSideStreams;
     ps->side_idx = ps->side_alt;
     ps->side = ps->sides[ps->side_idx];
 }
@@ -243,6 +246,8 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
         ss.group_done = ss.sort_ctl + kSortCtlWords;
         ss.rec = (uint4*)(ps->ws + l.rec[b]);
         ss.cellpos = (uint32_t*)(ps->ws + l.cellpos[b]);
+        ss.mf_dup = (uint4*)(ps->ws + l.mf_dup[b]);
+        ss.mf_tickets = (unsigned int*)(ps->ws + l.mf_tickets[b]);
         ss.starters = (uint4*)(ps->ws + l.starters[b]);
         ss.starter_count = (unsigned int*)(ps->ws + l.starter_count[b]);
         ss.used = false;
@@ -277,9 +282,12 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     // the side stream's small kernels should not queue behind the gradient kernel's waves of blocks
     int prio_lo = 0, prio_hi = 0;
     cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-    if (cudaStreamCreateWithPriority(&ps->sides[0], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
-        cudaStreamCreateWithPriority(&ps->sides[1], cudaStreamNonBlocking, prio_hi) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+    for (int b = 0; b < kSideStreams; ++b)
+        if (cudaStreamCreateWithPriority(&ps->sides[b], cudaStreamNonBlocking, prio_hi) != cudaSuccess) {
+            delete ps;
+            return PS_ERR_CUDA;
+        }
+    if (cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
@@ -311,8 +319,7 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
-    cudaStreamDestroy(ps->sides[0]);
-    cudaStreamDestroy(ps->sides[1]);
+    for (int b = 0; b < kSideStreams; ++b) cudaStreamDestroy(ps->sides[b]);
     cudaStreamDestroy(ps->copy);
     for (int b = 0; b < kHostStages; ++b) {
         cudaEventDestroy(ps->ev_copied[b]);
@@ -329,7 +336,7 @@ ps_status_t ps_destroy(ps_store_t* ps) {
 ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
     PS_BEGIN_CALL(ps);
     launch_init_range_partition(ps, s);
-    ps->table_dirty[0] = ps->table_dirty[1] = true;
+    for (int b = 0; b < kSideStreams; ++b) ps->table_dirty[b] = true;
     return after_launch();
 }
 
@@ -376,7 +383,7 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, nullptr, 0);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
     run_localize(ps, worker, (uint32_t)n, which, s);
-    ps->table_dirty[0] = ps->table_dirty[1] = true;
+    for (int b = 0; b < kSideStreams; ++b) ps->table_dirty[b] = true;
     return release_set(ss, s);
 }
 
@@ -392,8 +399,18 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (!fork_side(ps, ss, s, true)) return PS_ERR_CUDA;
     // rows short enough to be staged whole, and row numbers that fit the 32-bit fields of the sort's records
     const bool fused = ps->cfg.row_len <= 128 && (uint64_t)ps->cfg.num_workers * ps->cfg.slots_per_part < (1ull << 32);
+    // The one-launch form over the column side is taken on request only: on the 10M x 1M matrix it runs at 49 us
+    // per step against 45 for the symmetric form (its launch takes 35 to 41 us, the two of the symmetric form 42,
+    // but it adds a kernel to the internal stream, whose sort is what bounds the step).
+    const bool by_column = fused && ps->mf_path == 1;
     const int which = radix_sort_mf(ps, d_i, d_j, d_v, (uint32_t)n, col_key_base, fused, ps->side, ps->starter_count,
                                     div_up_u32(2 * n, fused ? 64 * 8 : kGroupSpan));
+    if (by_column) {
+        launch_mf_plan(ps, (uint32_t)n, which, ps->side);
+        if (!join_side(ps, s)) return PS_ERR_CUDA;
+        run_mf_col(ps, (uint32_t)n, which, lr, lambda, d_loss_accum, s);
+        return release_set(ss, s);
+    }
     if (fused) {
         // gradient and reduction in one kernel over the sorted occurrences: no update rows
         if (!join_side(ps, s)) return PS_ERR_CUDA;
@@ -688,6 +705,12 @@ ps_status_t ps_set_host_overlap(ps_store_t* ps, int on) {
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on) {
     if (!ps) return PS_ERR_INVALID_ARG;
     ps->pipelined = on != 0;
+    return PS_OK;
+}
+
+ps_status_t ps_set_mf_path(ps_store_t* ps, int path) {
+    if (!ps || path < 0 || path > 2) return PS_ERR_INVALID_ARG;
+    ps->mf_path = path;
     return PS_OK;
 }
 

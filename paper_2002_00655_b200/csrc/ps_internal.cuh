@@ -22,7 +22,8 @@ constexpr int kReduceTile = 32;                  // sorted occurrences per warp 
 constexpr int kGroupSpan = 64 * kReduceTile;      // sorted positions whose parked parts are pre-added together
 constexpr int kMaxLossBlocks = 4096;
 constexpr int kHostStages = 3;                   // staging areas for batches that arrive from host memory
-constexpr int kSortSets = 3;                     // calls whose key sort may be in flight at once (see SortSet)
+constexpr int kSortSets = 4;                     // calls whose key sort may be in flight at once (see SortSet)
+constexpr int kSideStreams = 3;                  // internal streams that calls with a long sort take in turn
 
 // Device-resident status words.  An error is latched per call with the call's
 // epoch, so no kernel has to clear anything before a call starts.
@@ -50,6 +51,8 @@ struct SortSet {
     uint32_t* cellpos;
     uint4* starters;
     unsigned int* starter_count;
+    uint4* mf_dup;
+    unsigned int* mf_tickets;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
     bool used;
 };
@@ -76,6 +79,8 @@ struct ps_store {
     uint32_t* sort_ctl;             // the sort's grid barrier (two words) in kSortCtlWords, followed by group_done
     uint4* rec;                     // MF: {cell, cell value, row of the key, row of the other factor} per sorted position
     uint32_t* cellpos;              // MF: sorted position of each cell's row-factor occurrence
+    uint4* mf_dup;                  // MF by column: per column position {first position, count, rank} of its cell's row key
+    unsigned int* mf_tickets;       // MF by column: a ticket counter per row-side position, then one per block, then one
     unsigned int* group_done;       // per group of 64 reduction tiles: reduction blocks that have finished
     double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
@@ -94,9 +99,9 @@ struct ps_store {
     int sm_count;
     psb::Profile* prof;             // per-kernel event timing, off unless ps_profile_start was called
     cudaStream_t side;              // key extraction and sort of the current call run here, beside the gradient kernel:
-    cudaStream_t sides[2];          // one of these two; calls whose sort is longer than the rest of the step take them
-    int side_idx, side_alt;         // in turn, so that the sorts of two later steps run beside each other
-    unsigned long long side_capture_id[2];  // graph capture each of them was last forked into (0 = none)
+    cudaStream_t sides[psb::kSideStreams];  // one of these; calls whose sort is longer than the rest of the step take them
+    int side_idx, side_alt;         // in turn, so that the sorts of several later steps run beside each other
+    unsigned long long side_capture_id[psb::kSideStreams];  // graph capture each of them was last forked into (0 = none)
     cudaEvent_t ev_fork, ev_join;
     psb::SortSet sets[psb::kSortSets];           // keysA .. starter_count above always point into sets[cur_set]
     int cur_set;
@@ -107,7 +112,8 @@ struct ps_store {
     bool host_overlap;
     cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
-    bool table_dirty[2];            // per side stream: the location table was rewritten since that stream last waited
+    int mf_path;                    // see ps_set_mf_path
+    bool table_dirty[psb::kSideStreams];   // per side stream: the location table was rewritten since that stream last waited
                                     // for the caller's (a sort that reads the table must not start before the rewrite)
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
 };
@@ -116,7 +122,7 @@ namespace psb {
 
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
-        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], scan_sums, loc_counts, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], mf_dup[kSortSets], mf_tickets[kSortSets], scan_sums, loc_counts, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
         loss_partial, apply_rows, staging[kHostStages], total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
@@ -197,6 +203,12 @@ void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, do
 // then the fix-up launch that also moves the staged rows into the store
 void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
                   double* d_loss_accum, cudaStream_t s);
+// ---- mf_col.cu ----
+// MF step as one launch over the column side of the sorted occurrences (rows of at most 128 values).  launch_mf_plan
+// goes on the stream the sort ran on, right after it; run_mf_col on the caller's stream after the join.
+void launch_mf_plan(ps_store* ps, uint32_t n_cells, int which, cudaStream_t side);
+void run_mf_col(ps_store* ps, uint32_t n_cells, int which, float lr, float lambda, double* d_loss_accum, cudaStream_t s);
+
 // ComplEx: reduce GRADIENT rows (2 dim values per occurrence, in ps->upd) into AdaGrad steps per key; dim even, <= 128
 void run_kge_reduce(ps_store* ps, uint32_t n, int which, uint32_t dim, float lr, float eps, double* d_loss_accum,
                     uint32_t loss_blocks, cudaStream_t s);

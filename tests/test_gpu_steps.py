@@ -25,13 +25,19 @@ def mf_data(cfg):
     return W.mf_cells(cfg, planted, 0, cfg.n_cells, "cpu")
 
 
-def test_mf_tiny_epoch_free_running_and_localize_transparency():
+MF_PATHS = [ps.PS_MF_SYMMETRIC, ps.PS_MF_BY_COLUMN]      # both sets of kernels on every small case (auto picks by size)
+
+
+@pytest.mark.parametrize("path", MF_PATHS)
+def test_mf_tiny_epoch_free_running_and_localize_transparency(path):
     cfg = W.MF_TINY
     rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
     i, j, v = mf_data(cfg)
     g, o = make_pair(cfg.num_keys, cfg.rank, rows=rows, max_batch_keys=2 * cfg.batch)
     g2, _ = make_pair(cfg.num_keys, cfg.rank, 8, cfg.num_keys, rows=rows,
                       max_batch_keys=2 * cfg.batch)           # same run with relocations in between
+    ps.ps_set_mf_path(g.h, path)
+    ps.ps_set_mf_path(g2.h, path)
     di, dj, dv = i.cuda(), j.cuda(), v.cuda()
     rng = np.random.default_rng(0)
     for b in range(cfg.n_batches):
@@ -51,12 +57,16 @@ def test_mf_tiny_epoch_free_running_and_localize_transparency():
 
 
 @pytest.mark.parametrize("R,Cc,L,n,zipf", [(3000, 500, 100, 5000, 1.1), (400, 300, 8, 1024, None), (1000, 50, 128, 2047, 1.1),
-                                           (200, 200, 260, 999, None), (90, 70, 640, 300, 1.1)])
-def test_mf_single_steps(R, Cc, L, n, zipf):
+                                           (200, 200, 260, 999, None), (90, 70, 640, 300, 1.1),
+                                           (200_000, 300, 100, 6000, 1.1), (50_000, 40, 64, 3000, 1.3),
+                                           (7, 5000, 24, 1500, None)])
+@pytest.mark.parametrize("path", MF_PATHS)
+def test_mf_single_steps(R, Cc, L, n, zipf, path):
     cfg = W.MFConfig("t", R, Cc, L, 4 * n, n, 0.002, 0.05, 0.1, 0.5, zipf)
     rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
     i, j, v = mf_data(cfg)
     g, o = make_pair(cfg.num_keys, L, rows=rows, max_batch_keys=2 * n)
+    ps.ps_set_mf_path(g.h, path)
     for b in range(cfg.n_batches):
         s, c = cfg.batch_range(b)
         if b == cfg.n_batches - 1:
@@ -217,7 +227,8 @@ def test_host_batch_variants_match_the_device_calls():
 
 
 # ---------------------------------------------------------- pipelining ----
-def test_pipelined_mode_gives_identical_results():
+@pytest.mark.parametrize("path", MF_PATHS)
+def test_pipelined_mode_gives_identical_results(path):
     """ps_set_pipelining lets the key sort of step t+1 run beside step t's kernels; nothing may change."""
     cfg = W.scaled(W.MF_TINY, rows=3000, cols=400, rank=100, n_cells=40 * 2048, batch=2048, col_zipf=1.1, lr=0.0005)
     rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
@@ -227,6 +238,7 @@ def test_pipelined_mode_gives_identical_results():
     for pipelined in (False, True):
         g, _ = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
         ps.ps_set_pipelining(g.h, pipelined)
+        ps.ps_set_mf_path(g.h, path)
         torch.cuda.synchronize()
         rng = np.random.default_rng(1)
         for b in range(cfg.n_batches):
@@ -243,7 +255,8 @@ def test_pipelined_mode_gives_identical_results():
     assert np.isfinite(out[0][1])
 
 
-def test_mf_pipelined_steps_with_relocations_in_between():
+@pytest.mark.parametrize("path", MF_PATHS)
+def test_mf_pipelined_steps_with_relocations_in_between(path):
     """In pipelined mode the key sort of a step starts early and reads the location table (it writes the row
     addresses the gradient kernel uses): a localize between two steps must still be seen by the next step."""
     cfg = W.MFConfig("t", 2000, 300, 100, 6 * 1500, 1500, 0.002, 0.05, 0.1, 0.5, 1.1)
@@ -251,6 +264,7 @@ def test_mf_pipelined_steps_with_relocations_in_between():
     i, j, v = mf_data(cfg)
     g, o = make_pair(cfg.num_keys, cfg.rank, 6, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
     ps.ps_set_pipelining(g.h, True)
+    ps.ps_set_mf_path(g.h, path)
     di, dj, dv = i.cuda(), j.cuda(), v.cuda()
     torch.cuda.synchronize()
     rng = np.random.default_rng(3)
@@ -270,8 +284,9 @@ def test_mf_pipelined_steps_with_relocations_in_between():
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
 
 
+@pytest.mark.parametrize("path", MF_PATHS)
 @pytest.mark.parametrize("graph", [False, True])
-def test_two_pipelined_mf_steps_right_after_a_large_localize(graph):
+def test_two_pipelined_mf_steps_right_after_a_large_localize(graph, path):
     """MF steps sort on two internal streams in turn.  After a call that rewrites the location table BOTH streams
     must wait for it before a sort that reads the table: here a localize of 100,000 keys (long enough to be still
     running when the second step's sort could start) is followed by two steps whose cells all use moved keys."""
@@ -280,6 +295,7 @@ def test_two_pipelined_mf_steps_right_after_a_large_localize(graph):
     i, j, v = mf_data(cfg)
     g, o = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=1 << 17)
     ps.ps_set_pipelining(g.h, True)
+    ps.ps_set_mf_path(g.h, path)
     di, dj, dv = i.cuda(), j.cuda(), v.cuda()
     moved = np.concatenate([np.arange(0, 96_000), cfg.col_key_base + np.arange(0, 4_000)]).astype(np.int64)
     d_moved = dev(moved)
@@ -344,7 +360,8 @@ def test_overlapped_host_batches_give_identical_results():
         assert h_loss[0] == loss_of(g)
 
 
-def test_steps_captured_into_a_graph_give_the_same_results_as_eager_calls():
+@pytest.mark.parametrize("path", MF_PATHS)
+def test_steps_captured_into_a_graph_give_the_same_results_as_eager_calls(path):
     """The timed configuration: pipelined steps captured into one CUDA graph (the internal streams join the
     capture), replayed with one launch.  Eager calls before and after the capture use the same handle."""
     cfg = W.scaled(W.MF_TINY, rows=3000, cols=400, rank=100, n_cells=24 * 2048, batch=2048, col_zipf=1.1, lr=0.0005)
@@ -363,6 +380,7 @@ def test_steps_captured_into_a_graph_give_the_same_results_as_eager_calls():
     graphed, o = make_pair(cfg.num_keys, cfg.rank, 4, cfg.num_keys, rows=rows, max_batch_keys=2 * cfg.batch)
     for g in (eager, graphed):
         ps.ps_set_pipelining(g.h, True)
+        ps.ps_set_mf_path(g.h, path)
     for b in range(cfg.n_batches):
         run(eager, b)
     eager.sync()
