@@ -281,12 +281,60 @@ class MFWorkload:
         return cells
 
 
+class MFPushWorkload(MFWorkload):
+    """ps_push alone on the key occurrences of MF-large batches (131,072 keys of 100 values per call): the shape on
+    which the sorted push and the push by atomic adds (--atomic-push) are compared."""
+
+    example = "keys"
+
+    def __init__(self, cfg):
+        super().__init__(cfg)
+        self.example = "keys"
+
+    def describe(self):
+        return dict(super().describe(), workload="push_mf", call="ps_push of the batch's 2 x minibatch key occurrences")
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        super().setup(ps, device, n_steps, keep_host_init)
+        c = self.cfg
+        g = torch.Generator(device=device)
+        g.manual_seed(0)
+        self.upd = [torch.randn((2 * c.batch, c.rank), generator=g, device=device) * 1e-3 for _ in range(4)]
+        b = c.batch
+        self.keys = [torch.cat([self.i[k * b:(k + 1) * b].to(torch.int64),
+                                c.col_key_base + self.j[k * b:(k + 1) * b].to(torch.int64)]) for k in range(n_steps)]
+
+    def units(self, k):
+        return 2 * self.cfg.batch
+
+    def step(self, k):
+        self.ps.ps_push(self.store.h, self.keys[k], self.upd[k % len(self.upd)])
+
+    def host_setup(self, steps):
+        return None
+
+    def alg_bytes(self, k):
+        n, rb = 2 * self.cfg.batch, self.row_bytes
+        return n * (16 + rb) + n_unique(self.keys[k]) * 2 * rb
+
+    def kernel_bytes(self, k, moved=0.0):
+        n, rb = 2 * self.cfg.batch, self.row_bytes
+        u = n_unique(self.keys[k])
+        return {"push_reduce_kernel": n * (8 + rb) + u * (8 + 2 * rb), "push_fixup_kernel": fixup_bytes(self.keys[k], 32, rb),
+                "sort_all_kernel": sort_bytes(n, int(self.cfg.num_keys).bit_length()) + 4 * n,
+                "push_atomic_kernel": n * (16 + rb) + n * 2 * rb, "push_check_keys_kernel": n * 8}
+
+    def oracle_setup(self, device):
+        return None
+
+
 class KGEWorkload:
     """ComplEx + AdaGrad (Section 4.1 / Appendix A task): triples/s through ps_step_kge."""
 
-    def __init__(self, cfg):
+    def __init__(self, cfg, twin=None):
         self.cfg, self.example = cfg, "triples"
         self.row_bytes = cfg.row_len * 4
+        self.twin = twin                        # a store with fewer keys for the oracle leg, where the full one does not fit the host
 
     def describe(self):
         c = self.cfg
@@ -301,10 +349,15 @@ class KGEWorkload:
         c = self.cfg
         self.ps = ps
         self.store = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(3 + c.n_neg) * c.batch, device=device.index)
-        rows = W.kge_init_rows(c, 0, c.num_keys, device)
-        self.store.set_all_rows(rows)
-        self.host_init = rows.cpu() if keep_host_init else None
-        del rows
+        keep = keep_host_init and self.twin is None
+        self.host_init = torch.empty((c.num_keys, c.row_len), dtype=torch.float32) if keep else None
+        chunk = max(1, (1 << 28) // (c.row_len * 4))             # rows per 256 MB
+        for s in range(0, c.num_keys, chunk):
+            n = min(chunk, c.num_keys - s)
+            rows = W.kge_init_rows(c, s, n, device)
+            self.store.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=device), rows)
+            if keep:
+                self.host_init[s:s + n] = rows.cpu()
         self.s, self.r, self.o, self.neg, self.side = W.kge_triples(c, 0, n_steps * c.batch, device)
         torch.cuda.synchronize(device)
 
@@ -354,27 +407,43 @@ class KGEWorkload:
         occ, rb = (3 + c.n_neg) * b, self.row_bytes
         # the step kernel reads the embedding half of every row and writes a gradient row of the same size; the
         # reduction reads those and read-modify-writes every distinct row
-        kb["kge_step"] = b * (12 + c.n_neg * 5) + occ * (8 + rb // 2) + occ * (rb // 2)
-        kb["kge_reduce_kernel"] = occ * (8 + rb // 2) + u * (8 + 2 * rb)
+        if c.dim % 2 == 0 and c.dim <= 128:
+            kb["kge_step"] = b * (12 + c.n_neg * 5) + occ * (8 + rb // 2) + occ * (rb // 2)
+            kb["kge_reduce_kernel"] = occ * (8 + rb // 2) + u * (8 + 2 * rb)
+        # (wider rows: the step kernel reads whole rows and writes finished update rows, reduced like a push's)
         return kb
 
     def oracle_setup(self, device):
         from oracle import OracleStore
-        c = self.cfg
+        c = self.twin or self.cfg
+        if self.twin is not None:
+            self.oracle_name = (f"{c.name} ({c.entities} entities, the same rows and minibatch: a K-scaled twin of "
+                                f"{self.cfg.name}, whose store the oracle would have to hold in host memory)")
         o = OracleStore(c.num_keys, c.row_len, 1)
-        rows = self.host_init if getattr(self, "host_init", None) is not None else W.kge_init_rows(c, 0, c.num_keys, device).cpu()
-        o.set_rows(np.arange(c.num_keys), rows.numpy())
+        if getattr(self, "host_init", None) is not None:
+            o.set_rows(np.arange(c.num_keys), self.host_init.numpy())
+        else:
+            chunk = max(1, (1 << 28) // (c.row_len * 4))
+            for s in range(0, c.num_keys, chunk):
+                n = min(chunk, c.num_keys - s)
+                o.set_rows(np.arange(s, s + n), W.kge_init_rows(c, s, n, device).cpu().numpy())
         self.oracle = o
         return o
 
     def oracle_data(self, device, n_steps):
-        if not hasattr(self, "s"):
-            self.s, self.r, self.o, self.neg, self.side = W.kge_triples(self.cfg, 0, n_steps * self.cfg.batch, device)
-        n = n_steps * self.cfg.batch
-        self.od = [t[:n].cpu().numpy() for t in (self.s, self.r, self.o, self.neg, self.side)]
+        c = self.twin or self.cfg
+        if self.twin is not None or not hasattr(self, "s"):
+            n_steps = min(n_steps, 16)
+            d = W.kge_triples(c, 0, n_steps * c.batch, device)
+        else:
+            d = (self.s, self.r, self.o, self.neg, self.side)
+        n = n_steps * c.batch
+        self.od = [t[:n].cpu().numpy() for t in d]
+        self.o_steps = n_steps
 
     def oracle_step(self, k, n):
-        c, b = self.cfg, self.cfg.batch
+        c, b = self.twin or self.cfg, self.cfg.batch
+        k = k % self.o_steps
         sl = slice(k * b, k * b + n)
         s, r, o, neg, side = (t[sl] for t in self.od)
         self.oracle.step_kge(s, r, o, neg, side, c.rel_key_base, c.dim, c.lr, c.eps)
@@ -570,6 +639,7 @@ class StressWorkload:
         return {"pull_bulk_kernel": n * (16 + 2 * rb), "pull_kernel": n * (16 + 2 * rb),
                 "push_reduce_kernel": n * (8 + rb) + u * (8 + 2 * rb),
                 "push_fixup_kernel": fixup_bytes(self.keys[k], 32, rb),
+                "push_atomic_kernel": n * (16 + rb) + n * 2 * rb, "push_check_keys_kernel": n * 8,
                 # two sorts per step (push: 1M keys, localize: 100k keys), 64-bit caller keys in
                 "sort_all_kernel": (sort_bytes(n, bits) + 4 * n + sort_bytes(nl, bits) + 4 * nl) / 2,
                 # the relocation after its key sort: sorted keys and table entries in (twice: count, then assign),
@@ -611,9 +681,10 @@ class StressWorkload:
 
 
 def make_workload(name):
-    table = {"mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
+    table = {"push_mf": lambda: MFPushWorkload(W.MF_LARGE), "mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
              "mf_medium": lambda: MFWorkload(W.MF_MEDIUM),
              "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
+             "kge_4000": lambda: KGEWorkload(W.KGE_4000, twin=W.KGE_4000_TWIN),
              "sgns": lambda: SGNSWorkload(W.SGNS), "sgns_tiny": lambda: SGNSWorkload(W.SGNS_TINY),
              "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY),
              "stress_medium": lambda: StressWorkload(W.STRESS_MEDIUM)}
@@ -713,6 +784,10 @@ def run_ours(args):
     assert code == 0, f"device error during setup: {code}"
     # every batch array exists and is complete before the first step: the precondition of pipelined mode
     ps.ps_set_pipelining(h, not args.no_pipelining)
+    if args.atomic_push:
+        ps.ps_set_push_mode(h, ps.PS_PUSH_ATOMIC)
+    if args.mf_by_column:
+        ps.ps_set_mf_path(h, ps.PS_MF_BY_COLUMN)
 
     for k in range(args.warmup):
         wl.step(k)
@@ -833,7 +908,9 @@ def run_ours(args):
         "config": dict(wl.describe(), parallelism="replicas only" if world > 1 else "single GPU",
                        accumulation="per-key sums of update terms in f64 (a key that occurs once in the batch: one f32 "
                                     "add, the same single rounding); terms formed in f32; state f32",
-                       pipelining="off" if args.no_pipelining else "key sort of step t+1 beside step t (ps_set_pipelining)"),
+                       pipelining="off" if args.no_pipelining else "key sort of step t+1 beside step t (ps_set_pipelining)",
+                       push="atomic adds (no sort, not reproducible)" if args.atomic_push else "sorted segmented reduction",
+                       **({"mf_path": "one launch over the column side"} if args.mf_by_column else {})),
         "gpu_launches": int(round(launches_per_step * steps * repeats)), "launches_per_step": launches_per_step,
         "host_enqueue_ms_per_step": host_ms / len(timed),
         "launch_mode": "one CUDA graph per repeat" if graphs is not None else "eager",
@@ -915,12 +992,15 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mf_large",
-                    choices=["mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny",
+                    choices=["push_mf", "mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "kge_4000", "sgns", "sgns_tiny", "stress", "stress_tiny",
                              "stress_medium"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--repeats", type=int, default=0,
                     help="timed repeats of --steps steps, each on batches of its own (0: 5 to 30, more for short runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--atomic-push", action="store_true",
+                    help="ps_push by vector atomic adds instead of the sorted segmented reduction (measured alternative)")
+    ap.add_argument("--mf-by-column", action="store_true", help="ps_step_mf as one launch over the column side")
     ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host")
     ap.add_argument("--no-pipelining", action="store_true",
                     help="order each step's key sort after all earlier work instead of beside the previous step")

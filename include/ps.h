@@ -257,6 +257,17 @@ ps_status_t ps_set_pipelining(ps_store_t* ps, int on);
  * for the device.  Do not capture ps_step_*_host calls into a CUDA graph. */
 ps_status_t ps_set_host_overlap(ps_store_t* ps, int on);
 
+/* How ps_push adds (Section 2.1: the push is cumulative; the paper's servers serialise the adds of a key with
+ * latches, Section 3.7).
+ *   PS_PUSH_SORTED (default): occurrences sorted by key, per-key sums in fp64, one rounding, one write per key;
+ *     results are reproducible bit for bit.
+ *   PS_PUSH_ATOMIC: no sort; every occurrence adds its row with vector atomic adds.  Kept as a measured
+ *     alternative: each term is rounded into the row as it arrives and the order is the hardware's, so keys
+ *     with more than two terms in a call are not reproducible from run to run (and differ from the sorted
+ *     push in the last bits).  Integer-valued updates are exact either way.  Not limited by the workspace. */
+enum { PS_PUSH_SORTED = 0, PS_PUSH_ATOMIC = 1 };
+ps_status_t ps_set_push_mode(ps_store_t* ps, int mode);
+
 /* Which kernels ps_step_mf uses on rows of at most 128 values (results are the same to rounding order; both
  * sum a key's terms in fp64 in the order of the sorted occurrences and round once).
  *   PS_MF_BY_COLUMN: one launch that visits the column-factor occurrences only; each forms its cell's terms

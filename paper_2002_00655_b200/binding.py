@@ -27,6 +27,7 @@ PS_ERR_WORKSPACE = 5
 PS_ERR_CUDA = 6
 PS_ERR_UNSUPPORTED = 7
 PS_MF_AUTO, PS_MF_BY_COLUMN, PS_MF_SYMMETRIC = 0, 1, 2
+PS_PUSH_SORTED, PS_PUSH_ATOMIC = 0, 1
 PS_PUSH_STATIC_MAX_KEYS = 16384
 PS_PUSH_STATIC_MAX_ROW_LEN = 256
 
@@ -68,6 +69,7 @@ SIGNATURES = {
     "ps_set_pipelining": (C.c_int, [_vp, C.c_int]),
     "ps_set_host_overlap": (C.c_int, [_vp, C.c_int]),
     "ps_set_mf_path": (C.c_int, [_vp, C.c_int]),
+    "ps_set_push_mode": (C.c_int, [_vp, C.c_int]),
     "ps_launch_count": (C.c_uint64, [_vp]),
     "ps_rows_moved": (C.c_int, [_vp, C.POINTER(_u64)]),
     "ps_profile_start": (C.c_int, [_vp, _u32]),
@@ -249,6 +251,10 @@ def ps_set_host_overlap(ps, on: bool) -> None:
 
 def ps_set_pipelining(ps, on: bool) -> None:
     _check(load_library().ps_set_pipelining(ps, 1 if on else 0), "ps_set_pipelining")
+
+
+def ps_set_push_mode(ps, mode: int) -> None:
+    _check(load_library().ps_set_push_mode(ps, int(mode)), "ps_set_push_mode")
 
 
 def ps_set_mf_path(ps, path: int) -> None:

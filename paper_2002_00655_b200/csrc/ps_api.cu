@@ -360,6 +360,11 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
     PS_BEGIN_CALL(ps);
     if (n == 0) return PS_OK;
     if (!d_keys || !d_updates || ((uintptr_t)d_updates & 15)) return PS_ERR_INVALID_ARG;
+    if (ps->push_mode == PS_PUSH_ATOMIC) {
+        SortSet* ss = next_set(ps);                         // (for the call's number; nothing is sorted)
+        run_push_atomic(ps, d_keys, n, d_updates, s);
+        return release_set(ss, s);
+    }
     if (n > ps->max_keys) return PS_ERR_WORKSPACE;
     SortSet* ss = next_set(ps);
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;         // the keys are sorted beside earlier calls' kernels
@@ -705,6 +710,12 @@ ps_status_t ps_set_host_overlap(ps_store_t* ps, int on) {
 ps_status_t ps_set_pipelining(ps_store_t* ps, int on) {
     if (!ps) return PS_ERR_INVALID_ARG;
     ps->pipelined = on != 0;
+    return PS_OK;
+}
+
+ps_status_t ps_set_push_mode(ps_store_t* ps, int mode) {
+    if (!ps || (mode != PS_PUSH_SORTED && mode != PS_PUSH_ATOMIC)) return PS_ERR_INVALID_ARG;
+    ps->push_mode = mode;
     return PS_OK;
 }
 

@@ -113,6 +113,7 @@ struct ps_store {
     cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
     int mf_path;                    // see ps_set_mf_path
+    int push_mode;                  // see ps_set_push_mode
     bool table_dirty[psb::kSideStreams];   // per side stream: the location table was rewritten since that stream last waited
                                     // for the caller's (a sort that reads the table must not start before the rewrite)
     unsigned long long capture_id;  // graph capture the caller's stream was in at the last step call (0 = none)
@@ -198,6 +199,9 @@ void run_push_pipeline(ps_store* ps, uint32_t n, const float* d_upd, double* d_l
 int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s);
 void run_push_reduce(ps_store* ps, uint32_t n, int which, const float* d_upd, double* d_loss_accum,
                      uint32_t loss_blocks, cudaStream_t s, const float* d_scales = nullptr, uint32_t slots = 0);
+
+// push by atomic adds, no sort (ps_set_push_mode)
+void run_push_atomic(ps_store* ps, const uint64_t* d_keys, uint64_t n, const float* d_upd, cudaStream_t s);
 
 // MF step working on the sorted occurrences directly (rows of at most 512 values): gradient, reduction,
 // then the fix-up launch that also moves the staged rows into the store

@@ -1224,6 +1224,54 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
     }
 }
 
+// ------------------------------------------------- push by atomic adds (measured alternative) ----
+// The cumulative push without the sort: every occurrence adds its update row to the key's row with
+// `red.global.add.v4.f32`.  The order in which the terms of a key meet is whatever the hardware makes of it, so
+// sums of more than two terms are not reproducible from run to run, and every term is rounded into the row as
+// it arrives (fp32), not summed in fp64 and rounded once.  A first kernel checks the keys, so that a call with a
+// key out of range still changes nothing.
+__global__ void __launch_bounds__(256)
+push_check_keys_kernel(const uint64_t* __restrict__ keys, uint64_t n, uint64_t K, DevStatus* st, unsigned int epoch) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n && keys[t] >= K) latch_error(st, epoch, PS_ERR_KEY_RANGE);
+}
+
+__global__ void __launch_bounds__(256)
+push_atomic_kernel(const uint64_t* __restrict__ keys, uint64_t n, const float4* __restrict__ upd, float4* store,
+                   const uint2* __restrict__ table, uint64_t S, uint32_t L4, const DevStatus* st, unsigned int epoch) {
+    if (call_failed(st, epoch)) return;
+    const int lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t n_warps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    // a warp takes four occurrences at a time: four table look-ups and up to four update chunks per lane in flight
+    for (uint64_t t0 = warp * 4; t0 < n; t0 += n_warps * 4) {
+        uint64_t row[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) row[r] = t0 + r < n ? phys_row(table[keys[t0 + r]], S) : 0;
+        for (uint32_t f = lane; f < L4; f += 32) {
+            float4 u[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                u[r] = t0 + r < n ? __ldcs(upd + (t0 + r) * L4 + f) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (t0 + r < n) {
+                    float* d = reinterpret_cast<float*>(store + row[r] * L4 + f);
+                    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d), "f"(u[r].x), "f"(u[r].y),
+                                 "f"(u[r].z), "f"(u[r].w)
+                                 : "memory");
+                }
+        }
+    }
+}
+
+void run_push_atomic(ps_store* ps, const uint64_t* d_keys, uint64_t n, const float* d_upd, cudaStream_t s) {
+    PS_LAUNCH(ps, push_check_keys_kernel, div_up_u32(n, 256), 256, s, d_keys, n, ps->cfg.num_keys, ps->status, ps->epoch);
+    const uint32_t grid = (uint32_t)tmin<uint64_t>((n + 31) / 32, (uint64_t)ps->sm_count * 8);
+    PS_LAUNCH(ps, push_atomic_kernel, grid, 256, s, d_keys, n, (const float4*)d_upd, (float4*)ps->store, ps->table,
+              ps->cfg.slots_per_part, ps->cfg.row_len / 4, ps->status, ps->epoch);
+}
+
 int run_push_sort(ps_store* ps, uint32_t n, cudaStream_t s) {
     return radix_sort_pairs(ps, n, nullptr, ps->key_bits, s, 0, ps->starter_count, div_up_u32(n, kGroupSpan));
 }

@@ -204,6 +204,12 @@ class KGEConfig:
 
 KGE = KGEConfig("kge", 500_000, 1_000, 100, 3_000_000, 10, 8_192, 0.1, 1e-8, 0.1, 1.0)
 KGE_TINY = KGEConfig("kge_tiny", 2_000, 16, 12, 6_000, 10, 256, 0.1, 1e-8, 0.1, 1.0)
+# The paper's ComplEx-Large (Section 4.1, Tables 4 and 5): 4000 complex dimensions, i.e. 8000 values plus 8000 AdaGrad
+# accumulators per key (64 KB rows in fp32; a 32 GB store for the same 500k entities).  Minibatches of 2,048 triples:
+# the update rows of a step are materialised for rows this wide, 1.7 GB at this size.
+KGE_4000 = KGEConfig("kge_4000", 500_000, 1_000, 4000, 3_000_000, 10, 2_048, 0.1, 1e-8, 0.1, 1.0)
+# the same rows on 20,000 entities: what the CPU oracle can hold when it is timed beside the full size
+KGE_4000_TWIN = KGEConfig("kge_4000_twin", 20_000, 1_000, 4000, 3_000_000, 10, 2_048, 0.1, 1e-8, 0.1, 1.0)
 
 
 def kge_init_rows(cfg: KGEConfig, key_start: int, count: int, device) -> torch.Tensor:

@@ -154,6 +154,56 @@ def test_kge_steps():
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
 
 
+def test_kge_4000_single_steps():
+    """ComplEx with 4000 complex dimensions (the paper's ComplEx-Large: 8000 values and 8000 AdaGrad accumulators
+    per key, 64 KB rows, a 32 GB store).  The oracle cannot hold the store, but a step reads and writes only the
+    rows of its batch's keys: the oracle gets a store of exactly those keys, renumbered in key order (entities
+    before relations, as in the full numbering), and the batch with its keys renumbered the same way."""
+    c = W.KGE_4000
+    need(8, 48)
+    g = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(3 + c.n_neg) * c.batch)
+    chunk = 4096
+    for s in range(0, c.num_keys, chunk):
+        n = min(chunk, c.num_keys - s)
+        g.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=DEV), W.kge_init_rows(c, s, n, DEV))
+    ps.ps_set_pipelining(g.h, True)
+    small = 1024                                                # keys per pull or set call: 64 MB of rows
+    touched = []
+
+    def rows_of(keys):
+        out = np.empty((len(keys), c.row_len), dtype=np.float32)
+        for s in range(0, len(keys), small):
+            out[s:s + small] = g.pull(dev(keys[s:s + small])).cpu().numpy()
+        g.sync()
+        return out
+
+    for step, (first, n) in enumerate([(0, c.batch), (c.batch, c.batch), c.batch_range(c.n_batches - 1)]):
+        d = W.kge_triples(c, first, n, DEV)
+        s_, r_, o_, neg, side = (t.cpu().numpy() for t in d)
+        keys = np.unique(np.concatenate([s_, o_, neg.ravel(), r_.astype(np.int64) + c.rel_key_base]).astype(np.int64))
+        n_ent = int((keys < c.rel_key_base).sum())
+        touched.append(keys)
+        o = OracleStore(len(keys), c.row_len, 1)
+        before = rows_of(keys)
+        if step == 1:                                           # a step from accumulators that are not zero
+            before[:, 2 * c.dim:] = np.abs(np.random.default_rng(1).normal(0, 0.05, size=(len(keys), 2 * c.dim))).astype(np.float32)
+            for s in range(0, len(keys), small):
+                g.set_rows(dev(keys[s:s + small]), torch.from_numpy(before[s:s + small]).cuda())
+        o.set_rows(np.arange(len(keys)), before)
+        g.loss.zero_()
+        ps.ps_step_kge(g.h, *d, c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps, g.loss)
+        rn = lambda x: np.searchsorted(keys, x.astype(np.int64)).astype(np.int32)       # noqa: E731
+        o.step_kge(rn(s_), (np.searchsorted(keys, r_.astype(np.int64) + c.rel_key_base) - n_ent).astype(np.int32), rn(o_),
+                   rn(neg.ravel()).reshape(neg.shape), side, n_ent, c.dim, c.lr, c.eps)
+        g.sync()
+        assert_close(rows_of(keys), o.rows, f"kge_4000, step {step}")
+        assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+        del o
+    rest = np.setdiff1d(np.random.default_rng(5).integers(0, c.num_keys, size=300), np.concatenate(touched))
+    want = np.concatenate([W.kge_init_rows(c, int(k), 1, DEV).cpu().numpy() for k in rest[:64]])
+    assert (rows_of(rest[:64]) == want).all(), "kge_4000: a row no batch touched has changed"
+
+
 def test_sgns_steps():
     c = W.SGNS
     need(8, 16)

@@ -63,6 +63,32 @@ def test_push_matches_oracle(K, L, n, hot):
     compare_state(g, o, what="push")
 
 
+def test_push_by_atomic_adds_is_exact_on_integers_and_refuses_bad_keys():
+    """The measured alternative to the sorted push: no order of adds is promised, so only integer-valued updates
+    (exact in any order) are compared bit for bit; a call with a key out of range must still change nothing."""
+    import paper_2002_00655_b200 as ps
+    K, L, n = 3000, 100, 20_000
+    g, o = make_pair(K, L, 3, rows=f_row(np.arange(K), L), max_batch_keys=64)      # the call is larger than the workspace's batch
+    ps.ps_set_push_mode(g.h, ps.PS_PUSH_ATOMIC)
+    rng = np.random.default_rng(3)
+    keys = (rng.zipf(1.2, size=n) - 1) % K
+    upd = rng.integers(-3, 4, size=(n, L)).astype(np.float32)
+    g.push(dev(keys), dev(upd))
+    g.sync()
+    o.push(keys, upd)
+    compare_state(g, o, exact_rows=True, what="atomic push")
+    keys[n // 2] = K
+    g.push(dev(keys), dev(upd))
+    assert g.sync(check=False) == ps.PS_ERR_KEY_RANGE
+    compare_state(g, o, exact_rows=True, what="atomic push with a bad key")
+    ps.ps_set_push_mode(g.h, ps.PS_PUSH_SORTED)
+    small = rng.normal(size=(50, L)).astype(np.float32)
+    g.push(dev(keys[:50]), dev(small))
+    g.sync()
+    o.push(keys[:50], small)
+    compare_state(g, o, what="sorted push afterwards")
+
+
 def test_push_and_pull_reject_bad_keys_without_touching_the_store():
     import paper_2002_00655_b200 as ps
     K, L = 500, 12
