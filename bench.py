@@ -611,11 +611,21 @@ class StressWorkload:
     def units(self, k):
         return self.cfg.batch
 
+    prelocalize = None      # None: localize the batch's own keys after its push; "same": the NEXT batch's keys on the
+                            # same stream; "beside": the next batch's keys on a second stream, beside the push
+
     def step(self, k):
         c, h = self.cfg, self.store.h
         self.ps.ps_pull(h, self.keys[k], self.out)
         self.ps.ps_push(h, self.keys[k], self.upd[k % len(self.upd)])
-        self.ps.ps_localize(h, c.requester(k), self.keys[k][:c.localize_count])
+        if self.prelocalize is None:
+            self.ps.ps_localize(h, c.requester(k), self.keys[k][:c.localize_count])
+            return
+        nxt = self.keys[min(k + 1, len(self.keys) - 1)][:c.localize_count]
+        if self.prelocalize == "same":
+            self.ps.ps_localize(h, c.requester(k + 1), nxt)
+        else:
+            self.ps.ps_localize_beside(h, c.requester(k + 1), nxt, self.loc_stream)
 
     def host_setup(self, steps):
         return None
@@ -788,6 +798,12 @@ def run_ours(args):
         ps.ps_set_push_mode(h, ps.PS_PUSH_ATOMIC)
     if args.mf_by_column:
         ps.ps_set_mf_path(h, ps.PS_MF_BY_COLUMN)
+    if args.prelocalize:
+        assert hasattr(wl, "prelocalize"), "--prelocalize is for the stress workloads"
+        wl.prelocalize = args.prelocalize
+        wl.loc_stream = torch.cuda.Stream(device)
+        if args.prelocalize == "beside":
+            wl.graph_ok = False                                 # two caller streams: the calls are issued eagerly
 
     for k in range(args.warmup):
         wl.step(k)
@@ -910,7 +926,9 @@ def run_ours(args):
                                     "add, the same single rounding); terms formed in f32; state f32",
                        pipelining="off" if args.no_pipelining else "key sort of step t+1 beside step t (ps_set_pipelining)",
                        push="atomic adds (no sort, not reproducible)" if args.atomic_push else "sorted segmented reduction",
-                       **({"mf_path": "one launch over the column side"} if args.mf_by_column else {})),
+                       **({"mf_path": "one launch over the column side"} if args.mf_by_column else {}),
+                       **({"prelocalize": f"keys of the next batch, {args.prelocalize}",
+                           "localize_stats": ps.ps_localize_stats(h)} if args.prelocalize else {})),
         "gpu_launches": int(round(launches_per_step * steps * repeats)), "launches_per_step": launches_per_step,
         "host_enqueue_ms_per_step": host_ms / len(timed),
         "launch_mode": "one CUDA graph per repeat" if graphs is not None else "eager",
@@ -1001,6 +1019,9 @@ def main():
     ap.add_argument("--atomic-push", action="store_true",
                     help="ps_push by vector atomic adds instead of the sorted segmented reduction (measured alternative)")
     ap.add_argument("--mf-by-column", action="store_true", help="ps_step_mf as one launch over the column side")
+    ap.add_argument("--prelocalize", choices=["same", "beside"], default=None,
+                    help="stress workload: localize the NEXT batch's keys after each push, on the same stream or on a "
+                         "second stream beside the push (ps_localize_beside; eager launches)")
     ap.add_argument("--no-graph", action="store_true", help="issue every step's launches from the host")
     ap.add_argument("--no-pipelining", action="store_true",
                     help="order each step's key sort after all earlier work instead of beside the previous step")

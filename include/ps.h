@@ -124,6 +124,34 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
 ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n,
                         void* stream);
 
+/* Pre-localization (Section 2.2 "latency hiding", Section 2.3, Appendix A: while a worker processes one data
+ * point it localizes the parameters of the next one, negatives included).  The call is ps_localize for the keys
+ * of the NEXT batch, enqueued on `loc_stream`, a stream other than the one the handle's most recent call (the
+ * step or push of the current batch) was issued on, so that it runs beside that call:
+ *   - it starts once every call made before the most recent one has finished;
+ *   - keys that the most recent call does not touch are relocated beside it; keys that it does touch keep their
+ *     table entry and their row until it has finished, and are relocated then (both on `loc_stream`);
+ *   - every call made on the handle afterwards, on any stream, is ordered after the whole relocation.
+ * The result (table, free stacks, rows) is that of ps_localize issued right after the most recent call.
+ * If there is nothing to run beside (the most recent call was not a step or push, or was issued on
+ * `loc_stream`), or the store has more than 1024 partitions, the call is an ordinary ps_localize on `loc_stream`
+ * ordered after everything issued so far.  One such call per step; do not capture it into a CUDA graph. */
+ps_status_t ps_localize_beside(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n,
+                               void* loc_stream);
+
+/* Counters over all localize calls of the handle so far (Table 5 of the paper reports the like: relocations,
+ * local and non-local accesses).  Synchronous.
+ *   requested      keys handed in, repeats included
+ *   moved          keys relocated (= ps_rows_moved)
+ *   already_local  distinct keys of a call that the requester owned already
+ *   moved_again    relocated keys that had left their initial partition before, i.e. that were taken from a
+ *                  worker that had localized them earlier: the localization conflicts of Section 3.2
+ *   deferred       relocated keys that had to wait for the call running beside a ps_localize_beside */
+typedef struct {
+    uint64_t requested, moved, already_local, moved_again, deferred;
+} ps_localize_stats_t;
+ps_status_t ps_localize_stats(ps_store_t* ps, ps_localize_stats_t* h_out);
+
 /* One SGD minibatch of low-rank matrix factorization (task of Section 4.1).
  * Key i is row factor w_i (i < col_key_base); key col_key_base + j is column
  * factor h_j.  For each of n cells (d_i[t], d_j[t], d_v[t]), at the pre-batch

@@ -54,6 +54,8 @@ SIGNATURES = {
     "ps_pull": (C.c_int, [_vp, _vp, _u64, _vp, _vp]),
     "ps_push": (C.c_int, [_vp, _vp, _u64, _vp, _vp]),
     "ps_localize": (C.c_int, [_vp, _u32, _vp, _u64, _vp]),
+    "ps_localize_beside": (C.c_int, [_vp, _u32, _vp, _u64, _vp]),
+    "ps_localize_stats": (C.c_int, [_vp, _vp]),
     "ps_step_mf": (C.c_int, [_vp, _vp, _vp, _vp, _u64, _u64, _f32, _f32, _vp, _vp]),
     "ps_step_kge": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _u32, _f32, _f32, _vp, _vp]),
     "ps_step_sgns": (C.c_int, [_vp, _vp, _u64, _u64, _u64, _u32, _vp, _u32, _u64, _f32, _vp, _vp]),
@@ -176,6 +178,22 @@ def ps_push(ps, d_keys, d_updates):
 
 def ps_localize(ps, worker, d_keys):
     _check(load_library().ps_localize(ps, worker, _dptr(d_keys, _U64), d_keys.numel(), _stream()), "ps_localize")
+
+
+def ps_localize_beside(ps, worker, d_keys, loc_stream):
+    """loc_stream: a torch.cuda.Stream other than the current one."""
+    _check(load_library().ps_localize_beside(ps, worker, _dptr(d_keys, _U64), d_keys.numel(), loc_stream.cuda_stream),
+           "ps_localize_beside")
+
+
+class ps_localize_stats_t(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("requested", "moved", "already_local", "moved_again", "deferred")]
+
+
+def ps_localize_stats(ps) -> dict:
+    out = ps_localize_stats_t()
+    _check(load_library().ps_localize_stats(ps, C.byref(out)), "ps_localize_stats")
+    return {n: getattr(out, n) for n, _ in out._fields_}
 
 
 def ps_step_mf(ps, d_i, d_j, d_v, col_key_base, lr, lam, d_loss_accum=None):

@@ -17,8 +17,9 @@ struct LocScratch {
     uint32_t *flag, *mkey, *mowner, *mslot, *mnew;
 };
 
+// (a region of its own, not the update-row scratch: a relocation may run beside a step that is using that)
 static LocScratch loc_scratch(ps_store* ps) {
-    uint32_t* base = (uint32_t*)ps->upd;
+    uint32_t* base = ps->loc_scratch;
     LocScratch s;
     s.flag = base;
     s.mkey = base + ps->max_keys;
@@ -170,11 +171,13 @@ __global__ void __launch_bounds__(256, 2)
 loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uint2* table, uint32_t worker,
                  uint32_t N, uint64_t S, uint32_t K, unsigned long long* tops, uint32_t* stacks, char* store,
                  uint32_t row_bytes, uint32_t* block_counts, uint32_t* owner_counts, LocScratch sc,
-                 unsigned int* bar, DevStatus* st, unsigned int epoch) {
+                 const uint32_t* __restrict__ busy_keys, uint32_t n_busy, uint32_t part_size, unsigned int* bar,
+                 DevStatus* st, unsigned int epoch) {
     __shared__ uint32_t s_hist[kLocFastWorkers];    // phase 2a: keys leaving each owner from this block; phase 3: next stack position
     __shared__ uint32_t s_top[kLocFastWorkers];     // stack heights before the call (S < 2^32)
     __shared__ uint32_t s_part[2][256];
     __shared__ uint32_t sm[8];
+    __shared__ uint32_t s_stat[2];
     __shared__ int s_ok;
     __shared__ __align__(8) uint64_t bars[8][kLocStages];
     extern __shared__ __align__(128) char loc_stage[];
@@ -190,9 +193,18 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         return table[key].x != worker;
     };
     // ---- phase 1 ----
-    uint32_t cnt = 0;
-    for (uint32_t t0 = lo; t0 < hi; t0 += 256) cnt += (uint32_t)__syncthreads_count(must_move(t0 + tid));
-    if (tid == 0) block_counts[b] = cnt;
+    uint32_t cnt = 0, n_local = 0;
+    for (uint32_t t0 = lo; t0 < hi; t0 += 256) {
+        const uint32_t pos = t0 + tid;
+        const bool mv = must_move(pos);
+        const bool first = pos < hi && sk[pos] < K && (pos == 0 || sk[pos - 1] != sk[pos]);
+        cnt += (uint32_t)__syncthreads_count(mv);
+        n_local += (uint32_t)__syncthreads_count(first && !mv);
+    }
+    if (tid == 0) {
+        block_counts[b] = cnt;
+        if (b == 0) st->deferred_now = 0u;                      // (added to after the barrier)
+    }
     if (!grid_barrier(bar, G, &s_ok)) {
         if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
         return;
@@ -208,7 +220,10 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
     block_exclusive_scan_256(before, sm, &m0);
     block_exclusive_scan_256(all, sm, &total);
     const unsigned long long top_w = tops[worker];
-    if (b == 0 && tid == 0) st->moved_total = total;
+    if (b == 0 && tid == 0) {
+        st->moved_total = total;
+        st->loc_requested += n;
+    }
     if ((unsigned long long)total > top_w) {                    // the same decision in every block: nothing has changed yet
         if (b == 0 && tid == 0) latch_error(st, epoch, PS_ERR_CAPACITY);
         grid_leave(bar, G);
@@ -218,6 +233,7 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         s_hist[i] = 0u;
         s_top[i] = (uint32_t)tops[i];
     }
+    if (tid < 2) s_stat[tid] = 0u;
     __syncthreads();
     uint32_t running = 0;
     for (uint32_t t0 = lo; t0 < hi; t0 += 256) {
@@ -229,15 +245,36 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
             const uint32_t m = m0 + running + ex;
             const uint2 e = table[key];
             const uint32_t new_slot = stacks[(uint64_t)worker * S + (top_w - 1 - m)];
+            // A key that the call running beside this one also touches keeps its table entry and its row until
+            // that call is through (loc_deferred_kernel); its slot and its old owner's stack are settled now.
+            bool wait_for_it = false;
+            if (busy_keys) {
+                uint32_t lo2 = 0, hi2 = n_busy;
+                while (lo2 < hi2) {
+                    const uint32_t mid = (lo2 + hi2) >> 1;
+                    if (busy_keys[mid] < key) lo2 = mid + 1; else hi2 = mid;
+                }
+                wait_for_it = lo2 < n_busy && busy_keys[lo2] == key;
+            }
+            sc.mkey[m] = key;
+            sc.flag[m] = wait_for_it ? 1u : 0u;
             sc.mowner[m] = e.x;
             sc.mslot[m] = e.y;
             sc.mnew[m] = new_slot;
-            table[key] = make_uint2(worker, new_slot);
+            if (!wait_for_it) table[key] = make_uint2(worker, new_slot);
             atomicAdd(&s_hist[e.x], 1u);
+            if (wait_for_it) atomicAdd(&s_stat[0], 1u);
+            if (e.x != key / part_size) atomicAdd(&s_stat[1], 1u);      // it had left its initial partition before
         }
         running += tot;
     }
     __syncthreads();
+    if (tid == 0) {
+        if (s_stat[0]) atomicAdd(&st->loc_deferred, (unsigned long long)s_stat[0]);
+        if (s_stat[1]) atomicAdd(&st->loc_moved_again, (unsigned long long)s_stat[1]);
+        if (n_local) atomicAdd(&st->loc_already_local, (unsigned long long)n_local);
+        if (s_stat[0]) atomicAdd(&st->deferred_now, s_stat[0]);
+    }
     for (uint32_t i = tid; i < N; i += 256) owner_counts[(size_t)b * N + i] = s_hist[i];
     __threadfence();
     grid_arrive(bar);                                           // (has a __syncthreads: the block's records are complete)
@@ -259,19 +296,20 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
             rows_of[stage] = 0;
             if (r >= n_rounds) return;
             const uint32_t i = r * per_round + lane;
-            const bool mine = (uint32_t)lane < per_round && i < cnt;
+            bool mine = (uint32_t)lane < per_round && i < cnt;
             uint64_t src = 0;
             if (mine) {
                 const uint32_t m = m0 + i;
+                mine = sc.flag[m] == 0u;                        // (rows that wait for the call beside this one move later)
                 src = (uint64_t)sc.mowner[m] * S + sc.mslot[m];
                 dst_of[stage] = (uint64_t)worker * S + sc.mnew[m];
             }
-            const uint32_t rows = tmin<uint32_t>(per_round, cnt - r * per_round);
+            const uint32_t rows = (uint32_t)__popc(__ballot_sync(0xffffffffu, mine));
             mine_of[stage] = mine;
             rows_of[stage] = rows;
             bulk_wait_read<kLocStages - 2>();                   // the stores that last read this stage have let go of it
             __syncwarp();
-            if (lane == 0) mbar_expect_tx(&bars[w][stage], rows * row_bytes);
+            if (lane == 0) mbar_expect_tx(&bars[w][stage], rows * row_bytes);   // (rows may be 0: the phase completes at once)
             __syncwarp();
             if (mine) bulk_g2s(my + (size_t)stage * kLocStageBytes + (size_t)lane * row_bytes, store + src * row_bytes,
                                row_bytes, &bars[w][stage]);
@@ -311,6 +349,7 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         float4* st4 = reinterpret_cast<float4*>(store);
         for (uint32_t i = w; i < cnt; i += 8) {
             const uint32_t m = m0 + i;
+            if (sc.flag[m]) continue;
             const uint64_t src = (uint64_t)sc.mowner[m] * S + sc.mslot[m], dst = (uint64_t)worker * S + sc.mnew[m];
             for (uint32_t f = lane; f < L4; f += 32) st4[dst * L4 + f] = st4[src * L4 + f];
         }
@@ -380,8 +419,55 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
     grid_leave(bar, G);
 }
 
+// Second half of a relocation that ran beside another call: the moving keys that call touched (flag[m] = 1) get
+// their rows moved and their table entries rewritten now that it is through.
+__global__ void __launch_bounds__(256)
+loc_deferred_kernel(LocScratch sc, uint2* table, float4* store, uint32_t worker, uint64_t S, uint32_t L4,
+                    const DevStatus* st, unsigned int epoch) {
+    if (call_failed(st, epoch) || st->deferred_now == 0u) return;
+    const uint32_t total = st->moved_total;
+    const int lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t m0 = warp * 32; m0 < total; m0 += n_warps * 32) {
+        const uint32_t m = m0 + lane;
+        const bool mine = m < total && sc.flag[m] != 0u;
+        unsigned todo = __ballot_sync(0xffffffffu, mine);
+        if (mine) table[sc.mkey[m]] = make_uint2(worker, sc.mnew[m]);
+        const uint64_t my_src = mine ? (uint64_t)sc.mowner[m] * S + sc.mslot[m] : 0;
+        const uint64_t my_dst = mine ? (uint64_t)worker * S + sc.mnew[m] : 0;
+        while (todo) {                                          // the warp moves the rows, four in flight at a time
+            int q[4];
+            uint64_t src[4], dst[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                q[a] = todo ? __ffs(todo) - 1 : -1;
+                todo &= todo - 1;                               // 0 stays 0
+                src[a] = __shfl_sync(0xffffffffu, my_src, q[a] & 31);
+                dst[a] = __shfl_sync(0xffffffffu, my_dst, q[a] & 31);
+            }
+            for (uint32_t f = lane; f < L4; f += 32) {
+                float4 x[4];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+                    if (q[a] >= 0) x[a] = store[src[a] * L4 + f];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+                    if (q[a] >= 0) store[dst[a] * L4 + f] = x[a];
+            }
+        }
+    }
+}
+
+void run_localize_deferred(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s) {
+    LocScratch sc = loc_scratch(ps);
+    const uint32_t grid = tmin<uint32_t>(div_up_u32(n, 256), (uint32_t)ps->sm_count * 8);
+    PS_LAUNCH(ps, loc_deferred_kernel, grid, 256, s, sc, ps->table, (float4*)ps->store, worker, ps->cfg.slots_per_part,
+              ps->cfg.row_len / 4, ps->status, ps->epoch);
+}
+
 // The call's keys (range-checked) have been sorted already; `which` says into which buffers.
-void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s) {
+void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s, const uint32_t* busy_keys,
+                  uint32_t n_busy) {
     LocScratch sc = loc_scratch(ps);
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     uint32_t* owner_keys = which ? ps->keysA : ps->keysB;    // the buffer the sorted keys are not in
@@ -406,9 +492,11 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
         unsigned int* bar = ps->sort_ctl + 2;                   // words 0 and 1 belong to the sort
         DevStatus* st = ps->status;
         unsigned int epoch = ps->epoch;
+        uint32_t part_size = div_up_u32(ps->cfg.num_keys, ps->cfg.num_workers);
         void* args[] = {(void*)&sk, (void*)&n, (void*)&span, (void*)&table, (void*)&worker, (void*)&N, (void*)&S, (void*)&K,
                         (void*)&tops, (void*)&stacks, (void*)&store, (void*)&row_bytes, (void*)&block_counts,
-                        (void*)&owner_counts, (void*)&sc, (void*)&bar, (void*)&st, (void*)&epoch};
+                        (void*)&owner_counts, (void*)&sc, (void*)&busy_keys, (void*)&n_busy, (void*)&part_size,
+                        (void*)&bar, (void*)&st, (void*)&epoch};
         if (ps->prof) prof_before(ps, "loc_fused_kernel", s);
         cudaLaunchCooperativeKernel((const void*)loc_fused_kernel, dim3(grid_f), dim3(256), args, kLocSmem, s);
         if (ps->prof) prof_after(ps, s);

@@ -48,6 +48,7 @@ WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys) {
     // localize in one launch: a count per block (at most 512 blocks), then one per block and partition (stores of
     // at most 1024 partitions; larger ones take the path that sorts by old owner)
     l.loc_counts = take((size_t)512 * 4 + (size_t)512 * (cfg.num_workers <= 1024 ? cfg.num_workers : 1) * 4);
+    l.loc_scratch = take(mk * 5 * 4);
     l.upd = take(mk * (row_bytes > 32 ? row_bytes : 32));
     l.carry = take(reduce_tiles * 2 * (size_t)cfg.row_len * 8);
     l.group_sum = take(groups * (size_t)cfg.row_len * 8);
@@ -150,6 +151,13 @@ static void alternate_side(ps_store* ps) {
 // Pipelined mode: it starts as soon as the buffer set's previous user is done, i.e. beside the previous
 // step's kernels; the batch arrays must then be complete when the call is made.
 static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_table = false) {
+    // for a relocation that may be asked to run beside this call (ps_localize_beside): everything earlier ends here
+    ss->sorted_which = -1;
+    if (cudaEventRecord(ps->ev_before, s) != cudaSuccess) return false;
+    if (ss->loc_reader) {                           // a relocation on another stream was reading this set's sorted keys
+        ss->loc_reader = false;
+        if (cudaStreamWaitEvent(ps->side, ps->ev_loc, 0) != cudaSuccess) return false;
+    }
     // When the caller's stream enters or leaves a CUDA-graph capture, events recorded on the other side of
     // that border cannot be waited on, and the side stream has to join (or leave) the capture: the first
     // call after such a change forks in ordered mode and forgets the older events.
@@ -177,6 +185,13 @@ static bool fork_side(ps_store* ps, SortSet* ss, cudaStream_t s, bool reads_tabl
 }
 static bool join_side(ps_store* ps, cudaStream_t s) {
     return cudaEventRecord(ps->ev_join, ps->side) == cudaSuccess && cudaStreamWaitEvent(s, ps->ev_join, 0) == cudaSuccess;
+}
+// after the call's sort has been enqueued on the side stream: where its sorted keys are, for ps_localize_beside
+static bool sorted_keys_at(ps_store* ps, SortSet* ss, int which, uint32_t n) {
+    ss->sorted_which = which;
+    ss->sorted_n = n;
+    ps->last_set = ss;
+    return cudaEventRecord(ps->ev_sorted, ps->side) == cudaSuccess;
 }
 // after the last kernel of a call that used the set
 static ps_status_t release_set(SortSet* ss, cudaStream_t s) {
@@ -256,6 +271,7 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
     next_set(ps);
     ps->scan_sums = (uint32_t*)(ps->ws + l.scan_sums);
     ps->loc_counts = (uint32_t*)(ps->ws + l.loc_counts);
+    ps->loc_scratch = (uint32_t*)(ps->ws + l.loc_scratch);
     ps->upd = (float*)(ps->ws + l.upd);
     ps->carry = (double*)(ps->ws + l.carry);
     ps->group_sum = (double*)(ps->ws + l.group_sum);
@@ -288,7 +304,10 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
             return PS_ERR_CUDA;
         }
     if (cudaEventCreateWithFlags(&ps->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&ps->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_before, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_sorted, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ps->ev_loc, cudaEventDisableTiming) != cudaSuccess) {
         delete ps;
         return PS_ERR_CUDA;
     }
@@ -318,6 +337,9 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     if (ps->prof) ps_profile_stop(ps, nullptr, 0);
     cudaEventDestroy(ps->ev_fork);
     cudaEventDestroy(ps->ev_join);
+    cudaEventDestroy(ps->ev_before);
+    cudaEventDestroy(ps->ev_sorted);
+    cudaEventDestroy(ps->ev_loc);
     for (int b = 0; b < kSortSets; ++b) cudaEventDestroy(ps->sets[b].ev_free);
     for (int b = 0; b < kSideStreams; ++b) cudaStreamDestroy(ps->sides[b]);
     cudaStreamDestroy(ps->copy);
@@ -329,9 +351,17 @@ ps_status_t ps_destroy(ps_store_t* ps) {
     return PS_OK;
 }
 
+// a relocation enqueued on another stream by ps_localize_beside comes before every later call of the handle
+static bool after_relocation(ps_store* ps, cudaStream_t s) {
+    ps->last_set = nullptr;
+    ps->last_stream = s;
+    return !ps->loc_pending || cudaStreamWaitEvent(s, ps->ev_loc, 0) == cudaSuccess;
+}
+
 #define PS_BEGIN_CALL(ps)                                            \
     if (!(ps)) return PS_ERR_INVALID_ARG;                           \
-    cudaStream_t s = (cudaStream_t)stream;
+    cudaStream_t s = (cudaStream_t)stream;                          \
+    if (!after_relocation(ps, s)) return PS_ERR_CUDA;
 
 ps_status_t ps_init_range_partition(ps_store_t* ps, void* stream) {
     PS_BEGIN_CALL(ps);
@@ -370,7 +400,7 @@ ps_status_t ps_push(ps_store_t* ps, const uint64_t* d_keys, uint64_t n, const fl
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;         // the keys are sorted beside earlier calls' kernels
     const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ps->side, ps->starter_count,
                                         div_up_u32(n, kGroupSpan));
-    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    if (!sorted_keys_at(ps, ss, which, (uint32_t)n) || !join_side(ps, s)) return PS_ERR_CUDA;
     run_push_reduce(ps, (uint32_t)n, which, d_updates, nullptr, 0, s);
     return release_set(ss, s);
 }
@@ -392,6 +422,65 @@ ps_status_t ps_localize(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys,
     return release_set(ss, s);
 }
 
+ps_status_t ps_localize_beside(ps_store_t* ps, uint32_t worker, const uint64_t* d_keys, uint64_t n, void* loc_stream) {
+    if (!ps) return PS_ERR_INVALID_ARG;
+    cudaStream_t ls = (cudaStream_t)loc_stream;
+    // Nothing to run beside (the most recent call sorted no keys, or was made on this very stream), or a store
+    // with more partitions than the one-launch relocation serves: an ordinary localize, after everything so far.
+    SortSet* busy = ps->last_set;
+    if (!busy || busy->sorted_which < 0 || ps->last_stream == ls || ps->cfg.num_workers > 1024) {
+        if (ps->last_stream != ls) {
+            if (cudaEventRecord(ps->ev_before, ps->last_stream) != cudaSuccess ||
+                cudaStreamWaitEvent(ls, ps->ev_before, 0) != cudaSuccess)
+                return PS_ERR_CUDA;
+        }
+        const cudaStream_t was = ps->last_stream;
+        const ps_status_t c = ps_localize(ps, worker, d_keys, n, loc_stream);
+        if (c != PS_OK || n == 0 || was == ls) return c;
+        if (cudaEventRecord(ps->ev_loc, ls) != cudaSuccess) return PS_ERR_CUDA;
+        ps->loc_pending = true;
+        return PS_OK;
+    }
+    if (worker >= ps->cfg.num_workers) return PS_ERR_WORKER_RANGE;
+    if (n == 0) return PS_OK;
+    if (!d_keys) return PS_ERR_INVALID_ARG;
+    if (n > ps->max_keys) return PS_ERR_WORKSPACE;
+    // an earlier relocation of this kind comes first; so does everything before the call to run beside, and that
+    // call's key sort, whose result says which keys it touches
+    if (ps->loc_pending && cudaStreamWaitEvent(ls, ps->ev_loc, 0) != cudaSuccess) return PS_ERR_CUDA;
+    if (cudaStreamWaitEvent(ls, ps->ev_before, 0) != cudaSuccess || cudaStreamWaitEvent(ls, ps->ev_sorted, 0) != cudaSuccess)
+        return PS_ERR_CUDA;
+    const uint32_t* busy_keys = busy->sorted_which ? busy->keysB : busy->keysA;
+    const uint32_t n_busy = busy->sorted_n;
+    const cudaEvent_t busy_done = busy->ev_free;
+    SortSet* ss = next_set(ps);
+    ss->sorted_which = -1;
+    const int which = radix_sort_keys64(ps, d_keys, (uint32_t)n, ls, nullptr, 0);
+    run_localize(ps, worker, (uint32_t)n, which, ls, busy_keys, n_busy);
+    if (cudaStreamWaitEvent(ls, busy_done, 0) != cudaSuccess) return PS_ERR_CUDA;
+    run_localize_deferred(ps, worker, (uint32_t)n, ls);
+    // (a later sort that reads the table forks after the caller's stream, which waits for ev_loc: table_dirty)
+    for (int b = 0; b < kSideStreams; ++b) ps->table_dirty[b] = true;
+    busy->loc_reader = true;
+    if (cudaEventRecord(ps->ev_loc, ls) != cudaSuccess) return PS_ERR_CUDA;
+    ps->loc_pending = true;
+    ps->last_set = nullptr;                         // (a second relocation beside the same call would have to wait for this one's deferred half)
+    return release_set(ss, ls);
+}
+
+ps_status_t ps_localize_stats(ps_store_t* ps, ps_localize_stats_t* h_out) {
+    if (!ps || !h_out) return PS_ERR_INVALID_ARG;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PS_ERR_CUDA;
+    DevStatus st;
+    if (cudaMemcpy(&st, ps->status, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
+    h_out->requested = st.loc_requested;
+    h_out->moved = st.rows_moved;
+    h_out->already_local = st.loc_already_local;
+    h_out->moved_again = st.loc_moved_again;
+    h_out->deferred = st.loc_deferred;
+    return PS_OK;
+}
+
 ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v, uint64_t n,
                        uint64_t col_key_base, float lr, float lambda, double* d_loss_accum, void* stream) {
     PS_BEGIN_CALL(ps);
@@ -410,6 +499,7 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     const bool by_column = fused && ps->mf_path == 1;
     const int which = radix_sort_mf(ps, d_i, d_j, d_v, (uint32_t)n, col_key_base, fused, ps->side, ps->starter_count,
                                     div_up_u32(2 * n, fused ? 64 * 8 : kGroupSpan));
+    if (!sorted_keys_at(ps, ss, which, (uint32_t)(2 * n))) return PS_ERR_CUDA;
     if (by_column) {
         launch_mf_plan(ps, (uint32_t)n, which, ps->side);
         if (!join_side(ps, s)) return PS_ERR_CUDA;
@@ -444,6 +534,7 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_kge(ps, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base, ps->side);
     const int which = run_push_sort(ps, occ, ps->side);
+    if (!sorted_keys_at(ps, ss, which, occ)) return PS_ERR_CUDA;
     // gradient rows + AdaGrad inside the reduction where a gradient row is whole float4s and fits the reduction's staging
     const bool grad_only = dim_complex % 2 == 0 && dim_complex <= 128;
     const uint32_t lb = launch_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim_complex,
@@ -478,6 +569,7 @@ ps_status_t ps_step_sgns(ps_store_t* ps, const uint32_t* d_tokens, uint64_t firs
     if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
     launch_keys_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg, out_key_base, ps->side);
     const int which = run_push_sort(ps, (uint32_t)occ, ps->side);
+    if (!sorted_keys_at(ps, ss, which, (uint32_t)occ)) return PS_ERR_CUDA;
     const uint32_t lb = launch_step_sgns(ps, d_tokens, 0, first_pos, n_centers, corpus_len, window, d_negs, n_neg,
                                          out_key_base, lr, s);
     if (!join_side(ps, s)) return PS_ERR_CUDA;
@@ -607,6 +699,7 @@ ps_status_t ps_step_sgns_host(ps_store_t* ps, const uint32_t* h_tokens, uint64_t
     if (tok_first > need_lo || tok_first + tok_count <= need_hi) return PS_ERR_INVALID_ARG;
     if ((tok_count + n_negs) * 4 > ps->max_keys * 8) return PS_ERR_WORKSPACE;
     cudaStream_t s = (cudaStream_t)stream;
+    if (!after_relocation(ps, s)) return PS_ERR_CUDA;
     HostBatch hb;
     if (!host_batch_begin(ps, s, &hb)) return PS_ERR_CUDA;
     uint32_t* d_tok = (uint32_t*)hb.buf;
@@ -687,6 +780,10 @@ ps_status_t ps_sync(ps_store_t* ps, void* stream) {
     if (!ps) return PS_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaStreamSynchronize(s) != cudaSuccess) return PS_ERR_CUDA;
+    if (ps->loc_pending) {                          // a relocation on another stream belongs to what this call waits for
+        if (cudaEventSynchronize(ps->ev_loc) != cudaSuccess) return PS_ERR_CUDA;
+        ps->loc_pending = false;
+    }
     unsigned int code = 0;
     if (cudaMemcpy(&code, &ps->status->sticky, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return PS_ERR_CUDA;
     if (code != 0 && cudaMemset(&ps->status->sticky, 0, 4) != cudaSuccess) return PS_ERR_CUDA;

@@ -33,7 +33,13 @@ struct DevStatus {
                                     // (up to kSortSets such calls of one handle are in flight: later ones' sorts
                                     // beside the current one's kernels; only calls that take a buffer set are numbered)
     unsigned int moved_total;       // localize: number of keys that move in the current call
+    unsigned int deferred_now;      // ... of which wait for the call that runs beside the relocation (ps_localize_beside)
     unsigned long long rows_moved;  // rows relocated by all successful localize calls so far
+    unsigned long long loc_requested;       // keys handed to localize calls, repeats included
+    unsigned long long loc_already_local;   // distinct keys per call that the requester owned already
+    unsigned long long loc_moved_again;     // moved keys that had left their initial partition before (taken from a
+                                            // worker that had localized them: localization conflicts, Section 3.2)
+    unsigned long long loc_deferred;        // moved keys that had to wait for the call running beside the relocation
 };
 
 static_assert(kSortSets <= 4, "one error-epoch word per call in flight");
@@ -55,6 +61,9 @@ struct SortSet {
     unsigned int* mf_tickets;
     cudaEvent_t ev_free;            // recorded after the last kernel that used the set
     bool used;
+    bool loc_reader;                // a relocation on another stream reads this set's sorted keys (ps_localize_beside)
+    int sorted_which;               // which key buffer holds the call's sorted keys (-1: the call sorted none)
+    uint32_t sorted_n;
 };
 
 }  // namespace psb
@@ -85,6 +94,7 @@ struct ps_store {
     double* group_sum;              // per group: pre-added parked parts of the segment entering it (row_len)
     uint32_t* scan_sums;            // block sums of the device-wide scan
     uint32_t* loc_counts;           // localize: moving keys per block (512 words), then per block and old owner
+    uint32_t* loc_scratch;          // localize: five words per key of the call (old and new places of the moving keys)
     float* upd;                     // max_keys x row_len update rows (also localize scratch)
     double* carry;                  // nReduceTiles x 2 x row_len partial sums of segments that span tiles
     uint4* starters;                // {tile, key, row} of the tiles that start a border-crossing segment
@@ -113,6 +123,11 @@ struct ps_store {
     cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
     int mf_path;                    // see ps_set_mf_path
+    psb::SortSet* last_set;         // the most recent call's buffer set if that call sorted its keys (else null)
+    cudaStream_t last_stream;       // the stream of the most recent call
+    cudaEvent_t ev_before, ev_sorted;       // most recent sorting call: the caller's stream before its first kernel; after its sort
+    cudaEvent_t ev_loc;             // end of the most recent ps_localize_beside
+    bool loc_pending;               // ... which later calls still have to be ordered after
     int push_mode;                  // see ps_set_push_mode
     bool table_dirty[psb::kSideStreams];   // per side stream: the location table was rewritten since that stream last waited
                                     // for the caller's (a sort that reads the table must not start before the rewrite)
@@ -123,7 +138,7 @@ namespace psb {
 
 struct WsLayout {
     size_t status, keysA[kSortSets], keysB[kSortSets], valsA[kSortSets], valsB[kSortSets], tile_state[kSortSets],
-        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], mf_dup[kSortSets], mf_tickets[kSortSets], scan_sums, loc_counts, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
+        sort_ctl[kSortSets], rec[kSortSets], cellpos[kSortSets], mf_dup[kSortSets], mf_tickets[kSortSets], scan_sums, loc_counts, loc_scratch, upd, carry, group_sum, starters[kSortSets], starter_count[kSortSets],
         loss_partial, apply_rows, staging[kHostStages], total;
 };
 WsLayout ws_layout(const ps_config_t& cfg, uint64_t max_keys);
@@ -218,7 +233,11 @@ void run_kge_reduce(ps_store* ps, uint32_t n, int which, uint32_t dim, float lr,
                     uint32_t loss_blocks, cudaStream_t s);
 
 // ---- localize.cu ----
-void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s);
+// busy_keys: sorted keys of a call that may run beside this relocation (null: none); moving keys among them keep
+// table entry and row until run_localize_deferred, which the caller enqueues once that call is through.
+void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStream_t s,
+                  const uint32_t* busy_keys = nullptr, uint32_t n_busy = 0);
+void run_localize_deferred(ps_store* ps, uint32_t worker, uint32_t n, cudaStream_t s);
 
 // ---- steps.cu ----
 // launch_keys_* write the keys of a batch's occurrence slots to keysA (they depend on the batch
