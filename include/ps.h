@@ -327,6 +327,46 @@ ps_status_t ps_rows_moved(ps_store_t* ps, uint64_t* h_out);
 ps_status_t ps_profile_start(ps_store_t* ps, uint32_t max_launches);
 ps_status_t ps_profile_stop(ps_store_t* ps, char* h_report, size_t capacity);
 
+/* One epoch of matrix factorization under parameter blocking (Section 2.2 "parameter blocking", Section 4.1,
+ * Appendix A: the schedule of distributed SGD).  The handle's N workers split the rows into N contiguous blocks of
+ * ceil(rows / N) and the columns into N blocks of ceil(cols / N); worker w keeps row block w for the whole
+ * epoch (its row factors are localized to it first); the epoch has N subepochs; in subepoch s worker w localizes
+ * the column factors of block (w + s) mod N and then runs minibatches of `batch` cells (ps_step_mf) over the
+ * cells of (row block w, that column block).  Within a subepoch no two workers touch a common parameter; stream
+ * order is the barrier between subepochs.
+ * The cells must be grouped by stratum: h_offsets (host, N * N + 1 entries) gives for stratum (s, w), at index
+ * s * N + w, the range [h_offsets[x], h_offsets[x + 1]) of its cells in d_i, d_j, d_v.  Key i is row factor i,
+ * key rows + j column factor j; rows + cols = num_keys.  Every partition needs room for its row block, its column
+ * block and the keys still on their way out (slots_per_part of 1.5 times the initial partition size suffices for
+ * the initial range partition).  Enqueues on `stream`; errors as for ps_localize and ps_step_mf. */
+ps_status_t ps_dsgd_epoch_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
+                             const uint64_t* h_offsets, uint64_t rows, uint64_t cols, uint64_t batch, float lr,
+                             float lambda, double* d_loss_accum, void* stream);
+
+/* ---- sparse-map front end (Section 3.7: a server keeps its parameters "in dense arrays or sparse maps") ----
+ * Translates arbitrary 64-bit keys into the dense keys 0 .. capacity-1 that every call above takes, so that a
+ * store created with num_keys = capacity serves non-contiguous keys.  A key gets the next unused dense key the
+ * first time it is seen; within one call new keys are numbered in order of first occurrence, so the translation
+ * is reproducible by a sequential program.  The key with all 64 bits set is reserved.
+ * The map lives in caller-allocated device memory (256-byte aligned) of ps_keymap_query_bytes bytes; calls of up
+ * to max_batch_keys keys.  ps_keymap_create enqueues the clearing of that memory on `stream`.
+ *   ps_keymap_insert   d_dense[t] = dense key of d_sparse[t], adding unseen keys.  A call that would exceed the
+ *                      capacity adds nothing, writes all ones to d_dense and latches PS_ERR_CAPACITY; a call that
+ *                      holds the reserved key adds nothing and latches PS_ERR_KEY_RANGE.
+ *   ps_keymap_lookup   the same without adding: all ones for a key that was never inserted.
+ *   ps_keymap_sync     waits for `stream`, returns and clears the latched code; *h_size (may be NULL) = dense keys
+ *                      handed out so far.  After a failed insert, sync before the next insert.
+ * Calls on one map are ordered by the caller (one stream, or events). */
+typedef struct ps_keymap ps_keymap_t;
+ps_status_t ps_keymap_query_bytes(uint64_t capacity, uint64_t max_batch_keys, size_t* out);
+ps_status_t ps_keymap_create(uint64_t capacity, uint64_t max_batch_keys, void* d_mem, size_t bytes, int32_t device,
+                             void* stream, ps_keymap_t** out);
+ps_status_t ps_keymap_destroy(ps_keymap_t* map);
+ps_status_t ps_keymap_insert(ps_keymap_t* map, const uint64_t* d_sparse, uint64_t n, uint64_t* d_dense, void* stream);
+ps_status_t ps_keymap_lookup(ps_keymap_t* map, const uint64_t* d_sparse, uint64_t n, uint64_t* d_dense, void* stream);
+ps_status_t ps_keymap_sync(ps_keymap_t* map, void* stream, uint64_t* h_size);
+uint64_t ps_keymap_launch_count(const ps_keymap_t* map);
+
 const char* ps_status_string(ps_status_t status);
 
 #ifdef __cplusplus

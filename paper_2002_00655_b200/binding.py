@@ -76,6 +76,14 @@ SIGNATURES = {
     "ps_rows_moved": (C.c_int, [_vp, C.POINTER(_u64)]),
     "ps_profile_start": (C.c_int, [_vp, _u32]),
     "ps_profile_stop": (C.c_int, [_vp, C.c_char_p, _sz]),
+    "ps_dsgd_epoch_mf": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _u64, _u64, _u64, _f32, _f32, _vp, _vp]),
+    "ps_keymap_query_bytes": (C.c_int, [_u64, _u64, C.POINTER(_sz)]),
+    "ps_keymap_create": (C.c_int, [_u64, _u64, _vp, _sz, C.c_int32, _vp, C.POINTER(_vp)]),
+    "ps_keymap_destroy": (C.c_int, [_vp]),
+    "ps_keymap_insert": (C.c_int, [_vp, _vp, _u64, _vp, _vp]),
+    "ps_keymap_lookup": (C.c_int, [_vp, _vp, _u64, _vp, _vp]),
+    "ps_keymap_sync": (C.c_int, [_vp, _vp, C.POINTER(_u64)]),
+    "ps_keymap_launch_count": (C.c_uint64, [_vp]),
     "ps_status_string": (C.c_char_p, [C.c_int]),
 }
 
@@ -306,6 +314,86 @@ def ps_profile_stop(ps) -> dict:
 
 def ps_status_string(code: int) -> str:
     return load_library().ps_status_string(code).decode()
+
+
+def ps_dsgd_epoch_mf(ps, d_i, d_j, d_v, h_offsets, rows, cols, batch, lr, lam, d_loss_accum=None):
+    """h_offsets: CPU int64 tensor of N * N + 1 stratum boundaries."""
+    _check(load_library().ps_dsgd_epoch_mf(ps, _dptr(d_i, _U32), _dptr(d_j, _U32), _dptr(d_v, _F32), _hptr(h_offsets, _U64),
+                                           rows, cols, batch, lr, lam, _dptr(d_loss_accum, _F64), _stream()),
+           "ps_dsgd_epoch_mf")
+
+
+def ps_keymap_query_bytes(capacity: int, max_batch_keys: int) -> int:
+    out = _sz(0)
+    _check(load_library().ps_keymap_query_bytes(capacity, max_batch_keys, C.byref(out)), "ps_keymap_query_bytes")
+    return out.value
+
+
+def ps_keymap_create(capacity: int, max_batch_keys: int, d_mem, device: int = 0):
+    h = _vp()
+    _check(load_library().ps_keymap_create(capacity, max_batch_keys, _dptr(d_mem), d_mem.numel() * d_mem.element_size(),
+                                           device, _stream(), C.byref(h)), "ps_keymap_create")
+    return h
+
+
+def ps_keymap_destroy(m):
+    _check(load_library().ps_keymap_destroy(m), "ps_keymap_destroy")
+
+
+def ps_keymap_insert(m, d_sparse, d_dense):
+    _check(load_library().ps_keymap_insert(m, _dptr(d_sparse, _U64), d_sparse.numel(), _dptr(d_dense, _U64), _stream()),
+           "ps_keymap_insert")
+
+
+def ps_keymap_lookup(m, d_sparse, d_dense):
+    _check(load_library().ps_keymap_lookup(m, _dptr(d_sparse, _U64), d_sparse.numel(), _dptr(d_dense, _U64), _stream()),
+           "ps_keymap_lookup")
+
+
+def ps_keymap_sync(m):
+    """(latched status code, number of dense keys handed out so far)."""
+    size = _u64(0)
+    code = load_library().ps_keymap_sync(m, _stream(), C.byref(size))
+    return code, size.value
+
+
+def ps_keymap_launch_count(m) -> int:
+    return load_library().ps_keymap_launch_count(m)
+
+
+class KeyMap:
+    """A sparse-key map whose device memory is a torch tensor (memory only)."""
+
+    def __init__(self, capacity: int, max_batch_keys: int = 1 << 20, device: int = 0):
+        self.device = torch.device("cuda", device)
+        n = ps_keymap_query_bytes(capacity, max_batch_keys)
+        with torch.cuda.device(self.device):
+            self.mem = torch.empty((n + 7) // 8, dtype=torch.int64, device=self.device)
+            self.h = ps_keymap_create(capacity, max_batch_keys, self.mem, device)
+
+    def insert(self, sparse):
+        out = torch.empty(sparse.numel(), dtype=torch.int64, device=self.device)
+        ps_keymap_insert(self.h, sparse, out)
+        return out
+
+    def lookup(self, sparse):
+        out = torch.empty(sparse.numel(), dtype=torch.int64, device=self.device)
+        ps_keymap_lookup(self.h, sparse, out)
+        return out
+
+    def sync(self):
+        return ps_keymap_sync(self.h)
+
+    def close(self):
+        if getattr(self, "h", None):
+            ps_keymap_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 # ---- convenience: torch-owned buffers around one handle -------------------------------

@@ -545,6 +545,65 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     return release_set(ss, s);
 }
 
+// ---- parameter blocking for matrix factorization ----
+__global__ void key_range_kernel(uint64_t* out, uint64_t first, uint64_t n) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n) out[t] = first + t;
+}
+
+// localize(worker, keys first .. first + count), in pieces the workspace has room for
+static ps_status_t localize_range(ps_store* ps, uint32_t worker, uint64_t first, uint64_t count, void* stream) {
+    cudaStream_t s = (cudaStream_t)stream;
+    uint64_t* d_keys = (uint64_t*)ps->stagings[0];
+    for (uint64_t done = 0; done < count;) {
+        const uint64_t c = tmin<uint64_t>(count - done, ps->max_keys);
+        key_range_kernel<<<div_up_u32(c, 256), 256, 0, s>>>(d_keys, first + done, c);
+        ps->launches++;
+        const ps_status_t rc = ps_localize(ps, worker, d_keys, c, stream);
+        if (rc != PS_OK) return rc;
+        done += c;
+    }
+    return PS_OK;
+}
+
+ps_status_t ps_dsgd_epoch_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
+                             const uint64_t* h_offsets, uint64_t rows, uint64_t cols, uint64_t batch, float lr,
+                             float lambda, double* d_loss_accum, void* stream) {
+    if (!ps || !d_i || !d_j || !d_v || !h_offsets || batch == 0) return PS_ERR_INVALID_ARG;
+    const uint64_t N = ps->cfg.num_workers;
+    if (rows == 0 || cols == 0 || rows + cols != ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    for (uint64_t x = 0; x < N * N; ++x)
+        if (h_offsets[x] > h_offsets[x + 1]) return PS_ERR_INVALID_ARG;
+    const uint64_t rsize = (rows + N - 1) / N, csize = (cols + N - 1) / N;
+    // The key lists of the relocations are written on the caller's stream right before use: their sorts must
+    // not start ahead of that, so the relocations run in ordered mode whatever the handle is set to.
+    const bool was = ps->pipelined;
+    ps_status_t rc = PS_OK;
+    ps->pipelined = false;
+    for (uint64_t w = 0; w < N && rc == PS_OK; ++w)            // a worker's row factors live with it throughout
+        if (w * rsize < rows) rc = localize_range(ps, (uint32_t)w, w * rsize, tmin<uint64_t>(rsize, rows - w * rsize), stream);
+    for (uint64_t sub = 0; sub < N && rc == PS_OK; ++sub) {
+        // subepoch start: worker w localizes column block (w + sub) mod N (stream order is the barrier between subepochs)
+        ps->pipelined = false;
+        for (uint64_t w = 0; w < N && rc == PS_OK; ++w) {
+            const uint64_t blk = (w + sub) % N;
+            if (blk * csize < cols)
+                rc = localize_range(ps, (uint32_t)w, rows + blk * csize, tmin<uint64_t>(csize, cols - blk * csize), stream);
+        }
+        ps->pipelined = was;
+        // the workers' strata: no two of them share a parameter, so their minibatches are independent
+        for (uint64_t w = 0; w < N && rc == PS_OK; ++w) {
+            const uint64_t lo = h_offsets[sub * N + w], hi = h_offsets[sub * N + w + 1];
+            for (uint64_t at = lo; at < hi && rc == PS_OK; at += batch) {
+                const uint64_t c = tmin<uint64_t>(batch, hi - at);
+                rc = ps_step_mf(ps, d_i + at, d_j + at, d_v + at, c, rows, lr, lambda, d_loss_accum, stream);
+            }
+        }
+    }
+    ps->pipelined = was;
+    return rc;
+}
+
 static ps_status_t sgns_checks(ps_store_t* ps, uint64_t first_pos, uint64_t n_centers, uint64_t corpus_len,
                                uint32_t window, uint32_t n_neg, uint64_t out_key_base, uint64_t* occ) {
     if (first_pos + n_centers > corpus_len) return PS_ERR_INVALID_ARG;

@@ -163,6 +163,22 @@ def mf_cells(cfg: MFConfig, planted, start: int, count: int, device, chunk: int 
     return i_out, j_out, v_out
 
 
+def mf_stratify(i, j, v, rows: int, cols: int, n_workers: int):
+    """Groups cells by stratum for the parameter-blocking schedule: stratum (s, w) holds the cells of row block w and
+    column block (w + s) mod N (blocks are contiguous ranges of ceil(count / N)), strata in (s, w) order, the cells of
+    a stratum in their input order.  Returns i, j, v regrouped and the N * N + 1 stratum boundaries (CPU int64)."""
+    N = n_workers
+    rb = i.to(torch.int64) // (-(-rows // N))
+    cb = j.to(torch.int64) // (-(-cols // N))
+    sub = (cb - rb) % N
+    stratum = sub * N + rb
+    order = torch.sort(stratum, stable=True).indices
+    counts = torch.bincount(stratum, minlength=N * N)
+    offsets = torch.zeros(N * N + 1, dtype=torch.int64)
+    offsets[1:] = torch.cumsum(counts, 0).cpu()
+    return i[order].contiguous(), j[order].contiguous(), v[order].contiguous(), offsets
+
+
 # --------------------------------------------------------------------------
 # ComplEx knowledge-graph embeddings
 # --------------------------------------------------------------------------
