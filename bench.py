@@ -328,6 +328,132 @@ class MFPushWorkload(MFWorkload):
         return None
 
 
+class MFDsgdWorkload(MFWorkload):
+    """Matrix factorization under parameter blocking (Section 2.2, Appendix A): ps_dsgd_epoch_mf with 8 workers.
+    One timed repeat is ONE call over the cells of its steps (an epoch over that sample: the row blocks are
+    localized once, the column blocks once per subepoch, then the minibatches of every stratum)."""
+
+    WORKERS = 8
+    graph_ok = False
+
+    def describe(self):
+        return dict(super().describe(), workload=self.cfg.name + "_dsgd", workers=self.WORKERS,
+                    schedule="ps_dsgd_epoch_mf: 8 x 8 strata, one call per timed repeat over the repeat's cells")
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c, N = self.cfg, self.WORKERS
+        self.ps = ps
+        slots = -(-c.num_keys // N) + -(-c.rows // N) + -(-c.cols // N)      # initial keys + a row block + a column block
+        self.store = ps.Store(c.num_keys, c.rank, N, slots, max_batch_keys=max(2 * c.batch, 1 << 18),
+                              device=device.index)
+        for s, rows in self.gen_init(device):
+            self.store.set_rows(torch.arange(s, s + rows.shape[0], dtype=torch.int64, device=device), rows)
+        self.host_init = None
+        planted = W.mf_planted(c, device)
+        self.i, self.j, self.v = W.mf_cells(c, planted, 0, n_steps * c.batch, device)
+        del planted
+        self.grouped = {}
+        torch.cuda.synchronize(device)
+
+    def run_steps(self, ks):
+        c, b = self.cfg, self.cfg.batch
+        key = (ks[0], len(ks))
+        if key not in self.grouped:                             # regrouping the cells by stratum is input preparation
+            sl = slice(ks[0] * b, (ks[-1] + 1) * b)
+            self.grouped[key] = W.mf_stratify(self.i[sl], self.j[sl], self.v[sl], c.rows, c.cols, self.WORKERS)
+            torch.cuda.synchronize()
+        gi, gj, gv, off = self.grouped[key]
+        self.ps.ps_dsgd_epoch_mf(self.store.h, gi, gj, gv, off, c.rows, c.cols, b, c.lr, c.lam, self.store.loss)
+
+    def prepare(self, chunks):
+        for ch in chunks:
+            c, b = self.cfg, self.cfg.batch
+            sl = slice(ch[0] * b, (ch[-1] + 1) * b)
+            self.grouped[(ch[0], len(ch))] = W.mf_stratify(self.i[sl], self.j[sl], self.v[sl], c.rows, c.cols, self.WORKERS)
+        torch.cuda.synchronize()
+
+    def host_setup(self, steps):
+        return None
+
+    def kernel_bytes(self, k, moved=0.0):
+        kb = super().kernel_bytes(k, moved)
+        c, rb = self.cfg, self.row_bytes
+        # per step: the relocations' share (rows moved per step from the device counter; keys and table entries in)
+        kb["loc_fused_kernel"] = None
+        kb["key_range_kernel"] = None
+        return kb
+
+    def oracle_setup(self, device):
+        return None
+
+
+class KeyMapWorkload:
+    """A store behind the sparse-map front end (Section 3.7): per step the batch's sparse 64-bit keys are
+    translated (ps_keymap_insert: known keys are found, unseen ones added) and the rows pulled by dense key."""
+
+    def __init__(self, cfg):
+        self.cfg, self.example = cfg, "keys"
+        self.row_bytes = cfg.row_len * 4
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": "keymap_" + c.name, "keys": c.num_keys, "row_len": c.row_len, "batch_keys": c.batch,
+                "store_gb": round(c.num_keys * c.row_len * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def max_steps(self):
+        return min(self.cfg.n_batches, 400)
+
+    def side_stream_kernels(self):
+        return ()
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        self.store = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=c.batch, device=device.index)
+        self.map = ps.KeyMap(c.num_keys, max_batch_keys=c.batch, device=device.index)
+        # a sparse name per dense key of the generator: an odd multiplier makes a bijection on 64 bits
+        self.keys = [(W.stress_keys(c, k, device) * 0x9E3779B97F4A7C15 + 12345) for k in range(n_steps)]
+        self.dense = torch.empty(c.batch, dtype=torch.int64, device=device)
+        self.out = torch.empty((c.batch, c.row_len), dtype=torch.float32, device=device)
+        torch.cuda.synchronize(device)
+
+    def units(self, k):
+        return self.cfg.batch
+
+    def step(self, k):
+        self.ps.ps_keymap_insert(self.map.h, self.keys[k], self.dense)
+        self.ps.ps_pull(self.store.h, self.dense, self.out)
+
+    def host_setup(self, steps):
+        return None
+
+    def alg_bytes(self, k):
+        n, rb = self.cfg.batch, self.row_bytes
+        return n * (8 + 16 + 8) + n * (16 + 2 * rb)             # key in, slot (key word + value word) read, dense key out; then the pull
+
+    def kernel_bytes(self, k, moved=0.0):
+        n, rb = self.cfg.batch, self.row_bytes
+        return {"map_insert_kernel": n * (8 + 16 + 8 + 8), "pull_bulk_kernel": n * (16 + 2 * rb)}
+
+    def extra_profile(self):
+        """The map's kernels are not launched through the store handle: time them here, alone, with CUDA events."""
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        us = []
+        for k in range(5):
+            torch.cuda.synchronize()
+            a.record()
+            self.ps.ps_keymap_insert(self.map.h, self.keys[k], self.dense)
+            b.record()
+            torch.cuda.synchronize()
+            us.append(a.elapsed_time(b) * 1e3)
+        n = getattr(self, "_prof_steps", 1)
+        return {"map_insert_kernel": (n, float(np.median(us)) * n)}
+
+    def oracle_setup(self, device):
+        return None
+
+
 class KGEWorkload:
     """ComplEx + AdaGrad (Section 4.1 / Appendix A task): triples/s through ps_step_kge."""
 
@@ -691,7 +817,9 @@ class StressWorkload:
 
 
 def make_workload(name):
-    table = {"push_mf": lambda: MFPushWorkload(W.MF_LARGE), "mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
+    table = {"mf_dsgd": lambda: MFDsgdWorkload(W.MF_LARGE), "mf_medium_dsgd": lambda: MFDsgdWorkload(W.MF_MEDIUM),
+             "keymap": lambda: KeyMapWorkload(W.STRESS_MEDIUM),
+             "push_mf": lambda: MFPushWorkload(W.MF_LARGE), "mf_large": lambda: MFWorkload(W.MF_LARGE), "mf_tiny": lambda: MFWorkload(W.MF_TINY),
              "mf_medium": lambda: MFWorkload(W.MF_MEDIUM),
              "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
              "kge_4000": lambda: KGEWorkload(W.KGE_4000, twin=W.KGE_4000_TWIN),
@@ -805,11 +933,17 @@ def run_ours(args):
         if args.prelocalize == "beside":
             wl.graph_ok = False                                 # two caller streams: the calls are issued eagerly
 
-    for k in range(args.warmup):
-        wl.step(k)
+    if hasattr(wl, "run_steps"):
+        wl.run_steps(list(range(args.warmup)))
+    else:
+        for k in range(args.warmup):
+            wl.step(k)
     torch.cuda.synchronize(device)
     # repeat r works on steps chunks[r]; chunk 0 is run once untimed (first launch of the graphs, caches, clocks)
     chunks = [list(range(args.warmup + r * steps, args.warmup + (r + 1) * steps)) for r in range(repeats + 1)]
+    if hasattr(wl, "prepare"):
+        wl.prepare(chunks)
+    wl._prof_steps = prof_steps
     # The launch-bound loop of steps is captured into CUDA graphs (one per repeat, every step with its own batch
     # pointers) and each is replayed with one launch; --no-graph issues the calls one by one instead.
     graphs = None
@@ -830,6 +964,8 @@ def run_ours(args):
     def run_chunk(r):
         if graphs is not None:
             return timed_loop(lambda _k: graphs[r].replay(), [0], device, world)
+        if hasattr(wl, "run_steps"):                            # a call that takes a whole run of steps (an epoch schedule)
+            return timed_loop(lambda _k: wl.run_steps(chunks[r]), [0], device, world)
         return timed_loop(wl.step, chunks[r], device, world)
 
     run_chunk(0)                                                # untimed
@@ -884,10 +1020,16 @@ def run_ours(args):
 
     # per-kernel times from event pairs around every launch (a separate, untimed pass)
     launches_a = ps.ps_launch_count(h)
-    ps.ps_profile_start(h, 64 * prof_steps + 64)
-    for k in chunks[1][:prof_steps]:
-        wl.step(k)
+    if hasattr(wl, "run_steps"):
+        prof_steps = steps
+    ps.ps_profile_start(h, 64 * prof_steps + 4096)
+    if hasattr(wl, "run_steps"):
+        wl.run_steps(chunks[1])
+    else:
+        for k in chunks[1][:prof_steps]:
+            wl.step(k)
     prof = ps.ps_profile_stop(h)
+    prof.update(wl.extra_profile() if hasattr(wl, "extra_profile") else {})
     launches_per_step = (ps.ps_launch_count(h) - launches_a) / prof_steps
     tot_us = sum(us for _, us in prof.values()) or 1.0
     kb = {}
@@ -1010,7 +1152,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mf_large",
-                    choices=["push_mf", "mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "kge_4000", "sgns", "sgns_tiny", "stress", "stress_tiny",
+                    choices=["mf_dsgd", "mf_medium_dsgd", "keymap", "push_mf", "mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "kge_4000", "sgns", "sgns_tiny", "stress", "stress_tiny",
                              "stress_medium"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--repeats", type=int, default=0,

@@ -336,9 +336,9 @@ ps_status_t ps_profile_stop(ps_store_t* ps, char* h_report, size_t capacity);
  * order is the barrier between subepochs.
  * The cells must be grouped by stratum: h_offsets (host, N * N + 1 entries) gives for stratum (s, w), at index
  * s * N + w, the range [h_offsets[x], h_offsets[x + 1]) of its cells in d_i, d_j, d_v.  Key i is row factor i,
- * key rows + j column factor j; rows + cols = num_keys.  Every partition needs room for its row block, its column
- * block and the keys still on their way out (slots_per_part of 1.5 times the initial partition size suffices for
- * the initial range partition).  Enqueues on `stream`; errors as for ps_localize and ps_step_mf. */
+ * key rows + j column factor j; rows + cols = num_keys.  A partition holds at most the keys it started with, its
+ * row block and one column block: slots_per_part >= ceil(K / N) + ceil(rows / N) + ceil(cols / N) always suffices.
+ * Enqueues on `stream`; errors as for ps_localize and ps_step_mf. */
 ps_status_t ps_dsgd_epoch_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j, const float* d_v,
                              const uint64_t* h_offsets, uint64_t rows, uint64_t cols, uint64_t batch, float lr,
                              float lambda, double* d_loss_accum, void* stream);
