@@ -153,13 +153,14 @@ loc_apply_kernel(const uint32_t* __restrict__ so, const uint32_t* __restrict__ s
 //   phase 2a  every block adds up the block counts (its own offset m0 among the moving keys, and the call's
 //             total: the capacity check, the same decision in every block); the m-th moving key takes the m-th
 //             slot from the top of the requester's stack, its old location is noted, its table entry rewritten;
-//             old owners are counted per block                                           -> arrive at barrier 2
-//   phase 2b  the block's rows travel old slot -> shared memory -> new slot as bulk asynchronous copies of
-//             whole rows, several rounds in flight per warp, while the other blocks arrive
-//   phase 3   (after barrier 2) per old owner: keys that leave it in earlier blocks = where this block's
-//             vacated slots go on that owner's stack; one warp ranks the block's keys per owner in key order
-//             (warp match, running counters in shared memory: stable) and pushes the vacated slots; the last
-//             block writes the new stack heights (every block read the old ones before barrier 2).
+//             old owners are counted per block                                           -> grid barrier 2
+//   phase 3   per old owner: keys that leave it in earlier blocks = where this block's vacated slots go on that
+//             owner's stack; one warp ranks the block's keys per owner in key order (warp match, running
+//             counters in shared memory: stable) and pushes the vacated slots; the last block writes the new
+//             stack heights (every block read the old ones before barrier 2)
+//   rows      every block moves an equal share of ALL moving keys (the spans hold very different numbers of
+//             them): old slot -> shared memory -> new slot as bulk asynchronous copies of whole rows, several
+//             rounds in flight per warp.
 // No second sort, no flag array, two grid barriers instead of four launches with four.
 constexpr uint32_t kLocFastWorkers = 1024;          // partitions the per-block owner counters have room for
 constexpr uint32_t kLocMaxGrid = 512;
@@ -193,8 +194,30 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         return table[key].x != worker;
     };
     // ---- phase 1 ----
+    // The first kKeep tiles of the span (all of it unless the call is very large) are looked at with every load of
+    // a kind in flight at once, and what was read (key, table entry) stays in registers for phase 2a.
+    constexpr int kKeep = 2;
+    uint32_t k_key[kKeep];
+    uint2 k_ent[kKeep];
+    bool k_first[kKeep];
+#pragma unroll
+    for (int q = 0; q < kKeep; ++q) {
+        const uint32_t pos = lo + q * 256 + tid;
+        k_key[q] = pos < hi ? sk[pos] : kSentinelPad;
+        const uint32_t before_it = (pos < hi && pos > 0) ? sk[pos - 1] : kSentinelPad;
+        k_first[q] = pos < hi && k_key[q] < K && (pos == 0 || before_it != k_key[q]);
+    }
+#pragma unroll
+    for (int q = 0; q < kKeep; ++q) k_ent[q] = k_first[q] ? table[k_key[q]] : make_uint2(worker, 0u);
     uint32_t cnt = 0, n_local = 0;
-    for (uint32_t t0 = lo; t0 < hi; t0 += 256) {
+#pragma unroll
+    for (int q = 0; q < kKeep; ++q) {
+        if (lo + q * 256 >= hi) break;
+        const bool mv = k_first[q] && k_ent[q].x != worker;
+        cnt += (uint32_t)__syncthreads_count(mv);
+        n_local += (uint32_t)__syncthreads_count(k_first[q] && !mv);
+    }
+    for (uint32_t t0 = lo + kKeep * 256; t0 < hi; t0 += 256) {
         const uint32_t pos = t0 + tid;
         const bool mv = must_move(pos);
         const bool first = pos < hi && sk[pos] < K && (pos == 0 || sk[pos - 1] != sk[pos]);
@@ -237,13 +260,23 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
     __syncthreads();
     uint32_t running = 0;
     for (uint32_t t0 = lo; t0 < hi; t0 += 256) {
-        const bool f = must_move(t0 + tid);
+        const uint32_t q = (t0 - lo) >> 8;
+        bool f;
+        uint32_t key = 0;
+        uint2 e = make_uint2(0u, 0u);
+        if (q == 0) { f = k_first[0] && k_ent[0].x != worker; key = k_key[0]; e = k_ent[0]; }
+        else if (q == 1) { f = k_first[1] && k_ent[1].x != worker; key = k_key[1]; e = k_ent[1]; }
+        else {
+            f = must_move(t0 + tid);
+            if (f) {
+                key = sk[t0 + tid];
+                e = table[key];
+            }
+        }
         uint32_t tot;
         const uint32_t ex = block_exclusive_scan_256(f ? 1u : 0u, sm, &tot);
         if (f) {
-            const uint32_t key = sk[t0 + tid];
             const uint32_t m = m0 + running + ex;
-            const uint2 e = table[key];
             const uint32_t new_slot = stacks[(uint64_t)worker * S + (top_w - 1 - m)];
             // A key that the call running beside this one also touches keeps its table entry and its row until
             // that call is through (loc_deferred_kernel); its slot and its old owner's stack are settled now.
@@ -276,16 +309,93 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         if (s_stat[0]) atomicAdd(&st->deferred_now, s_stat[0]);
     }
     for (uint32_t i = tid; i < N; i += 256) owner_counts[(size_t)b * N + i] = s_hist[i];
+    // ---- phase 3 ----
     __threadfence();
-    grid_arrive(bar);                                           // (has a __syncthreads: the block's records are complete)
-    // ---- phase 2b: the block's rows, m0 .. m0 + cnt ----
+    if (!grid_barrier(bar, 2 * G, &s_ok)) {
+        if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
+        return;
+    }
+    {
+        // owner p's column of the per-block counts, added up by 256 / Np threads (Np = N rounded up to a power of two)
+        uint32_t Np = 1;
+        while (Np < N && Np < 256) Np <<= 1;
+        const uint32_t nq = 256 / Np, q = tid / Np;
+        for (uint32_t p0 = 0; p0 < N; p0 += Np) {
+            const uint32_t p = p0 + (tid % Np);
+            uint32_t base = 0, tot = 0;
+            if (p < N) {
+                for (uint32_t r0 = q; r0 < G; r0 += 16 * nq) {        // sixteen of the column's values asked for at a time
+                    uint32_t c[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k)
+                        c[k] = r0 + k * nq < G ? __ldcg(owner_counts + (size_t)(r0 + k * nq) * N + p) : 0u;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        tot += c[k];
+                        if (r0 + k * nq < b) base += c[k];
+                    }
+                }
+            }
+            s_part[0][tid] = base;
+            s_part[1][tid] = tot;
+            __syncthreads();
+            if (q == 0 && p < N) {
+                for (uint32_t i = 1; i < nq; ++i) {
+                    base += s_part[0][tid + i * Np];
+                    tot += s_part[1][tid + i * Np];
+                }
+                s_hist[p] = s_top[p] + base;
+                if (b == G - 1 && tot) tops[p] = (unsigned long long)s_top[p] + tot;    // never the requester's stack
+            }
+            __syncthreads();
+        }
+        if (b == G - 1 && tid == 0) {
+            tops[worker] = top_w - total;
+            st->rows_moved += total;
+        }
+    }
+    if (w == 0) {
+        const unsigned lt = (1u << lane) - 1u;
+        // the block's keys in rounds of 32; the old places of the first rounds are asked for all at once, so that
+        // the walk below (one round after the other: the counters run on) does not wait for memory in every round
+        constexpr int kAhead = 16;
+        uint32_t own_r[kAhead], slot_r[kAhead];
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k) {
+            const uint32_t i = k * 32 + lane;
+            own_r[k] = i < cnt ? sc.mowner[m0 + i] : 0u;
+            slot_r[k] = i < cnt ? sc.mslot[m0 + i] : 0u;
+        }
+        auto place = [&](bool valid, uint32_t owner, uint32_t slot) {
+            const unsigned peers = __match_any_sync(0xffffffffu, valid ? owner : (0x80000000u + lane));
+            const int leader = __ffs(peers) - 1;
+            uint32_t old = 0;
+            if (valid && lane == leader) {
+                old = s_hist[owner];
+                s_hist[owner] = old + __popc(peers);
+            }
+            old = __shfl_sync(0xffffffffu, old, leader);
+            if (valid) stacks[(uint64_t)owner * S + old + __popc(peers & lt)] = slot;
+            __syncwarp();
+        };
+#pragma unroll
+        for (int k = 0; k < kAhead; ++k)
+            if ((uint32_t)k * 32 < cnt) place((uint32_t)k * 32 + lane < cnt, own_r[k], slot_r[k]);
+        for (uint32_t i0 = kAhead * 32; i0 < cnt; i0 += 32) {
+            const bool valid = i0 + lane < cnt;
+            place(valid, valid ? sc.mowner[m0 + i0 + lane] : 0u, valid ? sc.mslot[m0 + i0 + lane] : 0u);
+        }
+    }
+    // ---- the rows: every block moves an equal share of the call's moving keys (their old and new places are
+    // in memory since barrier 2), whatever its own span of positions held ----
+    const uint32_t mlo = (uint32_t)((uint64_t)b * total / G), mcnt = (uint32_t)((uint64_t)(b + 1) * total / G) - mlo;
     if (row_bytes <= kLocStageBytes) {
         char* my = loc_stage + (size_t)w * kLocStages * kLocStageBytes;
         if (lane < kLocStages) mbar_init(&bars[w][lane], 1);
         mbar_init_fence();
         __syncwarp();
         const uint32_t per_round = tmin<uint32_t>(32u, kLocStageBytes / row_bytes);
-        const uint32_t n_rounds = (cnt + per_round - 1) / per_round;
+        const uint32_t n_rounds = (mcnt + per_round - 1) / per_round;
         uint32_t uses = 0;
         // rounds w, w + 8, ...; the loads of up to kLocStages - 1 later rounds are in flight while one is written out
         uint64_t dst_of[kLocStages];
@@ -296,13 +406,13 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
             rows_of[stage] = 0;
             if (r >= n_rounds) return;
             const uint32_t i = r * per_round + lane;
-            bool mine = (uint32_t)lane < per_round && i < cnt;
+            bool mine = (uint32_t)lane < per_round && i < mcnt;
             uint64_t src = 0;
             if (mine) {
-                const uint32_t m = m0 + i;
-                mine = sc.flag[m] == 0u;                        // (rows that wait for the call beside this one move later)
-                src = (uint64_t)sc.mowner[m] * S + sc.mslot[m];
-                dst_of[stage] = (uint64_t)worker * S + sc.mnew[m];
+                const uint32_t m = mlo + i;
+                mine = __ldcg(sc.flag + m) == 0u;               // (rows that wait for the call beside this one move later)
+                src = (uint64_t)__ldcg(sc.mowner + m) * S + __ldcg(sc.mslot + m);
+                dst_of[stage] = (uint64_t)worker * S + __ldcg(sc.mnew + m);
             }
             const uint32_t rows = (uint32_t)__popc(__ballot_sync(0xffffffffu, mine));
             mine_of[stage] = mine;
@@ -347,73 +457,11 @@ loc_fused_kernel(const uint32_t* __restrict__ sk, uint32_t n, uint32_t span, uin
         // rows too long for the staging: a warp per row, 128-bit loads and stores
         const uint32_t L4 = row_bytes / 16;
         float4* st4 = reinterpret_cast<float4*>(store);
-        for (uint32_t i = w; i < cnt; i += 8) {
-            const uint32_t m = m0 + i;
-            if (sc.flag[m]) continue;
-            const uint64_t src = (uint64_t)sc.mowner[m] * S + sc.mslot[m], dst = (uint64_t)worker * S + sc.mnew[m];
+        for (uint32_t i = w; i < mcnt; i += 8) {
+            const uint32_t m = mlo + i;
+            if (__ldcg(sc.flag + m)) continue;
+            const uint64_t src = (uint64_t)__ldcg(sc.mowner + m) * S + __ldcg(sc.mslot + m), dst = (uint64_t)worker * S + __ldcg(sc.mnew + m);
             for (uint32_t f = lane; f < L4; f += 32) st4[dst * L4 + f] = st4[src * L4 + f];
-        }
-    }
-    // ---- phase 3 ----
-    if (!grid_wait(bar, 2 * G, &s_ok)) {
-        if (tid == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
-        return;
-    }
-    {
-        // owner p's column of the per-block counts, added up by 256 / Np threads (Np = N rounded up to a power of two)
-        uint32_t Np = 1;
-        while (Np < N && Np < 256) Np <<= 1;
-        const uint32_t nq = 256 / Np, q = tid / Np;
-        for (uint32_t p0 = 0; p0 < N; p0 += Np) {
-            const uint32_t p = p0 + (tid % Np);
-            uint32_t base = 0, tot = 0;
-            if (p < N) {
-                for (uint32_t r0 = q; r0 < G; r0 += 4 * nq) {
-                    uint32_t c[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        c[k] = r0 + k * nq < G ? __ldcg(owner_counts + (size_t)(r0 + k * nq) * N + p) : 0u;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        tot += c[k];
-                        if (r0 + k * nq < b) base += c[k];
-                    }
-                }
-            }
-            s_part[0][tid] = base;
-            s_part[1][tid] = tot;
-            __syncthreads();
-            if (q == 0 && p < N) {
-                for (uint32_t i = 1; i < nq; ++i) {
-                    base += s_part[0][tid + i * Np];
-                    tot += s_part[1][tid + i * Np];
-                }
-                s_hist[p] = s_top[p] + base;
-                if (b == G - 1 && tot) tops[p] = (unsigned long long)s_top[p] + tot;    // never the requester's stack
-            }
-            __syncthreads();
-        }
-        if (b == G - 1 && tid == 0) {
-            tops[worker] = top_w - total;
-            st->rows_moved += total;
-        }
-    }
-    if (w == 0) {
-        const unsigned lt = (1u << lane) - 1u;
-        for (uint32_t i0 = 0; i0 < cnt; i0 += 32) {
-            const bool valid = i0 + lane < cnt;
-            const uint32_t m = m0 + i0 + lane;
-            const uint32_t owner = valid ? sc.mowner[m] : 0u;
-            const unsigned peers = __match_any_sync(0xffffffffu, valid ? owner : (0x80000000u + lane));
-            const int leader = __ffs(peers) - 1;
-            uint32_t old = 0;
-            if (valid && lane == leader) {
-                old = s_hist[owner];
-                s_hist[owner] = old + __popc(peers);
-            }
-            old = __shfl_sync(0xffffffffu, old, leader);
-            if (valid) stacks[(uint64_t)owner * S + old + __popc(peers & lt)] = sc.mslot[m];
-            __syncwarp();
         }
     }
     grid_leave(bar, G);
@@ -478,9 +526,9 @@ void run_localize(ps_store* ps, uint32_t worker, uint32_t n, int which, cudaStre
     if (ps->cfg.num_workers <= kLocFastWorkers) {
         static std::atomic<unsigned long long> smem_set{0};
         opt_in_smem((const void*)loc_fused_kernel, kLocSmem, &smem_set);
-        // two blocks per SM at most (all of them resident: they meet at grid barriers), spans of whole tiles of 256
+        // two blocks per SM at most (all of them resident: they meet at grid barriers)
         const uint32_t max_grid = tmin<uint32_t>((uint32_t)ps->sm_count * 2, kLocMaxGrid);
-        uint32_t span = div_up_u32(div_up_u32(n, max_grid), 256) * 256;
+        uint32_t span = tmax<uint32_t>(div_up_u32(n, max_grid), 32u);
         const uint32_t grid_f = div_up_u32(n, span);
         uint2* table = ps->table;
         unsigned long long* tops = ps->tops;
