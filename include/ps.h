@@ -309,6 +309,13 @@ ps_status_t ps_set_push_mode(ps_store_t* ps, int mode);
 enum { PS_MF_AUTO = 0, PS_MF_BY_COLUMN = 1, PS_MF_SYMMETRIC = 2 };
 ps_status_t ps_set_mf_path(ps_store_t* ps, int path);
 
+/* Self-test of the bounded device-side waits.  Every wait inside the kernels (the grid barrier of the one-launch
+ * sort and relocation, the arrival of bulk copies) gives up after a bounded number of polls, latches PS_ERR_CUDA and
+ * lets the kernel return, so that a lost arrival never hangs the GPU.  This call makes that happen on purpose, the
+ * harmless way: two blocks wait at the sort's barrier for a third that does not exist, for about a fifth of a
+ * second.  The next ps_sync returns PS_ERR_CUDA and puts the barrier back in order; the handle is usable after it. */
+ps_status_t ps_selftest_barrier_timeout(ps_store_t* ps, void* stream);
+
 /* Number of kernels this handle has launched so far. */
 uint64_t ps_launch_count(const ps_store_t* ps);
 

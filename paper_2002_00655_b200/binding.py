@@ -72,6 +72,7 @@ SIGNATURES = {
     "ps_set_host_overlap": (C.c_int, [_vp, C.c_int]),
     "ps_set_mf_path": (C.c_int, [_vp, C.c_int]),
     "ps_set_push_mode": (C.c_int, [_vp, C.c_int]),
+    "ps_selftest_barrier_timeout": (C.c_int, [_vp, _vp]),
     "ps_launch_count": (C.c_uint64, [_vp]),
     "ps_rows_moved": (C.c_int, [_vp, C.POINTER(_u64)]),
     "ps_profile_start": (C.c_int, [_vp, _u32]),
@@ -285,6 +286,10 @@ def ps_set_push_mode(ps, mode: int) -> None:
 
 def ps_set_mf_path(ps, path: int) -> None:
     _check(load_library().ps_set_mf_path(ps, int(path)), "ps_set_mf_path")
+
+
+def ps_selftest_barrier_timeout(ps) -> None:
+    _check(load_library().ps_selftest_barrier_timeout(ps, _stream()), "ps_selftest_barrier_timeout")
 
 
 def ps_launch_count(ps) -> int:

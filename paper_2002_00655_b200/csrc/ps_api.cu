@@ -545,6 +545,26 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     return release_set(ss, s);
 }
 
+// ---- self-test of the bounded waits ----
+// Two blocks meet at the sort's grid barrier and wait for a third arrival that never comes.  The wait is bounded
+// (kBarrierSpins polls, about a fifth of a second): the blocks give up, latch PS_ERR_CUDA and return, leaving the
+// barrier's count where it stood, which is the state ps_sync has to clean up after a sort that gave up.
+__global__ void barrier_timeout_kernel(unsigned int* bar, DevStatus* st) {
+    __shared__ int s_ok;
+    if (!grid_barrier(bar, gridDim.x + 1, &s_ok) && threadIdx.x == 0) atomicCAS(&st->sticky, 0u, (unsigned int)PS_ERR_CUDA);
+}
+
+ps_status_t ps_selftest_barrier_timeout(ps_store_t* ps, void* stream) {
+    PS_BEGIN_CALL(ps);
+    SortSet* ss = next_set(ps);
+    unsigned int* bar = ps->sort_ctl;
+    DevStatus* st = ps->status;
+    void* args[] = {(void*)&bar, (void*)&st};
+    cudaLaunchCooperativeKernel((const void*)barrier_timeout_kernel, dim3(2), dim3(64), args, 0, s);
+    ps->launches++;
+    return release_set(ss, s);
+}
+
 // ---- parameter blocking for matrix factorization ----
 __global__ void key_range_kernel(uint64_t* out, uint64_t first, uint64_t n) {
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;

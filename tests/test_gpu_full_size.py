@@ -51,7 +51,7 @@ def pull_host(g, keys):
     return out
 
 
-def check_rows(g, o, keys, what, loose=False):
+def check_rows(g, o, keys, what, loose=False, acc_before=None):
     """Rows of `keys` on the GPU against the oracle's."""
     keys = np.unique(np.asarray(keys, dtype=np.int64))
     got = pull_host(g, keys)
@@ -59,12 +59,23 @@ def check_rows(g, o, keys, what, loose=False):
     if not loose:
         assert_close(got, want, what)
     else:
-        # Several AdaGrad steps in a row.  The first step on a component with accumulator 0 is -lr g / (|g| + eps):
-        # where g is within rounding of zero the two sides may step by lr in opposite directions, so a few values
-        # in ten thousand leave the single-step tolerance; none may differ by more than such a pair of steps.
+        # Several AdaGrad steps in a row on rows [embedding | accumulators].  The first step on a component with
+        # accumulator 0 is -lr g / (|g| + eps): where g is within rounding of zero the two sides may step by lr in
+        # opposite directions.  Such a component is recognisable: its accumulator was 0 before the run and is still
+        # next to nothing after it (acc_before: the oracle's accumulators of `keys` before the run).  Those
+        # components may differ by up to 2 lr (0.2); what they feed into later steps (the scores of their triples, and
+        # through them other components' gradients, which AdaGrad divides by accumulators that are still small) may
+        # leave the single-step tolerance too: a few values in ten thousand, by a tenth of such a step at most.
         ok = close(got, want)
-        assert (~ok).mean() <= 1e-4, (what, int((~ok).sum()))
-        assert np.abs(got.astype(np.float64) - want).max() <= 0.2, what
+        half = want.shape[1] // 2
+        bad_e = ~ok[:, :half]
+        flip = (acc_before == 0) & (want[:, half:] < 1e-10)                     # per embedding component
+        diff = np.abs(got.astype(np.float64) - want)
+        assert (diff[:, :half][bad_e & flip] <= 0.2 + 1e-6).all(), what
+        rest = ~ok
+        rest[:, :half] &= ~flip
+        assert rest.mean() <= 1e-4, (what, int(rest.sum()))
+        assert diff[rest].max(initial=0.0) <= 2e-2, (what, float(diff[rest].max(initial=0.0)))
     return keys
 
 
@@ -144,7 +155,9 @@ def test_kge_steps():
         assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
         resync(g, o, touched)
     # three steps back to back, the sort of one beside the reduction of the one before
-    touched = check_rows(g, o, run(2 * c.batch, 3 * c.batch, 3), "kge, three steps in a row", loose=True)
+    acc0 = o.rows[:, 2 * c.dim:].copy()                     # the oracle's accumulators before the run
+    keys3 = run(2 * c.batch, 3 * c.batch, 3)
+    touched = check_rows(g, o, keys3, "kge, three steps in a row", loose=True, acc_before=acc0[np.unique(keys3.astype(np.int64))])
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
     check_untouched(g, o, touched, c.num_keys, "kge")
     resync(g, o, touched)
@@ -304,3 +317,73 @@ def test_stress_batches():
     got = pull_host(g, base)
     for x, key in enumerate(base):
         assert (got[x] == W.stress_init_rows(c, int(key), 1, DEV).cpu().numpy()[0]).all(), "an untouched row changed"
+
+
+@pytest.mark.parametrize("workload", ["kge", "sgns", "stress"])
+def test_pipelined_and_ordered_calls_agree_bit_for_bit_at_full_size(workload):
+    """Three steps back to back, once with every call ordered after the one before and once with the key sorts of
+    later calls running beside earlier calls' kernels (ps_set_pipelining): every touched row, the loss and (where
+    relocations run) the location table must come out identical, bit for bit.  A hazard between the sort of one
+    step and the reduction of the step before would show here, whatever tolerance the oracle comparison needs."""
+    def run(pipelined):
+        if workload == "kge":
+            c = W.KGE
+            need(2, 8)
+            g = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(3 + c.n_neg) * c.batch)
+            for s in range(0, c.num_keys, 1 << 18):
+                n = min(1 << 18, c.num_keys - s)
+                g.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=DEV), W.kge_init_rows(c, s, n, DEV))
+            ps.ps_set_pipelining(g.h, pipelined)
+            d = W.kge_triples(c, 0, 3 * c.batch, DEV)
+            torch.cuda.synchronize()
+            for b in range(3):
+                sl = slice(b * c.batch, (b + 1) * c.batch)
+                ps.ps_step_kge(g.h, *(t[sl] for t in d), c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps, g.loss)
+            s_, r_, o_, neg, _ = (t.cpu().numpy() for t in d)
+            keys = np.unique(np.concatenate([s_, o_, neg.ravel(), r_.astype(np.int64) + c.rel_key_base]).astype(np.int64))
+        elif workload == "sgns":
+            c = W.SGNS
+            need(4, 16)
+            occ = c.batch * (1 + 2 * c.window * (1 + c.n_neg))
+            g = ps.Store(c.num_keys, c.dim, 1, max_batch_keys=occ)
+            for s in range(0, c.num_keys, 1 << 18):
+                n = min(1 << 18, c.num_keys - s)
+                g.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=DEV), W.sgns_init_rows(c, s, n, DEV))
+            ps.ps_set_pipelining(g.h, pipelined)
+            tokens = W.sgns_tokens(c, 0, 3 * c.batch + c.window + 1, DEV)
+            negs = [W.sgns_negatives(c, b * c.batch, c.batch, DEV) for b in range(3)]
+            torch.cuda.synchronize()
+            for b in range(3):
+                ps.ps_step_sgns(g.h, tokens, b * c.batch, c.batch, c.window, negs[b], c.n_neg, c.out_key_base, c.lr, g.loss)
+            h_tok = tokens.cpu().numpy().astype(np.int64)
+            keys = np.unique(np.concatenate([h_tok, h_tok + c.out_key_base] + [t.cpu().numpy().astype(np.int64) + c.out_key_base for t in negs]))
+        else:
+            c = W.STRESS
+            need(6, 80)
+            g = ps.Store(c.num_keys, c.row_len, c.workers, c.slots_per_part, max_batch_keys=c.batch)
+            for s in range(0, c.num_keys, 1 << 21):
+                n = min(1 << 21, c.num_keys - s)
+                g.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=DEV), W.stress_init_rows(c, s, n, DEV))
+            ps.ps_set_pipelining(g.h, pipelined)
+            ks = [W.stress_keys(c, k, DEV) for k in range(3)]
+            upd = W.stress_updates(c, 0, DEV)
+            out = torch.empty((c.batch, c.row_len), dtype=torch.float32, device=DEV)
+            torch.cuda.synchronize()
+            for k in range(3):
+                ps.ps_pull(g.h, ks[k], out)
+                ps.ps_push(g.h, ks[k], upd)
+                ps.ps_localize(g.h, c.requester(k), ks[k][:c.localize_count])
+            keys = np.unique(np.concatenate([t.cpu().numpy() for t in ks]))
+        g.sync()
+        rows = pull_host(g, keys)
+        extra = g.export(rows=False)[1:] if workload == "stress" else ()
+        res = (rows, loss_of(g)) + tuple(t.numpy().copy() for t in extra)
+        g.close()
+        del g
+        torch.cuda.empty_cache()
+        return res
+
+    a, b = run(False), run(True)
+    assert a[1] == b[1] or (np.isnan(a[1]) and np.isnan(b[1])), "loss differs"
+    for x, y in zip(a[:1] + a[2:], b[:1] + b[2:]):
+        assert (x.view(np.uint32) == y.view(np.uint32)).all(), "pipelined calls gave other bits than ordered calls"

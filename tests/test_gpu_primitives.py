@@ -89,6 +89,29 @@ def test_push_by_atomic_adds_is_exact_on_integers_and_refuses_bad_keys():
     compare_state(g, o, what="sorted push afterwards")
 
 
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable():
+    """Device-side waits are bounded.  The self-test call lets two blocks wait at the sort's grid barrier for an
+    arrival that never comes: they give up, ps_sync reports PS_ERR_CUDA and re-arms the barrier (which was left
+    mid-count), and the calls after it work as if nothing had happened, the sort in the same buffer set included."""
+    import paper_2002_00655_b200 as ps
+    K, L = 2000, 16
+    g, o = make_pair(K, L, 2, K, max_batch_keys=4096)
+    rng = np.random.default_rng(12)
+    for round_ in range(2):
+        ps.ps_selftest_barrier_timeout(g.h)
+        assert g.sync(check=False) == ps.PS_ERR_CUDA
+        assert g.sync(check=False) == ps.PS_OK                  # reported once
+        for _ in range(5):                                      # every buffer set comes round again
+            keys = rng.integers(0, K, size=3000)
+            upd = rng.integers(-2, 3, size=(3000, L)).astype(np.float32)
+            g.push(dev(keys), dev(upd))
+            o.push(keys, upd)
+        g.localize(1, dev(keys[:500]))
+        o.localize(1, keys[:500])
+        g.sync()
+        compare_state(g, o, exact_rows=True, what=f"after the wait ran out, round {round_}")
+
+
 def test_push_and_pull_reject_bad_keys_without_touching_the_store():
     import paper_2002_00655_b200 as ps
     K, L = 500, 12
