@@ -397,11 +397,10 @@ kge_step_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr
             for (int q = 0; q < kMaxNeg; ++q) {
                 const double na = na_f[q], nb = nb_f[q];
                 const double w = __shfl_sync(full, coef, (q + 1) & 31);
-                if ((subj_mask >> q) & 1u) {
-                    A0 = fma(w, na, A0); B0 = fma(w, nb, B0);
-                } else {
-                    A1 = fma(w, na, A1); B1 = fma(w, nb, B1);
-                }
+                const bool in_subject_place = (subj_mask >> q) & 1u;
+                const double w0 = in_subject_place ? w : 0.0, w1 = in_subject_place ? 0.0 : w;
+                A0 += w0 * na; B0 += w0 * nb;
+                A1 += w1 * na; B1 += w1 * nb;
             }
             gr_re += (A0 * e + B0 * f) + (a * A1 + b * B1); gr_im += (A0 * f - B0 * e) + (a * B1 - b * A1);
             go_re += cr * A0 - ci * B0; go_im += cr * B0 + ci * A0;
