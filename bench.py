@@ -946,8 +946,11 @@ def run_ours(args):
     wl._prof_steps = prof_steps
     # The launch-bound loop of steps is captured into CUDA graphs (one per repeat, every step with its own batch
     # pointers) and each is replayed with one launch; --no-graph issues the calls one by one instead.
+    # Short repeats are issued eagerly: replaying a graph of K multi-stream steps costs a launch of its own (about
+    # 60 us here) that K = 20 steps do not amortise (52 us per MF-large step from a graph, 50 from eager calls; from
+    # about 64 steps on the graph is the faster form, and it keeps host jitter out of the timed region).
     graphs = None
-    if not args.no_graph and getattr(wl, "graph_ok", True):
+    if not args.no_graph and steps >= 64 and getattr(wl, "graph_ok", True):
         try:
             graphs = []
             for ch in chunks:
@@ -1073,7 +1076,7 @@ def run_ours(args):
                            "localize_stats": ps.ps_localize_stats(h)} if args.prelocalize else {})),
         "gpu_launches": int(round(launches_per_step * steps * repeats)), "launches_per_step": launches_per_step,
         "host_enqueue_ms_per_step": host_ms / len(timed),
-        "launch_mode": "one CUDA graph per repeat" if graphs is not None else "eager",
+        "launch_mode": "one CUDA graph per repeat" if graphs is not None else "eager calls (graphs from 64 steps per repeat on)",
         # `roofline`: the kernel on the caller's stream that takes the largest share of a step, its own bytes over its
         # own time (launched alone, events on its stream, in the per-kernel pass after the timed region).
         # `roofline_step`: the bytes the METHOD must move per step (no update rows, no sort traffic) over the

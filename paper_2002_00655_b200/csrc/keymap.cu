@@ -35,7 +35,7 @@ struct ps_keymap {
 namespace psb {
 
 constexpr unsigned long long kEmptyKey = ~0ull;
-constexpr uint32_t kMapMaxGrid = 512;
+constexpr uint32_t kMapMaxGrid = 2048;
 
 __device__ __forceinline__ uint64_t mix64(uint64_t x) {         // an avalanche of xor-shifts and odd multiplications
     x ^= x >> 31;
@@ -256,10 +256,14 @@ ps_status_t ps_keymap_insert(ps_keymap_t* m, const uint64_t* d_sparse, uint64_t 
     if (n == 0) return PS_OK;
     if (!d_sparse || !d_dense) return PS_ERR_INVALID_ARG;
     if (n > m->max_batch) return PS_ERR_WORKSPACE;
-    // all blocks are resident at once (they meet at grid barriers): one per SM at most, spans of whole tiles of 256
-    const uint32_t max_grid = tmin<uint32_t>((uint32_t)m->sm_count, kMapMaxGrid);
+    // All blocks are resident at once (they meet at grid barriers).  The probes are chains of dependent random reads,
+    // so the kernel wants as many threads in flight as fit: eight blocks per SM (the kernel is light on registers).
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, (const void*)map_insert_kernel, 256, 0) != cudaSuccess || per_sm < 1)
+        return PS_ERR_CUDA;
+    const uint32_t max_grid = tmin<uint32_t>((uint32_t)m->sm_count * (uint32_t)tmin(per_sm, 8), kMapMaxGrid);
     uint32_t n32 = (uint32_t)n;
-    uint32_t span = div_up_u32(div_up_u32(n, max_grid), 256) * 256;
+    uint32_t span = tmax<uint32_t>(div_up_u32(n, max_grid), 256u);
     const uint32_t grid = div_up_u32(n, span);
     ps_keymap km = *m;
     void* args[] = {(void*)&km, (void*)&d_sparse, (void*)&n32, (void*)&span, (void*)&d_dense};
