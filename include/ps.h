@@ -303,10 +303,12 @@ ps_status_t ps_set_push_mode(ps_store_t* ps, int mode);
  *     cells, so a row factor nearly always has one cell).  Row keys with several cells in a batch are summed by
  *     the last of their cells to finish; a batch in which few row keys carry most cells is served slowly.
  *   PS_MF_SYMMETRIC: row and column occurrences are reduced alike, then a second launch finishes the
- *     segments that cross tile borders.
+ *     segments that cross tile borders.  The rows of four positions are fetched by one instruction of the TMA unit
+ *     (tile::gather4 on the store as a 2-D tensor); PS_MF_SYMMETRIC_ROW_COPIES: by one bulk copy per row instead
+ *     (also what is used where the tensor cannot be described: rows of more than 256 values, 2^31 rows or more).
  *   PS_MF_AUTO (default): symmetric (the faster of the two on the 10M x 1M matrix of Section 4.1 as measured on
  *     B200: 45 against 49 microseconds per step of 65,536 cells). */
-enum { PS_MF_AUTO = 0, PS_MF_BY_COLUMN = 1, PS_MF_SYMMETRIC = 2 };
+enum { PS_MF_AUTO = 0, PS_MF_BY_COLUMN = 1, PS_MF_SYMMETRIC = 2, PS_MF_SYMMETRIC_ROW_COPIES = 3 };
 ps_status_t ps_set_mf_path(ps_store_t* ps, int path);
 
 /* Self-test of the bounded device-side waits.  Every wait inside the kernels (the grid barrier of the one-launch

@@ -26,7 +26,7 @@ PS_ERR_CAPACITY = 4
 PS_ERR_WORKSPACE = 5
 PS_ERR_CUDA = 6
 PS_ERR_UNSUPPORTED = 7
-PS_MF_AUTO, PS_MF_BY_COLUMN, PS_MF_SYMMETRIC = 0, 1, 2
+PS_MF_AUTO, PS_MF_BY_COLUMN, PS_MF_SYMMETRIC, PS_MF_SYMMETRIC_ROW_COPIES = 0, 1, 2, 3
 PS_PUSH_SORTED, PS_PUSH_ATOMIC = 0, 1
 PS_PUSH_STATIC_MAX_KEYS = 16384
 PS_PUSH_STATIC_MAX_ROW_LEN = 256

@@ -326,6 +326,29 @@ ps_status_t ps_create(const ps_config_t* cfg, void* d_store, void* d_table, void
             delete ps;
             return PS_ERR_CUDA;
         }
+    // The store as a 2-D tensor for the TMA unit: one instruction of the matrix-factorization step then fetches four
+    // rows (tile::gather4).  Rows of up to 256 values, row numbers that fit a signed 32-bit coordinate; where the
+    // driver lacks the entry point or refuses the shape, the step uses one bulk copy per row instead.
+    ps->row_map_ok = false;
+    if (cfg->row_len <= 256 && (uint64_t)cfg->num_workers * cfg->slots_per_part < (1ull << 31)) {
+        typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) == cudaSuccess && fn &&
+            qr == cudaDriverEntryPointSuccess) {
+            const cuuint64_t dims[2] = {cfg->row_len, (cuuint64_t)cfg->num_workers * cfg->slots_per_part};
+            const cuuint64_t strides[1] = {(cuuint64_t)cfg->row_len * 4};
+            const cuuint32_t box[2] = {cfg->row_len, 1};
+            const cuuint32_t estr[2] = {1, 1};
+            const CUresult r = ((encode_fn)fn)(&ps->row_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, d_store, dims, strides, box,
+                                               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ps->row_map_ok = r == CUDA_SUCCESS;
+        }
+        cudaGetLastError();
+    }
     *out = ps;
     return PS_OK;
 }
@@ -509,7 +532,8 @@ ps_status_t ps_step_mf(ps_store_t* ps, const uint32_t* d_i, const uint32_t* d_j,
     if (fused) {
         // gradient and reduction in one kernel over the sorted occurrences: no update rows
         if (!join_side(ps, s)) return PS_ERR_CUDA;
-        run_mf_fused(ps, (uint32_t)n, which, col_key_base, lr, lambda, d_loss_accum, s);
+        run_mf_fused(ps, (uint32_t)n, which, col_key_base, lr, lambda, d_loss_accum, s,
+                     ps->row_map_ok && ps->mf_path != PS_MF_SYMMETRIC_ROW_COPIES);
         return release_set(ss, s);
     }
     const uint32_t lb = launch_step_mf(ps, d_i, d_j, d_v, n, col_key_base, lr, lambda, s);
@@ -896,7 +920,7 @@ ps_status_t ps_set_push_mode(ps_store_t* ps, int mode) {
 }
 
 ps_status_t ps_set_mf_path(ps_store_t* ps, int path) {
-    if (!ps || path < 0 || path > 2) return PS_ERR_INVALID_ARG;
+    if (!ps || path < 0 || path > 3) return PS_ERR_INVALID_ARG;
     ps->mf_path = path;
     return PS_OK;
 }

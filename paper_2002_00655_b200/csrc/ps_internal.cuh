@@ -3,6 +3,7 @@
 #pragma once
 
 #include <atomic>
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -122,6 +123,8 @@ struct ps_store {
     bool host_overlap;
     cudaEvent_t batch_ready;        // set while a call's batch is still on its way: the side stream waits for it
     bool pipelined;                 // see ps_set_pipelining
+    CUtensorMap row_map;            // the store as a 2-D tensor (row_len x rows, one row per box) for row gathers by the TMA unit
+    bool row_map_ok;
     int mf_path;                    // see ps_set_mf_path
     psb::SortSet* last_set;         // the most recent call's buffer set if that call sorted its keys (else null)
     cudaStream_t last_stream;       // the stream of the most recent call
@@ -221,7 +224,7 @@ void run_push_atomic(ps_store* ps, const uint64_t* d_keys, uint64_t n, const flo
 // MF step working on the sorted occurrences directly (rows of at most 512 values): gradient, reduction,
 // then the fix-up launch that also moves the staged rows into the store
 void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
-                  double* d_loss_accum, cudaStream_t s);
+                  double* d_loss_accum, cudaStream_t s, bool gather4);
 // ---- mf_col.cu ----
 // MF step as one launch over the column side of the sorted occurrences (rows of at most 128 values).  launch_mf_plan
 // goes on the stream the sort ran on, right after it; run_mf_col on the caller's stream after the join.
@@ -378,6 +381,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
 __device__ __forceinline__ void bulk_s2g(void* gmem, const void* smem, unsigned bytes) {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n" ::"l"(gmem), "r"(smem_addr(smem)), "r"(bytes)
                  : "memory");
+}
+// Four rows of a 2-D tensor (one row per box) into consecutive rows of shared memory with ONE instruction of the TMA
+// unit: column x (x times the element size a multiple of 16 bytes), rows y0..y3.  The destination is 128-byte aligned.
+__device__ __forceinline__ void tma_gather4(void* smem, const CUtensorMap* map, int x, int y0, int y1, int y2, int y3,
+                                            uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, "
+        "%5, %6}], [%7];\n" ::"r"(smem_addr(smem)),
+        "l"(map), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3), "r"(smem_addr(bar))
+        : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;\n" ::: "memory"); }
 // until at most kPending of this thread's bulk groups still have to READ their source

@@ -728,15 +728,19 @@ kge_reduce_kernel(const uint32_t* __restrict__ sk, const uint32_t* __restrict__ 
 // is updated.
 constexpr int kMfTile = 8;
 constexpr int kMfStages = 3;
-constexpr size_t kMfSmem = (size_t)8 * kMfStages * 4 * 64 * sizeof(float4);     // warp x stage x group x {partner, own}
+constexpr size_t kMfSmem = (size_t)8 * kMfStages * 4 * 64 * sizeof(float4) + 128;   // warp x stage x group x {partner, own}; room to align
 
 enum : uint32_t { kFUsable = 1, kFBegin = 2, kFEnd = 4, kFParked = 8, kFFromPrev = 16, kFBoth = 32, kFSingle = 64,
                   kFColumn = 128 };
 
-template <int kC>
+// kG4: the four partner rows of a walk step (one per group of eight lanes) are fetched by ONE instruction of the TMA
+// unit (tile::gather4 on the store seen as a 2-D tensor of rows) instead of four bulk copies: the rate at which an SM
+// gets such copies served is what bounds this kernel.  A stage of a warp is then laid out as {four partner rows, one
+// after the other | four own rows of 512 bytes}.
+template <int kC, bool kG4>
 __global__ void __launch_bounds__(256, 2)
-mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, const uint32_t* __restrict__ cellpos,
-              uint32_t n,
+mf_sub_kernel(const __grid_constant__ CUtensorMap row_map, const uint32_t* __restrict__ sk, const uint4* __restrict__ rec,
+              const uint32_t* __restrict__ cellpos, uint32_t n,
               uint32_t col_base, float lr, float lam, float4* store, uint32_t K,
               uint32_t L4, float4* __restrict__ staged, uint64_t* __restrict__ apply_row, double* __restrict__ carry,
               uint4* __restrict__ starters, unsigned int* __restrict__ starter_count,
@@ -813,7 +817,8 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
         kg_far = sk[gpos + 8 * kMfTile - 1];
     }
     const uint32_t L = L4 * 4;
-    float4* my_stage = stage_mem + (size_t)w * (kMfStages * 4 * 64);
+    // (the stages start on a 128-byte boundary of shared memory: the TMA unit asks for that)
+    float4* my_stage = stage_mem + ((128u - (smem_addr(stage_mem) & 127u)) & 127u) / 16 + (size_t)w * (kMfStages * 4 * 64);
     // Rows reach shared memory as bulk asynchronous copies of whole rows, issued by the lane that holds the
     // position; all copies of a walk step report to one barrier word of the warp.  (Per-lane 16-byte
     // asynchronous copies were measured too: 26 and 43 us per side against 20 and 20 with bulk copies.)
@@ -825,6 +830,21 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
     auto issue = [&](int s2, int stage) {
         if (s2 >= kMfTile) return;
         const unsigned sm = 0x01010101u << s2;
+        if (kG4) {
+            // the partner rows of the four groups' positions of this step (row 0 for a group that has none)
+            const uint32_t want = usable ? prow : 0u;
+            const int r0 = (int)__shfl_sync(full, want, s2), r1 = (int)__shfl_sync(full, want, 8 + s2);
+            const int r2 = (int)__shfl_sync(full, want, 16 + s2), r3 = (int)__shfl_sync(full, want, 24 + s2);
+            if (!(usable_mask & sm)) return;
+            float4* dst = my_stage + (size_t)stage * 256;
+            if (lane == 0) {
+                mbar_expect_tx(&bars[w][stage], (4u + __popc(begin_mask & sm)) * row_bytes);
+                tma_gather4(dst, &row_map, 0, r0, r1, r2, r3, &bars[w][stage]);
+            }
+            __syncwarp();
+            if (l8 == s2 && begin_me) bulk_g2s(dst + 128 + sg * 32, store + (uint64_t)row * L4, row_bytes, &bars[w][stage]);
+            return;
+        }
         const uint32_t n_rows = __popc(usable_mask & sm) + __popc(begin_mask & sm);
         if (n_rows == 0) return;
         if (lane == 0) mbar_expect_tx(&bars[w][stage], n_rows * row_bytes);
@@ -865,7 +885,10 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
             }
             uses ^= 1u << st_use;
         }
-        const float4* slot = my_stage + (size_t)(st_use * 4 + sg) * 64 + l8;
+        // where this group's partner row and own row of the step lie
+        const float4* slot = kG4 ? my_stage + (size_t)st_use * 256 + (size_t)sg * L4 + l8
+                                 : my_stage + (size_t)(st_use * 4 + sg) * 64 + l8;
+        const float4* oslot = kG4 ? my_stage + (size_t)st_use * 256 + 128 + sg * 32 + l8 : slot + 32;
         st_use = st_use + 1 == kMfStages ? 0 : st_use + 1;
         st_fill = st_fill + 1 == kMfStages ? 0 : st_fill + 1;
         const int src = 8 * sg + s2;
@@ -881,7 +904,7 @@ mf_sub_kernel(const uint32_t* __restrict__ sk, const uint4* __restrict__ rec, co
             nw = 0.f;
 #pragma unroll
             for (int c = 0; c < kC; ++c) {
-                own[c] = (uint32_t)(l8 + 8 * c) < L4 ? slot[32 + 8 * c] : make_float4(0.f, 0.f, 0.f, 0.f);
+                own[c] = (uint32_t)(l8 + 8 * c) < L4 ? oslot[8 * c] : make_float4(0.f, 0.f, 0.f, 0.f);
                 nw += own[c].x * own[c].x + own[c].y * own[c].y + own[c].z * own[c].z + own[c].w * own[c].w;
                 acc[c] = d4{0.0, 0.0, 0.0, 0.0};
             }
@@ -1303,20 +1326,29 @@ static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d
 // of at most 128 values.  One launch over all positions, then the fix-up launch, which also moves the staged rows
 // into the store.
 void run_mf_fused(ps_store* ps, uint32_t n_cells, int which, uint64_t col_key_base, float lr, float lambda,
-                  double* d_loss_accum, cudaStream_t s) {
+                  double* d_loss_accum, cudaStream_t s, bool gather4) {
     const uint32_t* sk = which ? ps->keysB : ps->keysA;
     const uint32_t n = 2 * n_cells;
     const uint32_t L4 = ps->cfg.row_len / 4;
     const uint32_t blocks = div_up_u32(n, 256);
 #define SUB_ARGS                                                                                                     \
-    sk, ps->rec, ps->cellpos, n, (uint32_t)col_key_base, lr, lambda, (float4*)ps->store, (uint32_t)ps->cfg.num_keys, \
+    ps->row_map, sk, ps->rec, ps->cellpos, n, (uint32_t)col_key_base, lr, lambda, (float4*)ps->store, (uint32_t)ps->cfg.num_keys, \
         L4, (float4*)ps->upd, ps->apply_rows, ps->carry, ps->starters, ps->starter_count, ps->group_done,            \
         ps->group_sum, ps->loss_partial, ps->status, ps->epoch
 #define SUB_LAUNCH(kC)                                                                                               \
     do {                                                                                                             \
-        static std::atomic<unsigned long long> smem_set{0};                                                          \
-        opt_in_smem((const void*)mf_sub_kernel<kC>, kMfSmem, &smem_set);                                             \
-        PS_LAUNCH_SMEM(ps, mf_sub_kernel<kC>, blocks, 256, kMfSmem, s, SUB_ARGS);                                    \
+        static std::atomic<unsigned long long> smem_set{0}, smem_set4{0};                                            \
+        if (gather4) {                                                                                               \
+            opt_in_smem((const void*)mf_sub_kernel<kC, true>, kMfSmem, &smem_set4);                                  \
+            if (ps->prof) prof_before(ps, "mf_sub_kernel<" #kC ",gather4>", s);                                      \
+            mf_sub_kernel<kC, true><<<blocks, 256, kMfSmem, s>>>(SUB_ARGS);                                          \
+        } else {                                                                                                     \
+            opt_in_smem((const void*)mf_sub_kernel<kC, false>, kMfSmem, &smem_set);                                  \
+            if (ps->prof) prof_before(ps, "mf_sub_kernel<" #kC ">", s);                                              \
+            mf_sub_kernel<kC, false><<<blocks, 256, kMfSmem, s>>>(SUB_ARGS);                                         \
+        }                                                                                                            \
+        if (ps->prof) prof_after(ps, s);                                                                             \
+        ps->launches++;                                                                                              \
     } while (0)
     if (L4 <= 8) SUB_LAUNCH(1);
     else if (L4 <= 16) SUB_LAUNCH(2);
