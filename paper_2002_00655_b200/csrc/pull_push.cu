@@ -800,7 +800,6 @@ mf_sub_kernel(const __grid_constant__ CUtensorMap row_map, const uint32_t* __res
     const bool stage_me = end_me && !parked;                        // a whole segment ends here: new row
     const uint32_t tile8 = tile32 * 4 + sg;
     if (runs_on && !from_prev) starters[atomicAdd(starter_count, 1u)] = make_uint4(tile8, key, row, 0u);
-    if (inside) apply_row[pos] = stage_me ? (uint64_t)row : ~0ull;
     const unsigned begin_mask = __ballot_sync(full, begin_me);
     const uint32_t flags = (usable ? kFUsable : 0u) | (begin_me ? kFBegin : 0u) | (end_me ? kFEnd : 0u) |
                            (parked ? kFParked : 0u) | (from_prev ? kFFromPrev : 0u) |
@@ -950,7 +949,8 @@ mf_sub_kernel(const __grid_constant__ CUtensorMap row_map, const uint32_t* __res
                     else staged[drow * L4 + l8 + 8 * c] = r;
                 }
             }
-            if (direct && l8 == 0) apply_row[drow] = ~0ull;     // nothing to move later
+            // a staged row goes on the (short) list of rows the fix-up launch moves into the store
+            if (!direct && l8 == 0) apply_row[atomicAdd(starter_count + 1, 1u)] = ((uint64_t)row_s << 32) | drow;
         } else if (live) {
 #pragma unroll
             for (int c = 0; c < kC; ++c) {
@@ -976,7 +976,8 @@ mf_sub_kernel(const __grid_constant__ CUtensorMap row_map, const uint32_t* __res
                         else staged[drow * L4 + fi] = r;
                     }
                 }
-                if (direct && !(f & kFParked) && l8 == 0) apply_row[drow] = ~0ull;
+                if (!direct && !(f & kFParked) && l8 == 0)
+                    apply_row[atomicAdd(starter_count + 1, 1u)] = ((uint64_t)row_s << 32) | drow;
             }
         }
     }
@@ -1017,35 +1018,37 @@ push_fixup_kernel(const uint32_t* __restrict__ sk, uint32_t n, float4* __restric
                   uint32_t apply_lo, const DevStatus* st, unsigned int epoch) {
     if (call_failed(st, epoch)) return;
     if (blockIdx.x > fix_blocks) {
-        // Blocks past the loss block move staged rows into the store (calls that stage rows only): a warp
-        // looks at 32 sorted positions at a time and copies the rows staged there, four in flight at once.
+        // Blocks past the loss block move staged rows into the store (calls that stage rows only): the reduction
+        // left a list of {row, staging position}; a warp takes 32 entries at a time and copies their rows, several
+        // in flight at once.
         const unsigned full = 0xffffffffu;
         const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-        const uint64_t stride = (uint64_t)(gridDim.x - fix_blocks - 1) * kFixupWarps * 32;
-        for (uint64_t b0 = apply_lo + ((uint64_t)(blockIdx.x - fix_blocks - 1) * kFixupWarps + w) * 32; b0 < n; b0 += stride) {
-            const uint64_t r = b0 + lane < n ? apply_row[b0 + lane] : ~0ull;
-            unsigned m = __ballot_sync(full, r != ~0ull);
+        const uint32_t listed = starter_count[1];
+        const uint32_t stride = (gridDim.x - fix_blocks - 1) * kFixupWarps * 32;
+        for (uint32_t b0 = ((blockIdx.x - fix_blocks - 1) * kFixupWarps + w) * 32; b0 < listed; b0 += stride) {
+            const uint64_t e = b0 + lane < listed ? apply_row[b0 + lane] : ~0ull;
+            unsigned m = __ballot_sync(full, b0 + lane < listed);
             constexpr int kFly = kCh == 1 ? 8 : 4;           // rows in flight per warp
             while (m) {
                 int q[kFly];
-                uint64_t rr[kFly];
+                uint64_t ee[kFly];
                 float4 x[kFly][kCh];
 #pragma unroll
                 for (int a = 0; a < kFly; ++a) {
                     q[a] = m ? __ffs(m) - 1 : -1;
                     m &= m - 1;                              // 0 stays 0
-                    rr[a] = __shfl_sync(full, r, q[a] & 31);
+                    ee[a] = __shfl_sync(full, e, q[a] & 31);
                 }
 #pragma unroll
                 for (int a = 0; a < kFly; ++a)
 #pragma unroll
                     for (int c = 0; c < kCh; ++c)
-                        if (q[a] >= 0 && lane + 32 * c < L4) x[a][c] = __ldcs(staged + (b0 + q[a]) * L4 + lane + 32 * c);
+                        if (q[a] >= 0 && lane + 32 * c < L4) x[a][c] = __ldcs(staged + (ee[a] & 0xffffffffu) * L4 + lane + 32 * c);
 #pragma unroll
                 for (int a = 0; a < kFly; ++a)
 #pragma unroll
                     for (int c = 0; c < kCh; ++c)
-                        if (q[a] >= 0 && lane + 32 * c < L4) store[rr[a] * L4 + lane + 32 * c] = x[a][c];
+                        if (q[a] >= 0 && lane + 32 * c < L4) store[(ee[a] >> 32) * L4 + lane + 32 * c] = x[a][c];
             }
         }
         return;
@@ -1307,9 +1310,11 @@ static void launch_fixup(ps_store* ps, const uint32_t* sk, uint32_t n, double* d
     const uint32_t tiles = div_up_u32(n, tile_len);
     const uint32_t L4 = ps->cfg.row_len / 4;
     // a warp per listed segment; there are fewer segments in the list than tiles
-    const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * 8);
-    const uint32_t apply_blocks =
-        apply ? tmax<uint32_t>(1u, tmin<uint32_t>(div_up_u32(n - apply_lo, 32 * kFixupWarps), (uint32_t)ps->sm_count * 8)) : 0;
+    const uint32_t fix_blocks = tmin<uint32_t>(div_up_u32(tiles, kFixupWarps), (uint32_t)ps->sm_count * (apply ? 4 : 8));
+    // the rows staged by a matrix-factorization step are few (row keys with several cells, and their columns): a
+    // handful of blocks works through their list
+    const uint32_t apply_blocks = apply ? 8u : 0u;
+    (void)apply_lo;
     const uint32_t grid = fix_blocks + 1 + apply_blocks;
 #define FIXUP_ARGS sk, n, (float4*)ps->store, ps->table, ps->cfg.slots_per_part, (uint32_t)ps->cfg.num_keys, L4,   \
                    ps->carry, ps->group_sum, ps->starters, ps->starter_count, ps->loss_partial, loss_blocks,      \

@@ -154,7 +154,7 @@ sort_all_kernel(Src src, Sink sink, SortParams P) {
     }
     if (b == 0) {
         for (uint32_t i = tid; i < P.n_zero_a; i += kThreads) P.zero_a[i] = 0u;
-        if (tid == 0 && P.zero_b) *P.zero_b = 0u;
+        if (tid == 0 && P.zero_b) P.zero_b[0] = P.zero_b[1] = 0u;     // (the list counter of the coming reduction and its neighbour)
     }
     __syncthreads();
     uint32_t key0[kItems];                           // keys of the chunk's first tile stay in registers for pass 0
