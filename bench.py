@@ -116,7 +116,7 @@ def smi_clocks():
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/,
 # keyed by (workload, kernel).  An entry is removed when its kernel changes after the capture.
 TRAFFIC = {
-    ("mf_large", "mf_sub_kernel<4>"): 46.5e6,                   # profiles/mf_step_kernels_ncu_full.md (same-batch twin)
+    ("mf_large", "mf_sub_kernel<4,gather4>"): 46.1e6,                 # profiles/mf_step_kernels_ncu_full.md (same-batch twin)
     ("kge", "kge_reduce_kernel<2>"): 321.6e6,                   # profiles/kge_step_kernels_ncu_full.md
     ("sgns", "push_reduce_kernel<3,true>"): 1561.1e6,           # profiles/sgns_step_kernels_ncu_full.md
 }
