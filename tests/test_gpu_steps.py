@@ -80,6 +80,39 @@ def test_mf_single_steps(R, Cc, L, n, zipf, path):
         assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
 
 
+def _random_mf_shapes(count, seed):
+    """Seeded shapes: few to many rows and columns (so that row keys repeat a lot, a little, or never), ranks that
+    are and are not multiples of 32 values, batches that end inside a tile."""
+    r = np.random.RandomState(seed)
+    out = []
+    for _ in range(count):
+        R = int(round(10 ** r.uniform(0.5, 4.7)))
+        Cc = int(round(10 ** r.uniform(0.3, 3.7)))
+        L = 4 * int(r.randint(1, 33))
+        n = int(r.randint(1, 4000))
+        zipf = None if r.rand() < 0.4 else float(r.uniform(1.05, 1.5))
+        out.append((R, Cc, L, n, zipf))
+    return out
+
+
+@pytest.mark.parametrize("path", [ps.PS_MF_SYMMETRIC, ps.PS_MF_SYMMETRIC_ROW_COPIES, ps.PS_MF_BY_COLUMN])
+def test_mf_seeded_random_shapes(path):
+    """One step each on two dozen seeded shapes, every row against the oracle; the symmetric form both with the
+    four-row TMA gather and with one bulk copy per row."""
+    for R, Cc, L, n, zipf in _random_mf_shapes(24, 20260101):
+        cfg = W.MFConfig("t", R, Cc, L, n, n, 0.002, 0.05, 0.1, 0.5, zipf)
+        rows = W.mf_init_rows(cfg, 0, cfg.num_keys, "cpu")
+        i, j, v = mf_data(cfg)
+        g, o = make_pair(cfg.num_keys, L, rows=rows, max_batch_keys=2 * n)
+        ps.ps_set_mf_path(g.h, path)
+        g.loss.zero_(); o.loss[0] = 0
+        ps.ps_step_mf(g.h, i.cuda(), j.cuda(), v.cuda(), cfg.col_key_base, cfg.lr, cfg.lam, g.loss)
+        o.step_mf(i, j, v, cfg.col_key_base, cfg.lr, cfg.lam)
+        g.sync()
+        compare_state(g, o, what=f"mf {R}x{Cc} rank {L} batch {n} zipf {zipf}")
+        assert close(loss_of(g), o.loss[0]), (R, Cc, L, n, zipf, loss_of(g), o.loss[0])
+
+
 def test_mf_bad_index_makes_the_step_a_no_op():
     g, o = make_pair(100, 8)
     i = dev(np.array([1, 2, 60, 3]), torch.int32)               # 60 >= col_key_base
