@@ -26,7 +26,9 @@
  * Parity unpinned by the paper (the paper prints no formula or number for
  * them; they are this repository's stated readings): the free-slot policy of
  * localize, the 1/2 convention and per-occurrence L2 of the MF loss, AdaGrad's
- * eps and per-data-point application, the fixed skip-gram window.
+ * eps and per-data-point application, the fixed skip-gram window, and for
+ * RESCAL the layout of a relation's matrix as one key per matrix row (the score
+ * itself is pinned against the bilinear form written with numpy).
  */
 #include <math.h>
 #include <stdint.h>
@@ -334,6 +336,101 @@ int ops_step_kge(ops_store *st, const uint32_t *ts, const uint32_t *tr, const ui
         }
     }
     free(key); free(rep); free(g);
+    apply_acc(st);
+    if (loss_accum) *loss_accum += loss;
+    return OPS_OK;
+}
+
+/* RESCAL with AdaGrad and negative sampling (Section 4.1 names the model; Table 4 gives entity dimension d = 100
+ * and relation dimension d * d = 10,000; training as for ComplEx, Appendix A).  All rows of the store have one
+ * length, so a relation's d x d matrix is held as d keys, one per matrix row:
+ *   key e < rel_key_base                    entity e,        row [x(0..d) | G(0..d)]
+ *   key rel_key_base + r * d + a            row a of R_r,    row [R_r[a][0..d) | G(0..d)]
+ * with G the element-wise AdaGrad accumulators (L = 2 d).
+ * Score of (s, r, o):  phi = x_s^T R_r x_o = sum_a sum_b x_s[a] R_r[a][b] x_o[b].
+ * Data points, negatives, loss softplus(-y phi), and the AdaGrad step per DISTINCT key of a data point from
+ * pre-batch (theta, G) are those of ops_step_kge; the d matrix-row keys of a data point are distinct by
+ * construction, entity keys may repeat among subject, object and negatives. */
+int ops_step_rescal(ops_store *st, const uint32_t *ts, const uint32_t *tr, const uint32_t *to,
+                    const uint32_t *neg_ent, const uint8_t *neg_side, uint64_t n, uint32_t n_neg,
+                    uint64_t rel_key_base, uint32_t dim, float lr_f, float eps_f, double *loss_accum) {
+    const uint32_t L = st->L, d = dim;
+    if (L != 2 * d) return OPS_ERR_INVALID_ARG;
+    const double lr = lr_f, eps = eps_f;
+    for (uint64_t t = 0; t < n; ++t) {
+        if (ts[t] >= rel_key_base || to[t] >= rel_key_base || rel_key_base + ((uint64_t)tr[t] + 1) * d > st->K)
+            return OPS_ERR_KEY_RANGE;
+        for (uint32_t q = 0; q < n_neg; ++q)
+            if (neg_ent[t * n_neg + q] >= rel_key_base) return OPS_ERR_KEY_RANGE;
+    }
+    const uint32_t n_slots = 2 + n_neg;             /* s, o, negatives: the entity keys of a data point */
+    uint64_t *key = (uint64_t *)malloc(n_slots * sizeof(uint64_t));
+    uint32_t *rep = (uint32_t *)malloc(n_slots * sizeof(uint32_t));
+    double *g = (double *)malloc((uint64_t)n_slots * d * sizeof(double));
+    double *gR = (double *)malloc((uint64_t)d * d * sizeof(double));
+    double loss = 0;
+    for (uint64_t t = 0; t < n; ++t) {
+        key[0] = ts[t]; key[1] = to[t];
+        for (uint32_t q = 0; q < n_neg; ++q) key[2 + q] = neg_ent[t * n_neg + q];
+        for (uint32_t u = 0; u < n_slots; ++u) {    /* first slot holding the same key */
+            rep[u] = u;
+            for (uint32_t z = 0; z < u; ++z)
+                if (key[z] == key[u]) { rep[u] = z; break; }
+        }
+        const uint64_t rk = rel_key_base + (uint64_t)tr[t] * d;     /* key of row 0 of R_r */
+        memset(g, 0, (uint64_t)n_slots * d * sizeof(double));
+        memset(gR, 0, (uint64_t)d * d * sizeof(double));
+        for (uint32_t q = 0; q <= n_neg; ++q) {     /* q = 0: the positive triple */
+            uint32_t us = 0, uo = 1;
+            double y = 1.0;
+            if (q > 0) {
+                y = -1.0;
+                if (neg_side[t * n_neg + q - 1] == 0) us = 2 + q - 1; else uo = 2 + q - 1;
+            }
+            const float *S = st->rows + key[us] * L, *O = st->rows + key[uo] * L;
+            double phi = 0;
+            for (uint32_t a = 0; a < d; ++a) {
+                const float *Ra = st->rows + (rk + a) * L;
+                double ro = 0;
+                for (uint32_t b = 0; b < d; ++b) ro += (double)Ra[b] * O[b];
+                phi += (double)S[a] * ro;
+            }
+            loss += softplus(-y * phi);
+            double coef = -y * sigmoid(-y * phi);   /* d loss / d phi */
+            double *gs = g + (uint64_t)rep[us] * d, *go = g + (uint64_t)rep[uo] * d;
+            for (uint32_t a = 0; a < d; ++a) {
+                const float *Ra = st->rows + (rk + a) * L;
+                for (uint32_t b = 0; b < d; ++b) {
+                    /* each += reads only pre-batch values, so aliasing gs == go is fine */
+                    gs[a] += coef * (double)Ra[b] * O[b];
+                    go[b] += coef * (double)S[a] * Ra[b];
+                    gR[(uint64_t)a * d + b] += coef * (double)S[a] * O[b];
+                }
+            }
+        }
+        for (uint32_t u = 0; u < n_slots; ++u) {
+            if (rep[u] != u) continue;
+            const float *G = st->rows + key[u] * L + d;
+            const double *gu = g + (uint64_t)u * d;
+            double *acc = acc_row(st, key[u]);
+            for (uint32_t c = 0; c < d; ++c) {
+                double g2 = gu[c] * gu[c];
+                acc[c] += -lr * gu[c] / (sqrt((double)G[c] + g2) + eps);
+                acc[d + c] += g2;
+            }
+        }
+        for (uint32_t a = 0; a < d; ++a) {
+            const float *G = st->rows + (rk + a) * L + d;
+            const double *gu = gR + (uint64_t)a * d;
+            double *acc = acc_row(st, rk + a);
+            for (uint32_t c = 0; c < d; ++c) {
+                double g2 = gu[c] * gu[c];
+                acc[c] += -lr * gu[c] / (sqrt((double)G[c] + g2) + eps);
+                acc[d + c] += g2;
+            }
+        }
+    }
+    free(key); free(rep); free(g); free(gR);
     apply_acc(st);
     if (loss_accum) *loss_accum += loss;
     return OPS_OK;

@@ -47,6 +47,7 @@ def _load():
             "ops_get_location": [vp, vp, u64, vp, vp],
             "ops_step_mf": [vp, vp, vp, vp, u64, u64, f32, f32, vp],
             "ops_step_kge": [vp, vp, vp, vp, vp, vp, u64, u32, u64, u32, f32, f32, vp],
+            "ops_step_rescal": [vp, vp, vp, vp, vp, vp, u64, u32, u64, u32, f32, f32, vp],
             "ops_step_sgns": [vp, vp, u64, u64, u64, u32, vp, u32, u64, f32, vp],
         }.items():
             getattr(lib, name).argtypes = args
@@ -178,6 +179,15 @@ class OracleStore:
         self._check(_load().ops_step_kge(self._h, _p(s), _p(r), _p(o), _p(neg_ent), _p(neg_side), s.size,
                                          n_neg, int(rel_key_base), int(dim), float(lr), float(eps),
                                          _p(self.loss)))
+
+    def step_rescal(self, s, r, o, neg_ent, neg_side, rel_key_base, dim, lr, eps):
+        s, r, o = _np(s, np.uint32), _np(r, np.uint32), _np(o, np.uint32)
+        neg_ent, neg_side = _np(neg_ent, np.uint32), _np(neg_side, np.uint8)
+        n_neg = neg_ent.size // max(s.size, 1)
+        assert neg_ent.size == s.size * n_neg == neg_side.size
+        self._check(_load().ops_step_rescal(self._h, _p(s), _p(r), _p(o), _p(neg_ent), _p(neg_side), s.size,
+                                            n_neg, int(rel_key_base), int(dim), float(lr), float(eps),
+                                            _p(self.loss)))
 
     def step_sgns(self, tokens, first_pos, n_centers, window, negs, n_neg, out_key_base, lr):
         tokens, negs = _np(tokens, np.uint32), _np(negs, np.uint32)
