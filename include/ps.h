@@ -78,6 +78,7 @@ typedef struct {
 /* Sizes of the four device buffers the caller must allocate (256-byte aligned).
  * `max_batch_keys` bounds the key occurrences of any later call: n for
  * pull/push/localize, 2n for ps_step_mf, (3 + n_neg) * n for ps_step_kge,
+ * (2 + n_neg + dim) * n for ps_step_rescal,
  * n_centers * (1 + 2 * window * (1 + n_neg)), and at least 3 * n_centers,
  * for ps_step_sgns. */
 ps_status_t ps_query_sizes(const ps_config_t* cfg, uint64_t max_batch_keys, ps_sizes_t* out);
@@ -177,6 +178,25 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
                         const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n,
                         uint32_t n_neg, uint64_t rel_key_base, uint32_t dim_complex, float lr,
                         float eps, double* d_loss_accum, void* stream);
+
+/* One minibatch of RESCAL with AdaGrad and negative sampling (Section 4.1 names the
+ * model, Table 4 its sizes: entity dimension dim, relation dimension dim * dim;
+ * training as for ComplEx, Appendix A).  All rows have one length, so a
+ * relation's matrix is dim keys, one per matrix row: key e < rel_key_base is
+ * entity e with row [x | G]; key rel_key_base + r * dim + a is row a of R_r with
+ * row [R_r[a][0..dim) | G]; G are the AdaGrad accumulators (row_len = 2 * dim).
+ * Score phi = x_s^T R_r x_o; data points, negatives, loss and the AdaGrad push
+ * per distinct key of a data point are those of ps_step_kge.
+ * dim: a multiple of 4 from 4 to 128; n_neg <= 29; a call has
+ * (2 + n_neg + dim) * n key occurrences.  Device arrays as for ps_step_kge.
+ * Errors: PS_ERR_INVALID_ARG (null array, row_len != 2 * dim, rel_key_base past
+ * the keys), PS_ERR_UNSUPPORTED (dim or n_neg outside the limits),
+ * PS_ERR_WORKSPACE; an index out of range makes the call a no-op and latches
+ * PS_ERR_KEY_RANGE. */
+ps_status_t ps_step_rescal(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                           const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n,
+                           uint32_t n_neg, uint64_t rel_key_base, uint32_t dim, float lr, float eps,
+                           double* d_loss_accum, void* stream);
 
 /* One minibatch of skip-gram with negative sampling (Section 4.1, Appendix A).
  * Key w is the input vector of word w (w < out_key_base), key out_key_base + w

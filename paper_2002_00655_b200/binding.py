@@ -58,6 +58,7 @@ SIGNATURES = {
     "ps_localize_stats": (C.c_int, [_vp, _vp]),
     "ps_step_mf": (C.c_int, [_vp, _vp, _vp, _vp, _u64, _u64, _f32, _f32, _vp, _vp]),
     "ps_step_kge": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _u32, _f32, _f32, _vp, _vp]),
+    "ps_step_rescal": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _u32, _f32, _f32, _vp, _vp]),
     "ps_step_sgns": (C.c_int, [_vp, _vp, _u64, _u64, _u64, _u32, _vp, _u32, _u64, _f32, _vp, _vp]),
     "ps_step_mf_host": (C.c_int, [_vp, _vp, _vp, _vp, _u64, _u64, _f32, _f32, _vp, _vp, _vp]),
     "ps_step_kge_host": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _u32, _f32, _f32, _vp, _vp, _vp]),
@@ -216,6 +217,13 @@ def ps_step_kge(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n_neg, rel_key_base, d
                                       _dptr(d_neg_ent, _U32), _dptr(d_neg_side, _U8), d_s.numel(), n_neg,
                                       rel_key_base, dim_complex, lr, eps, _dptr(d_loss_accum, _F64), _stream()),
            "ps_step_kge")
+
+
+def ps_step_rescal(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n_neg, rel_key_base, dim, lr, eps, d_loss_accum=None):
+    _check(load_library().ps_step_rescal(ps, _dptr(d_s, _U32), _dptr(d_r, _U32), _dptr(d_o, _U32),
+                                         _dptr(d_neg_ent, _U32), _dptr(d_neg_side, _U8), d_s.numel(), n_neg,
+                                         rel_key_base, dim, lr, eps, _dptr(d_loss_accum, _F64), _stream()),
+           "ps_step_rescal")
 
 
 def ps_step_sgns(ps, d_tokens, first_pos, n_centers, window, d_negs, n_neg, out_key_base, lr, d_loss_accum=None):

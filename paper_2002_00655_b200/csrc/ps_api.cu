@@ -569,6 +569,31 @@ ps_status_t ps_step_kge(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r
     return release_set(ss, s);
 }
 
+ps_status_t ps_step_rescal(ps_store_t* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                           const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
+                           uint64_t rel_key_base, uint32_t dim, float lr, float eps, double* d_loss_accum,
+                           void* stream) {
+    PS_BEGIN_CALL(ps);
+    if (n == 0) return PS_OK;
+    if (!d_s || !d_r || !d_o || (n_neg && (!d_neg_ent || !d_neg_side))) return PS_ERR_INVALID_ARG;
+    if (n_neg > 29 || dim < 4 || dim > 128 || dim % 4 != 0) return PS_ERR_UNSUPPORTED;
+    if (ps->cfg.row_len != 2 * (uint64_t)dim) return PS_ERR_INVALID_ARG;
+    if ((2 + (uint64_t)n_neg + dim) * n > ps->max_keys) return PS_ERR_WORKSPACE;
+    if (rel_key_base > ps->cfg.num_keys) return PS_ERR_INVALID_ARG;
+    const uint32_t occ = (uint32_t)((2 + (uint64_t)n_neg + dim) * n);
+    SortSet* ss = next_set(ps);
+    if (!fork_side(ps, ss, s)) return PS_ERR_CUDA;
+    launch_keys_rescal(ps, d_s, d_r, d_o, d_neg_ent, n, n_neg, rel_key_base, dim, ps->side);
+    const int which = run_push_sort(ps, occ, ps->side);
+    if (!sorted_keys_at(ps, ss, which, occ)) return PS_ERR_CUDA;
+    // gradient rows of dim values per occurrence; AdaGrad inside the reduction, to which a row [dim | dim] is what
+    // [Re Im | G_Re G_Im] of dim / 2 complex dimensions is
+    const uint32_t lb = launch_grad_rescal(ps, d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, s);
+    if (!join_side(ps, s)) return PS_ERR_CUDA;
+    run_kge_reduce(ps, occ, which, dim / 2, lr, eps, d_loss_accum, d_loss_accum ? lb : 0, s);
+    return release_set(ss, s);
+}
+
 // ---- self-test of the bounded waits ----
 // Two blocks meet at the sort's grid barrier and wait for a third arrival that never comes.  The wait is bounded
 // (kBarrierSpins polls, about a fifth of a second): the blocks give up, latch PS_ERR_CUDA and return, leaving the

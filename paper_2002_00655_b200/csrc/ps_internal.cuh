@@ -247,6 +247,13 @@ void run_localize_deferred(ps_store* ps, uint32_t worker, uint32_t n, cudaStream
 // only, so they and the sort can run beside the gradient kernel); launch_step_* write the slots'
 // update rows to `upd` (launch_step_sgns: two source rows per center and one factor per slot, to be
 // reduced with run_push_reduce's d_scales) and return the number of per-block loss partials they wrote.
+// ---- rescal.cu ----
+void launch_keys_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                        const uint32_t* d_neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_key_base, uint32_t dim,
+                        cudaStream_t s);
+uint32_t launch_grad_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
+                            const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
+                            uint64_t rel_key_base, uint32_t dim, cudaStream_t s);
 void launch_keys_kge(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                      const uint32_t* d_neg_ent, uint64_t n, uint32_t n_neg, uint64_t rel_key_base, cudaStream_t s);
 void launch_keys_sgns(ps_store* ps, const uint32_t* d_tokens, uint64_t tok_first, uint64_t first_pos,
