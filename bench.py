@@ -576,6 +576,94 @@ class KGEWorkload:
         return n
 
 
+class RescalWorkload(KGEWorkload):
+    """RESCAL + AdaGrad (the paper's second knowledge-graph model, Section 4.1 / Table 4): triples/s through
+    ps_step_rescal.  A relation's d x d matrix is d keys of the store, so a data point has 2 + n_neg + d occurrences."""
+
+    def __init__(self, cfg):
+        super().__init__(cfg)
+
+    def describe(self):
+        c = self.cfg
+        return {"workload": c.name, "entities": c.entities, "relations": c.relations, "dim": c.dim,
+                "relation_matrix": f"{c.dim} x {c.dim} as {c.dim} keys", "negatives": c.n_neg, "minibatch": c.batch,
+                "store_gb": round(c.num_keys * c.row_len * 4 / 1e9, 2),
+                "l2": "inputs larger than L2 (random rows of the store; no flush between steps)"}
+
+    def _occ(self):
+        c = self.cfg
+        return (2 + c.n_neg + c.dim) * c.batch
+
+    def setup(self, ps, device, n_steps, keep_host_init):
+        c = self.cfg
+        self.ps = ps
+        self.store = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=self._occ(), device=device.index)
+        self.host_init = torch.empty((c.num_keys, c.row_len), dtype=torch.float32) if keep_host_init else None
+        chunk = max(1, (1 << 28) // (c.row_len * 4))
+        for s in range(0, c.num_keys, chunk):
+            n = min(chunk, c.num_keys - s)
+            rows = W.rescal_init_rows(c, s, n, device)
+            self.store.set_rows(torch.arange(s, s + n, dtype=torch.int64, device=device), rows)
+            if keep_host_init:
+                self.host_init[s:s + n] = rows.cpu()
+        self.s, self.r, self.o, self.neg, self.side = W.kge_triples(c, 0, n_steps * c.batch, device)
+        torch.cuda.synchronize(device)
+
+    def side_stream_kernels(self):
+        return ("sort_all_kernel", "rescal_keys")
+
+    def step(self, k):
+        c, sl = self.cfg, self._sl(k)
+        self.ps.ps_step_rescal(self.store.h, self.s[sl], self.r[sl], self.o[sl], self.neg[sl], self.side[sl], c.n_neg,
+                               c.rel_key_base, c.dim, c.lr, c.eps, self.store.loss)
+
+    def host_setup(self, steps):
+        return None                                 # (no host-batch entry point for this step)
+
+    def _distinct(self, sl):
+        return n_unique(self.s[sl], self.o[sl], self.neg[sl]) + n_unique(self.r[sl]) * self.cfg.dim
+
+    def alg_bytes(self, k):
+        c, sl, b = self.cfg, self._sl(k), self.cfg.batch
+        return b * (12 + c.n_neg * 5) + self._occ() * (8 + self.row_bytes) + self._distinct(sl) * 2 * self.row_bytes
+
+    def kernel_bytes(self, k, moved=0.0):
+        c, sl, b = self.cfg, self._sl(k), self.cfg.batch
+        u, occ, rb = self._distinct(sl), self._occ(), self.row_bytes
+        rows_of = (c.rel_key_base + self.r[sl].to(torch.int64)[:, None] * c.dim +
+                   torch.arange(c.dim, device=self.r.device, dtype=torch.int64)[None, :])
+        keys = torch.cat([t.reshape(-1).to(torch.int64) for t in (self.s[sl], self.o[sl], self.neg[sl])] + [rows_of.reshape(-1)])
+        kb = kernel_bytes_of_step(b * (12 + c.n_neg * 5), occ, u, rb, "rescal_keys", "rescal_grad",
+                                  int(c.num_keys).bit_length(), keys)
+        # the gradient kernel reads the value half of every row (the matrix once per data point) and writes a gradient
+        # row of the same size per occurrence; the reduction reads those and read-modify-writes every distinct row
+        kb["rescal_grad"] = b * (12 + c.n_neg * 5) + occ * (8 + rb // 2) + occ * (rb // 2)
+        kb["kge_reduce_kernel"] = occ * (8 + rb // 2) + u * (8 + 2 * rb)
+        return kb
+
+    def oracle_setup(self, device):
+        from oracle import OracleStore
+        c = self.cfg
+        o = OracleStore(c.num_keys, c.row_len, 1)
+        if getattr(self, "host_init", None) is not None:
+            o.set_rows(np.arange(c.num_keys), self.host_init.numpy())
+        else:
+            chunk = max(1, (1 << 28) // (c.row_len * 4))
+            for s in range(0, c.num_keys, chunk):
+                n = min(chunk, c.num_keys - s)
+                o.set_rows(np.arange(s, s + n), W.rescal_init_rows(c, s, n, device).cpu().numpy())
+        self.oracle = o
+        return o
+
+    def oracle_step(self, k, n):
+        c, b = self.cfg, self.cfg.batch
+        k = k % self.o_steps
+        sl = slice(k * b, k * b + n)
+        s, r, o, neg, side = (t[sl] for t in self.od)
+        self.oracle.step_rescal(s, r, o, neg, side, c.rel_key_base, c.dim, c.lr, c.eps)
+        return n
+
+
 class SGNSWorkload:
     """Skip-gram with negative sampling (Section 4.1 / Appendix A task): center words/s through ps_step_sgns."""
 
@@ -823,6 +911,7 @@ def make_workload(name):
              "mf_medium": lambda: MFWorkload(W.MF_MEDIUM),
              "kge": lambda: KGEWorkload(W.KGE), "kge_tiny": lambda: KGEWorkload(W.KGE_TINY),
              "kge_4000": lambda: KGEWorkload(W.KGE_4000, twin=W.KGE_4000_TWIN),
+             "rescal": lambda: RescalWorkload(W.RESCAL), "rescal_tiny": lambda: RescalWorkload(W.RESCAL_TINY),
              "sgns": lambda: SGNSWorkload(W.SGNS), "sgns_tiny": lambda: SGNSWorkload(W.SGNS_TINY),
              "stress": lambda: StressWorkload(W.STRESS), "stress_tiny": lambda: StressWorkload(W.STRESS_TINY),
              "stress_medium": lambda: StressWorkload(W.STRESS_MEDIUM)}
@@ -1155,7 +1244,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="mf_large",
-                    choices=["mf_dsgd", "mf_medium_dsgd", "keymap", "push_mf", "mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "kge_4000", "sgns", "sgns_tiny", "stress", "stress_tiny",
+                    choices=["mf_dsgd", "mf_medium_dsgd", "keymap", "push_mf", "mf_large", "mf_medium", "mf_tiny", "kge", "kge_tiny", "kge_4000", "rescal", "rescal_tiny", "sgns", "sgns_tiny", "stress", "stress_tiny",
                              "stress_medium"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--repeats", type=int, default=0,

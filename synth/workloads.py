@@ -256,6 +256,61 @@ def kge_triples(cfg: KGEConfig, start: int, count: int, device):
 
 
 # --------------------------------------------------------------------------
+# RESCAL (the paper's other knowledge-graph model: entity dimension d, a d x d matrix per relation)
+# --------------------------------------------------------------------------
+@dataclass(frozen=True)
+class RescalConfig:
+    """Triples come from kge_triples (same fields as KGEConfig).  All rows have one length, so a relation's matrix is
+    `dim` keys, one per matrix row; a row is [dim values | dim AdaGrad accumulators]."""
+    name: str
+    entities: int
+    relations: int
+    dim: int
+    n_triples: int
+    n_neg: int
+    batch: int
+    lr: float
+    eps: float
+    init_std: float
+    ent_zipf: float
+    seed: int = 0
+
+    @property
+    def num_keys(self) -> int:
+        return self.entities + self.relations * self.dim
+
+    @property
+    def row_len(self) -> int:
+        return 2 * self.dim
+
+    @property
+    def rel_key_base(self) -> int:
+        return self.entities
+
+    @property
+    def n_batches(self) -> int:
+        return (self.n_triples + self.batch - 1) // self.batch
+
+    def batch_range(self, b: int) -> tuple[int, int]:
+        s = b * self.batch
+        return s, min(self.batch, self.n_triples - s)
+
+
+# Stand-in for the paper's RESCAL task on DBpedia-500k (Table 4: 490,598 entities and 573 relations, entity dimension
+# 100, relation dimension 10,000, 10 negatives per triple): synthetic triples with Zipf entities, not the dataset.
+RESCAL = RescalConfig("rescal", 500_000, 573, 100, 3_000_000, 10, 8_192, 0.1, 1e-8, 0.1, 1.0)
+RESCAL_TINY = RescalConfig("rescal_tiny", 2_000, 7, 12, 3_000, 10, 128, 0.1, 1e-8, 0.1, 1.0)
+
+
+def rescal_init_rows(cfg: RescalConfig, key_start: int, count: int, device) -> torch.Tensor:
+    """Value halves N(0, init_std) (entities and matrix rows alike); AdaGrad accumulator halves zero."""
+    d = cfg.dim
+    idx = rng.counter(key_start * d, count * d, device)
+    emb = rng.normal(cfg.seed, _S_INIT, idx, cfg.init_std).to(torch.float32).view(count, d)
+    return torch.cat([emb, torch.zeros_like(emb)], dim=1).contiguous()
+
+
+# --------------------------------------------------------------------------
 # Skip-gram with negative sampling
 # --------------------------------------------------------------------------
 @dataclass(frozen=True)

@@ -167,6 +167,47 @@ def test_kge_steps():
     assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
 
 
+def test_rescal_steps():
+    """RESCAL at the bench's full size (500k entities, 573 relations of 100 x 100, 8,192 data points of 112 key
+    occurrences per step), pipelined: two single steps (the second from accumulators > 0), two steps back to back, the
+    ragged last batch; every touched row against the oracle, a sample of untouched rows bit-exact."""
+    c = W.RESCAL
+    need(4, 12)
+    g = ps.Store(c.num_keys, c.row_len, 1, max_batch_keys=(2 + c.n_neg + c.dim) * c.batch)
+    o = OracleStore(c.num_keys, c.row_len, 1)
+    fill_both(g, o, lambda s, n: W.rescal_init_rows(c, s, n, DEV), c.num_keys, chunk=1 << 18)
+    ps.ps_set_pipelining(g.h, True)
+
+    def run(first, n, steps):
+        d = W.kge_triples(c, first, n, DEV)
+        h = [t.cpu().numpy() for t in d]
+        for b in range(steps):
+            sl = slice(b * c.batch, min((b + 1) * c.batch, n))
+            ps.ps_step_rescal(g.h, *(t[sl] for t in d), c.n_neg, c.rel_key_base, c.dim, c.lr, c.eps, g.loss)
+        for b in range(steps):
+            sl = slice(b * c.batch, min((b + 1) * c.batch, n))
+            o.step_rescal(*(t[sl] for t in h), c.rel_key_base, c.dim, c.lr, c.eps)
+        g.sync()
+        s, r, t, neg, _ = h
+        rel_rows = (c.rel_key_base + np.unique(r).astype(np.int64)[:, None] * c.dim + np.arange(c.dim)[None, :]).ravel()
+        return np.concatenate([s, t, neg.ravel(), rel_rows])
+
+    for b in range(2):
+        touched = check_rows(g, o, run(b * c.batch, c.batch, 1), f"rescal, step {b}")
+        assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+        resync(g, o, touched)
+    acc0 = o.rows[:, c.dim:].copy()
+    keys2 = run(2 * c.batch, 2 * c.batch, 2)
+    touched = check_rows(g, o, keys2, "rescal, two steps in a row", loose=True, acc_before=acc0[np.unique(keys2.astype(np.int64))])
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+    check_untouched(g, o, touched, c.num_keys, "rescal")
+    resync(g, o, touched)
+    last, n_last = c.batch_range(c.n_batches - 1)
+    assert 0 < n_last < c.batch
+    check_rows(g, o, run(last, n_last, 1), "rescal, last batch")
+    assert close(loss_of(g), o.loss[0]), (loss_of(g), o.loss[0])
+
+
 def test_kge_4000_single_steps():
     """ComplEx with 4000 complex dimensions (the paper's ComplEx-Large: 8000 values and 8000 AdaGrad accumulators
     per key, 64 KB rows, a 32 GB store).  The oracle cannot hold the store, but a step reads and writes only the
