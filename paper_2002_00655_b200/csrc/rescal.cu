@@ -14,10 +14,13 @@
 // Slots that hold the same entity are folded into the first of them before anything is written (AdaGrad is taken on
 // the gradient with respect to each DISTINCT key), as the key kernel marks the later ones "no key".
 //
-// One block works on one data point at a time: R in shared memory (fp32, odd row stride), the vectors in fp64.  It
-// writes, per occurrence slot (2 + n_neg entity slots, then d matrix rows), the gradient row of d values; the
-// ComplEx path's reduction (kge_reduce_kernel: AdaGrad inside the segmented reduction of gradient rows) does the rest,
-// a row of [d | d] values being to it what [Re Im | G_Re G_Im] of d / 2 complex dimensions is.
+// One block of eight warps works on one data point at a time.  Warp w owns the matrix rows w, w + 8, ...: it loads
+// them once (a lane holds four consecutive values of each of its rows) and uses them from registers for all four
+// matrix-vector products: a row's dot product with a vector is summed over the lanes by shuffles, its contribution to
+// a product with the transpose is kept per lane and the eight warps' parts are added in warp order.  The vectors live
+// in shared memory in fp64.  Written per occurrence slot (2 + n_neg entity slots, then d matrix rows): the gradient
+// row of d values; the ComplEx path's reduction (kge_reduce_kernel: AdaGrad inside the segmented reduction of gradient
+// rows) does the rest, a row of [d | d] values being to it what [Re Im | G_Re G_Im] of d / 2 complex dimensions is.
 #include "ps_internal.cuh"
 
 namespace psb {
@@ -32,14 +35,19 @@ __device__ __forceinline__ double rescal_sigmoid(double z) {
 constexpr int kRescalThreads = 256;
 constexpr int kRescalMaxNeg = 29;
 
-// shared memory of a block: R (d rows of d + 1 floats), then fp64: the entity slots' vectors, their gradients,
-// u, w, a, b, b'
+// shared memory of a block, fp64: the entity slots' vectors, their gradients, u, w, a, b, b', and the warps' parts of
+// a product with the transpose
 __host__ __device__ inline size_t rescal_smem(uint32_t d, uint32_t n_neg) {
-    const size_t r = ((size_t)d * (d + 1) * sizeof(float) + 15) & ~(size_t)15;
-    return r + ((size_t)2 * (2 + n_neg) + 5) * d * sizeof(double);
+    return ((size_t)2 * (2 + n_neg) + 5 + kRescalThreads / 32) * d * sizeof(double);
 }
 
-__global__ void __launch_bounds__(kRescalThreads)
+struct d4r {
+    double x, y, z, w;
+};
+
+// kRows: matrix rows per warp, at least d / 8 rounded up
+template <int kRows>
+__global__ void __launch_bounds__(kRescalThreads, 2)
 rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                    const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
                    uint32_t n_neg, uint64_t rel_base, uint32_t d, const float* __restrict__ store,
@@ -50,19 +58,43 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
     __shared__ uint32_t s_key[2 + kRescalMaxNeg];
     __shared__ int s_rep[2 + kRescalMaxNeg];                // first slot that holds the same key
     __shared__ double s_coef[1 + kRescalMaxNeg];
+    __shared__ double s_loss[1 + kRescalMaxNeg];
     __shared__ int s_bad;
-    const uint32_t L = 2 * d, ld = d + 1;
+    constexpr int kWarps = kRescalThreads / 32;
+    const unsigned full = 0xffffffffu;
+    const uint32_t L = 2 * d, d4 = d / 4;
     const uint32_t n_ent = 2 + n_neg, n_slots = n_ent + d;
-    float* Rm = reinterpret_cast<float*>(smem_raw);
-    double* X = reinterpret_cast<double*>(smem_raw + (((size_t)d * ld * sizeof(float) + 15) & ~(size_t)15));   // [n_ent][d]
+    double* X = reinterpret_cast<double*>(smem_raw);        // [n_ent][d]
     double* Gs = X + (size_t)n_ent * d;                     // [n_ent][d]: gradient per entity slot
     double* U = Gs + (size_t)n_ent * d;
     double* Wv = U + d;
     double* A = Wv + d;
     double* B = A + d;
     double* Bp = B + d;
+    double* Wp = Bp + d;                                    // [kWarps][d]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool col = (uint32_t)lane < d4;                   // this lane holds columns 4 lane .. 4 lane + 3
     double loss = 0;                                        // thread 0's
+    // One pass over the warp's rows: dot[a] = row a . v (to out_dot) and this warp's part of sum_a s[a] row a (to Wp).
+    auto products = [&](const float4 (&R)[kRows], const double* v, const double* sc, double* out_dot) {
+        d4r vv = {0, 0, 0, 0}, part = {0, 0, 0, 0};
+        if (col) vv = d4r{v[4 * lane], v[4 * lane + 1], v[4 * lane + 2], v[4 * lane + 3]};
+#pragma unroll
+        for (int j = 0; j < kRows; ++j) {
+            const uint32_t a = warp + kWarps * j;
+            if (a >= d) break;                              // (the same for the whole warp)
+            const double rx = R[j].x, ry = R[j].y, rz = R[j].z, rw = R[j].w;
+            double p = rx * vv.x + ry * vv.y + rz * vv.z + rw * vv.w;
+            p = warp_sum_d(p);
+            if (lane == 0) out_dot[a] = p;
+            const double sa = sc[a];
+            part.x += sa * rx; part.y += sa * ry; part.z += sa * rz; part.w += sa * rw;
+        }
+        if (col) {
+            double* wp = Wp + (size_t)warp * d + 4 * lane;
+            wp[0] = part.x; wp[1] = part.y; wp[2] = part.z; wp[3] = part.w;
+        }
+    };
     for (uint64_t t = blockIdx.x; t < n; t += gridDim.x) {
         __syncthreads();                                    // the data point before is written out
         if (tid < (int)n_ent) {
@@ -70,8 +102,11 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
             s_key[tid] = k;
         }
         if (tid == 0) s_bad = 0;
-        __syncthreads();
         const uint64_t rk = rel_base + (uint64_t)tr[t] * d; // key of row 0 of the matrix
+        // the warp's rows of the matrix: their table entries now, the rows below (zeros beyond the last column)
+        uint64_t my_rrow = 0;
+        if (lane < kRows && warp + kWarps * lane < d && rk + d <= K) my_rrow = phys_row(table[rk + warp + kWarps * lane], S);
+        __syncthreads();
         if (tid < (int)n_ent) {
             if (s_key[tid] >= rel_base) s_bad = 1;
             int rep = tid;
@@ -83,34 +118,30 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
         __syncthreads();
         if (s_bad) continue;                                // the key kernel has latched the error; nothing is written
         if (tid < (int)n_ent) s_row[tid] = phys_row(table[s_key[tid]], S);
-        // the matrix: row a from the store row of key rk + a (one warp per row, in turn)
-        for (uint32_t a = warp; a < d; a += kRescalThreads / 32) {
-            const float* src = store + phys_row(table[rk + a], S) * L;
-            for (uint32_t b2 = lane; b2 < d; b2 += 32) Rm[a * ld + b2] = src[b2];
+        float4 R[kRows];
+#pragma unroll
+        for (int j = 0; j < kRows; ++j) {
+            const uint64_t rr = __shfl_sync(full, my_rrow, j);
+            R[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (warp + kWarps * j < d && col) R[j] = *reinterpret_cast<const float4*>(store + rr * L + 4 * lane);
         }
         __syncthreads();
-        for (uint32_t i = tid; i < n_ent * d; i += kRescalThreads) {
-            const uint32_t u = i / d, c = i - u * d;
-            X[i] = (double)store[s_row[u] * L + c];
-        }
+        for (uint32_t u = warp; u < n_ent; u += kWarps)
+            for (uint32_t c = lane; c < d; c += 32) X[(size_t)u * d + c] = (double)store[s_row[u] * L + c];
         __syncthreads();
         const double* xs = X;                               // slot 0: subject, slot 1: object
         const double* xo = X + d;
-        // u = R x_o (thread per row), w = R^T x_s (thread per column)
-        for (uint32_t i = tid; i < 2 * d; i += kRescalThreads) {
-            double acc = 0;
-            if (i < d) {
-                for (uint32_t b2 = 0; b2 < d; ++b2) acc += (double)Rm[i * ld + b2] * xo[b2];
-                U[i] = acc;
-            } else {
-                const uint32_t b2 = i - d;
-                for (uint32_t a = 0; a < d; ++a) acc += xs[a] * (double)Rm[a * ld + b2];
-                Wv[b2] = acc;
-            }
+        // u = R x_o and the parts of w = R^T x_s
+        products(R, xo, xs, U);
+        __syncthreads();
+        for (uint32_t c = tid; c < d; c += kRescalThreads) {
+            double acc = Wp[c];
+            for (int w2 = 1; w2 < kWarps; ++w2) acc += Wp[(size_t)w2 * d + c];
+            Wv[c] = acc;
         }
         __syncthreads();
         // scores, one warp per triple of the data point (q = 0: the positive)
-        for (uint32_t q = warp; q <= n_neg; q += kRescalThreads / 32) {
+        for (uint32_t q = warp; q <= n_neg; q += kWarps) {
             const double* lhs = xs;
             const double* rhs = U;                          // x . u: the positive and the subject-negatives
             if (q > 0) {
@@ -123,14 +154,12 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
             if (lane == 0) {
                 const double y = q == 0 ? 1.0 : -1.0;
                 s_coef[q] = -y * rescal_sigmoid(-y * p);
-                // (the loss terms are added by thread 0 below, in the order of the triples)
-                Gs[q] = rescal_softplus(-y * p);            // parked in the gradient area, which is written after the sync
+                s_loss[q] = rescal_softplus(-y * p);        // (added by thread 0 below, in the order of the triples)
             }
         }
         __syncthreads();
         if (tid == 0)
-            for (uint32_t q = 0; q <= n_neg; ++q) loss += Gs[q];
-        __syncthreads();
+            for (uint32_t q = 0; q <= n_neg; ++q) loss += s_loss[q];
         // a, b', b
         for (uint32_t i = tid; i < 2 * d; i += kRescalThreads) {
             const bool is_a = i < d;
@@ -144,37 +173,48 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
             else { Bp[c] = acc; B[c] = s_coef[0] * xo[c] + acc; }
         }
         __syncthreads();
-        // gradients per entity slot: subject R b, object R^T a, negatives c_k u or c_k w
-        for (uint32_t i = tid; i < n_ent * d; i += kRescalThreads) {
-            const uint32_t u = i / d, c = i - u * d;
-            double g;
-            if (u == 0) {
-                g = 0;
-                for (uint32_t b2 = 0; b2 < d; ++b2) g += (double)Rm[c * ld + b2] * B[b2];
-            } else if (u == 1) {
-                g = 0;
-                for (uint32_t a = 0; a < d; ++a) g += A[a] * (double)Rm[a * ld + c];
-            } else {
-                g = s_coef[u - 1] * (neg_side[t * n_neg + u - 2] == 0 ? U[c] : Wv[c]);
-            }
-            Gs[i] = g;
+        // gradients per entity slot: subject R b, the parts of the object's R^T a, negatives c_k u or c_k w
+        products(R, B, A, Gs);
+        for (uint32_t u = 2 + warp; u < n_ent; u += kWarps) {
+            const double ck = s_coef[u - 1];
+            const double* from = neg_side[t * n_neg + u - 2] == 0 ? U : Wv;
+            for (uint32_t c = lane; c < d; c += 32) Gs[(size_t)u * d + c] = ck * from[c];
+        }
+        __syncthreads();
+        for (uint32_t c = tid; c < d; c += kRescalThreads) {
+            double acc = Wp[c];
+            for (int w2 = 1; w2 < kWarps; ++w2) acc += Wp[(size_t)w2 * d + c];
+            Gs[d + c] = acc;
         }
         __syncthreads();
         // entity gradient rows: slots with the same key folded into the first, in slot order
         float* out = grad + (uint64_t)t * n_slots * d;
-        for (uint32_t i = tid; i < n_ent * d; i += kRescalThreads) {
-            const uint32_t u = i / d, c = i - u * d;
+        for (uint32_t u = warp; u < n_ent; u += kWarps) {
             if (s_rep[u] != (int)u) continue;
-            double g = Gs[i];
-            for (uint32_t z = u + 1; z < n_ent; ++z)
-                if (s_rep[z] == (int)u) g += Gs[(size_t)z * d + c];
-            out[i] = (float)g;
+            for (uint32_t c = lane; c < d; c += 32) {
+                double g = Gs[(size_t)u * d + c];
+                for (uint32_t z = u + 1; z < n_ent; ++z)
+                    if (s_rep[z] == (int)u) g += Gs[(size_t)z * d + c];
+                out[(size_t)u * d + c] = (float)g;
+            }
         }
         // matrix rows: a[alpha] x_o + x_s[alpha] b'
         float* outR = out + (uint64_t)n_ent * d;
-        for (uint32_t i = tid; i < d * d; i += kRescalThreads) {
-            const uint32_t al = i / d, be = i - al * d;
-            outR[i] = (float)(A[al] * xo[be] + xs[al] * Bp[be]);
+        if (col) {
+            const d4r o4 = {xo[4 * lane], xo[4 * lane + 1], xo[4 * lane + 2], xo[4 * lane + 3]};
+            const d4r b4 = {Bp[4 * lane], Bp[4 * lane + 1], Bp[4 * lane + 2], Bp[4 * lane + 3]};
+#pragma unroll
+            for (int j = 0; j < kRows; ++j) {
+                const uint32_t al = warp + kWarps * j;
+                if (al >= d) break;
+                const double aa = A[al], sa = xs[al];
+                float4 g;
+                g.x = (float)(aa * o4.x + sa * b4.x);
+                g.y = (float)(aa * o4.y + sa * b4.y);
+                g.z = (float)(aa * o4.z + sa * b4.z);
+                g.w = (float)(aa * o4.w + sa * b4.w);
+                *reinterpret_cast<float4*>(outR + (size_t)al * d + 4 * lane) = g;
+            }
         }
     }
     if (tid == 0) loss_partial[blockIdx.x] = loss;
@@ -221,19 +261,25 @@ void launch_keys_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, 
 uint32_t launch_grad_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                             const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
                             uint64_t rel_key_base, uint32_t dim, cudaStream_t s) {
-    static std::atomic<unsigned long long> smem_set{0};
     const size_t smem = rescal_smem(dim, n_neg);
-    opt_in_smem((const void*)rescal_grad_kernel, rescal_smem(128, kRescalMaxNeg), &smem_set);
-    // as many blocks as the device holds at this size (shared memory decides), at most one per data point
-    const uint32_t per_sm = (uint32_t)tmax<size_t>(1, tmin<size_t>(8, (size_t)(220 * 1024) / (smem + 2048)));
-    uint64_t g = tmin<uint64_t>(n, (uint64_t)ps->sm_count * per_sm);
+    // two blocks per SM (registers: the warps hold the matrix), at most one block per data point
+    uint64_t g = tmin<uint64_t>(n, (uint64_t)ps->sm_count * 2);
     if (g > kMaxLossBlocks) g = kMaxLossBlocks;
     const uint32_t grid = (uint32_t)g;
-    if (ps->prof) prof_before(ps, "rescal_grad_kernel", s);
-    rescal_grad_kernel<<<grid, kRescalThreads, smem, s>>>(d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base,
-                                                         dim, (const float*)ps->store, ps->table,
-                                                         ps->cfg.slots_per_part, ps->cfg.num_keys, (float*)ps->upd,
-                                                         ps->loss_partial);
+#define RESCAL_LAUNCH(kRows)                                                                                        \
+    do {                                                                                                            \
+        static std::atomic<unsigned long long> smem_set{0};                                                         \
+        opt_in_smem((const void*)rescal_grad_kernel<kRows>, rescal_smem(128, kRescalMaxNeg), &smem_set);            \
+        if (ps->prof) prof_before(ps, "rescal_grad_kernel<" #kRows ">", s);                                         \
+        rescal_grad_kernel<kRows><<<grid, kRescalThreads, smem, s>>>(                                               \
+            d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, (const float*)ps->store, ps->table,  \
+            ps->cfg.slots_per_part, ps->cfg.num_keys, (float*)ps->upd, ps->loss_partial);                          \
+    } while (0)
+    if (dim <= 32) RESCAL_LAUNCH(4);
+    else if (dim <= 64) RESCAL_LAUNCH(8);
+    else if (dim <= 104) RESCAL_LAUNCH(13);
+    else RESCAL_LAUNCH(16);
+#undef RESCAL_LAUNCH
     if (ps->prof) prof_after(ps, s);
     ps->launches++;
     return grid;
