@@ -14,13 +14,16 @@
 // Slots that hold the same entity are folded into the first of them before anything is written (AdaGrad is taken on
 // the gradient with respect to each DISTINCT key), as the key kernel marks the later ones "no key".
 //
-// One block of eight warps works on one data point at a time.  Warp w owns the matrix rows w, w + 8, ...: it loads
-// them once (a lane holds four consecutive values of each of its rows) and uses them from registers for all four
-// matrix-vector products: a row's dot product with a vector is summed over the lanes by shuffles, its contribution to
-// a product with the transpose is kept per lane and the eight warps' parts are added in warp order.  The vectors live
-// in shared memory in fp64.  Written per occurrence slot (2 + n_neg entity slots, then d matrix rows): the gradient
-// row of d values; the ComplEx path's reduction (kge_reduce_kernel: AdaGrad inside the segmented reduction of gradient
-// rows) does the rest, a row of [d | d] values being to it what [Re Im | G_Re G_Im] of d / 2 complex dimensions is.
+// One WARP works on one data point at a time, with no block-wide synchronisation (a block of eight warps per data
+// point, the matrix in shared memory or in registers, spent its time in a dozen dependent phases: 660-700 us per
+// step of 8,192 data points).  Lane l holds elements l, l + 32, l + 64, l + 96 of every vector, in fp64.  A product
+// with R takes a lane per row (the lane reads its rows front to back, the vector comes from shared memory as
+// broadcasts), a product with R^T a lane per column (row by row, coalesced); neither needs a sum across lanes.
+// The gradient of an entity slot is c1 (R b) + c2 (R^T a) + c3 u + c4 w with four numbers per slot, so slots that
+// hold the same entity are folded by adding their numbers, and no gradient is stored before it is final.  Written per
+// occurrence slot (2 + n_neg entity slots, then d matrix rows): the gradient row of d values; the ComplEx path's
+// reduction (kge_reduce_kernel: AdaGrad inside the segmented reduction of gradient rows) does the rest, a row of
+// [d | d] values being to it what [Re Im | G_Re G_Im] of d / 2 complex dimensions is.
 #include "ps_internal.cuh"
 
 namespace psb {
@@ -35,18 +38,11 @@ __device__ __forceinline__ double rescal_sigmoid(double z) {
 constexpr int kRescalThreads = 256;
 constexpr int kRescalMaxNeg = 29;
 
-// shared memory of a block, fp64: the entity slots' vectors, their gradients, u, w, a, b, b', and the warps' parts of
-// a product with the transpose
-__host__ __device__ inline size_t rescal_smem(uint32_t d, uint32_t n_neg) {
-    return ((size_t)2 * (2 + n_neg) + 5 + kRescalThreads / 32) * d * sizeof(double);
-}
+// shared memory of a warp, fp64: x_o, x_s, b, a (read as broadcasts by the lanes)
+__host__ __device__ inline size_t rescal_smem(uint32_t d) { return (size_t)(kRescalThreads / 32) * 4 * d * sizeof(double); }
 
-struct d4r {
-    double x, y, z, w;
-};
-
-// kRows: matrix rows per warp, at least d / 8 rounded up
-template <int kRows>
+// kE: elements of a vector per lane, d <= 32 kE
+template <int kE>
 __global__ void __launch_bounds__(kRescalThreads, 2)
 rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__ tr, const uint32_t* __restrict__ to,
                    const uint32_t* __restrict__ neg_ent, const uint8_t* __restrict__ neg_side, uint64_t n,
@@ -54,170 +50,169 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
                    const uint2* __restrict__ table, uint64_t S, uint64_t K, float* __restrict__ grad,
                    double* __restrict__ loss_partial) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ uint64_t s_row[2 + kRescalMaxNeg];           // store row of each entity slot
-    __shared__ uint32_t s_key[2 + kRescalMaxNeg];
-    __shared__ int s_rep[2 + kRescalMaxNeg];                // first slot that holds the same key
-    __shared__ double s_coef[1 + kRescalMaxNeg];
-    __shared__ double s_loss[1 + kRescalMaxNeg];
-    __shared__ int s_bad;
+    __shared__ double s_wl[kRescalThreads / 32];
     constexpr int kWarps = kRescalThreads / 32;
     const unsigned full = 0xffffffffu;
     const uint32_t L = 2 * d, d4 = d / 4;
     const uint32_t n_ent = 2 + n_neg, n_slots = n_ent + d;
-    double* X = reinterpret_cast<double*>(smem_raw);        // [n_ent][d]
-    double* Gs = X + (size_t)n_ent * d;                     // [n_ent][d]: gradient per entity slot
-    double* U = Gs + (size_t)n_ent * d;
-    double* Wv = U + d;
-    double* A = Wv + d;
-    double* B = A + d;
-    double* Bp = B + d;
-    double* Wp = Bp + d;                                    // [kWarps][d]
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool col = (uint32_t)lane < d4;                   // this lane holds columns 4 lane .. 4 lane + 3
-    double loss = 0;                                        // thread 0's
-    // One pass over the warp's rows: dot[a] = row a . v (to out_dot) and this warp's part of sum_a s[a] row a (to Wp).
-    auto products = [&](const float4 (&R)[kRows], const double* v, const double* sc, double* out_dot) {
-        d4r vv = {0, 0, 0, 0}, part = {0, 0, 0, 0};
-        if (col) vv = d4r{v[4 * lane], v[4 * lane + 1], v[4 * lane + 2], v[4 * lane + 3]};
-#pragma unroll
-        for (int j = 0; j < kRows; ++j) {
-            const uint32_t a = warp + kWarps * j;
-            if (a >= d) break;                              // (the same for the whole warp)
-            const double rx = R[j].x, ry = R[j].y, rz = R[j].z, rw = R[j].w;
-            double p = rx * vv.x + ry * vv.y + rz * vv.z + rw * vv.w;
-            p = warp_sum_d(p);
-            if (lane == 0) out_dot[a] = p;
-            const double sa = sc[a];
-            part.x += sa * rx; part.y += sa * ry; part.z += sa * rz; part.w += sa * rw;
-        }
-        if (col) {
-            double* wp = Wp + (size_t)warp * d + 4 * lane;
-            wp[0] = part.x; wp[1] = part.y; wp[2] = part.z; wp[3] = part.w;
-        }
-    };
-    for (uint64_t t = blockIdx.x; t < n; t += gridDim.x) {
-        __syncthreads();                                    // the data point before is written out
-        if (tid < (int)n_ent) {
-            const uint32_t k = tid == 0 ? ts[t] : (tid == 1 ? to[t] : neg_ent[t * n_neg + (tid - 2)]);
-            s_key[tid] = k;
-        }
-        if (tid == 0) s_bad = 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double* sxo = reinterpret_cast<double*>(smem_raw) + (size_t)warp * 4 * d;
+    double* sxs = sxo + d;
+    double* sB = sxs + d;
+    double* sA = sB + d;
+    const uint64_t n_warps = (uint64_t)gridDim.x * kWarps;
+    double loss = 0;                                        // lane 0's
+    for (uint64_t t = (uint64_t)blockIdx.x * kWarps + warp; t < n; t += n_warps) {
+        // entity slots: subject, object, negatives (lane u holds slot u)
+        uint32_t key = 0;
+        if (lane < (int)n_ent) key = lane == 0 ? ts[t] : (lane == 1 ? to[t] : neg_ent[t * n_neg + (lane - 2)]);
+        const uint32_t side = (lane >= 2 && lane < (int)n_ent) ? neg_side[t * n_neg + (lane - 2)] : 0u;
         const uint64_t rk = rel_base + (uint64_t)tr[t] * d; // key of row 0 of the matrix
-        // the warp's rows of the matrix: their table entries now, the rows below (zeros beyond the last column)
-        uint64_t my_rrow = 0;
-        if (lane < kRows && warp + kWarps * lane < d && rk + d <= K) my_rrow = phys_row(table[rk + warp + kWarps * lane], S);
-        __syncthreads();
-        if (tid < (int)n_ent) {
-            if (s_key[tid] >= rel_base) s_bad = 1;
-            int rep = tid;
-            for (int z = tid - 1; z >= 0; --z)
-                if (s_key[z] == s_key[tid]) rep = z;
-            s_rep[tid] = rep;
+        if (__ballot_sync(full, lane < (int)n_ent && key >= rel_base) != 0u || rk + d > K) continue;   // (latched by the key kernel)
+        int rep = lane;                                     // first slot that holds the same key
+        for (int z = 0; z < (int)n_ent; ++z) {
+            const uint32_t kz = __shfl_sync(full, key, z);
+            if (lane < (int)n_ent && kz == key && z < rep) rep = z;
         }
-        if (tid == 0 && rk + d > K) s_bad = 1;
-        __syncthreads();
-        if (s_bad) continue;                                // the key kernel has latched the error; nothing is written
-        if (tid < (int)n_ent) s_row[tid] = phys_row(table[s_key[tid]], S);
-        float4 R[kRows];
+        uint64_t erow = 0;
+        if (lane < (int)n_ent) erow = phys_row(table[key], S);
+        // rows of the matrix this lane owns, and its elements of x_s and x_o
+        const float* rowp[kE];
+        double xs[kE], xo[kE];
+        const float* ps_ = store + __shfl_sync(full, erow, 0) * L;
+        const float* po_ = store + __shfl_sync(full, erow, 1) * L;
 #pragma unroll
-        for (int j = 0; j < kRows; ++j) {
-            const uint64_t rr = __shfl_sync(full, my_rrow, j);
-            R[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (warp + kWarps * j < d && col) R[j] = *reinterpret_cast<const float4*>(store + rr * L + 4 * lane);
-        }
-        __syncthreads();
-        for (uint32_t u = warp; u < n_ent; u += kWarps)
-            for (uint32_t c = lane; c < d; c += 32) X[(size_t)u * d + c] = (double)store[s_row[u] * L + c];
-        __syncthreads();
-        const double* xs = X;                               // slot 0: subject, slot 1: object
-        const double* xo = X + d;
-        // u = R x_o and the parts of w = R^T x_s
-        products(R, xo, xs, U);
-        __syncthreads();
-        for (uint32_t c = tid; c < d; c += kRescalThreads) {
-            double acc = Wp[c];
-            for (int w2 = 1; w2 < kWarps; ++w2) acc += Wp[(size_t)w2 * d + c];
-            Wv[c] = acc;
-        }
-        __syncthreads();
-        // scores, one warp per triple of the data point (q = 0: the positive)
-        for (uint32_t q = warp; q <= n_neg; q += kWarps) {
-            const double* lhs = xs;
-            const double* rhs = U;                          // x . u: the positive and the subject-negatives
-            if (q > 0) {
-                if (neg_side[t * n_neg + q - 1] == 0) lhs = X + (size_t)(2 + q - 1) * d;
-                else { lhs = Wv; rhs = X + (size_t)(2 + q - 1) * d; }
+        for (int k = 0; k < kE; ++k) {
+            const uint32_t e = lane + 32 * k;
+            rowp[k] = store;
+            xs[k] = xo[k] = 0;
+            if (e < d) {
+                rowp[k] = store + phys_row(table[rk + e], S) * L;
+                xs[k] = (double)ps_[e];
+                xo[k] = (double)po_[e];
             }
+        }
+        __syncwarp();                                       // the data point before is done with the warp's shared memory
+#pragma unroll
+        for (int k = 0; k < kE; ++k) {
+            const uint32_t e = lane + 32 * k;
+            if (e < d) { sxo[e] = xo[k]; sxs[e] = xs[k]; }
+        }
+        __syncwarp();
+        // v = R y (lane per row) and z = R^T s (lane per column), y and s in shared memory
+        auto products = [&](const double* sy, const double* ss, double (&v)[kE], double (&z)[kE]) {
+#pragma unroll
+            for (int k = 0; k < kE; ++k) v[k] = z[k] = 0;
+            for (uint32_t b4 = 0; b4 < d4; ++b4) {
+                const double2 y01 = *reinterpret_cast<const double2*>(sy + 4 * b4);
+                const double2 y23 = *reinterpret_cast<const double2*>(sy + 4 * b4 + 2);
+#pragma unroll
+                for (int k = 0; k < kE; ++k) {
+                    if ((uint32_t)(lane + 32 * k) < d) {
+                        const float4 r = *reinterpret_cast<const float4*>(rowp[k] + 4 * b4);
+                        v[k] += (double)r.x * y01.x + (double)r.y * y01.y + (double)r.z * y23.x + (double)r.w * y23.y;
+                    }
+                }
+            }
+            for (uint32_t a0 = 0; a0 < d; a0 += 32) {
+#pragma unroll
+                for (int kk = 0; kk < kE; ++kk) {
+                    if (a0 != 32u * kk) continue;           // the rows a0 .. a0 + 31 are the lanes' rows number kk
+                    const uint32_t cnt = d - a0 < 32u ? d - a0 : 32u;
+                    for (uint32_t j = 0; j < cnt; ++j) {
+                        const float* ra = reinterpret_cast<const float*>(__shfl_sync(full, (unsigned long long)rowp[kk], j));
+                        const double sa = ss[a0 + j];
+#pragma unroll
+                        for (int k = 0; k < kE; ++k)
+                            if ((uint32_t)(lane + 32 * k) < d) z[k] += sa * (double)ra[lane + 32 * k];
+                    }
+                }
+            }
+        };
+        double u[kE], w[kE];
+        products(sxo, sxs, u, w);
+        // scores and their coefficients, one triple after the other; a, b' as they come
+        double av[kE], bp[kE];
+        double phi = 0;
+#pragma unroll
+        for (int k = 0; k < kE; ++k) phi += xs[k] * u[k];
+        phi = warp_sum_d(phi);
+        const double c_pos = -rescal_sigmoid(-phi);
+        double my_coef = 0;                                 // lane 2 + q: the coefficient of negative q
+        double lsum = rescal_softplus(-phi);
+#pragma unroll
+        for (int k = 0; k < kE; ++k) { av[k] = c_pos * xs[k]; bp[k] = 0; }
+        for (uint32_t q = 0; q < n_neg; ++q) {
+            const float* pk = store + __shfl_sync(full, erow, 2 + q) * L;
+            const bool subj = __shfl_sync(full, side, 2 + q) == 0u;
+            double xk[kE];
             double p = 0;
-            for (uint32_t c = lane; c < d; c += 32) p += lhs[c] * rhs[c];
+#pragma unroll
+            for (int k = 0; k < kE; ++k) {
+                const uint32_t e = lane + 32 * k;
+                xk[k] = e < d ? (double)pk[e] : 0.0;
+                p += xk[k] * (subj ? u[k] : w[k]);
+            }
             p = warp_sum_d(p);
-            if (lane == 0) {
-                const double y = q == 0 ? 1.0 : -1.0;
-                s_coef[q] = -y * rescal_sigmoid(-y * p);
-                s_loss[q] = rescal_softplus(-y * p);        // (added by thread 0 below, in the order of the triples)
+            const double cq = rescal_sigmoid(p);            // y = -1: d softplus(phi) / d phi
+            lsum += rescal_softplus(p);
+            if (lane == (int)(2 + q)) my_coef = cq;
+#pragma unroll
+            for (int k = 0; k < kE; ++k) {
+                if (subj) av[k] += cq * xk[k];
+                else bp[k] += cq * xk[k];
             }
         }
-        __syncthreads();
-        if (tid == 0)
-            for (uint32_t q = 0; q <= n_neg; ++q) loss += s_loss[q];
-        // a, b', b
-        for (uint32_t i = tid; i < 2 * d; i += kRescalThreads) {
-            const bool is_a = i < d;
-            const uint32_t c = is_a ? i : i - d;
-            double acc = 0;
-            for (uint32_t q = 1; q <= n_neg; ++q) {
-                const bool subj = neg_side[t * n_neg + q - 1] == 0;
-                if (subj == is_a) acc += s_coef[q] * X[(size_t)(2 + q - 1) * d + c];
-            }
-            if (is_a) A[c] = s_coef[0] * xs[c] + acc;
-            else { Bp[c] = acc; B[c] = s_coef[0] * xo[c] + acc; }
+        if (lane == 0) loss += lsum;
+#pragma unroll
+        for (int k = 0; k < kE; ++k) {
+            const uint32_t e = lane + 32 * k;
+            if (e < d) { sB[e] = c_pos * xo[k] + bp[k]; sA[e] = av[k]; }
         }
-        __syncthreads();
-        // gradients per entity slot: subject R b, the parts of the object's R^T a, negatives c_k u or c_k w
-        products(R, B, A, Gs);
-        for (uint32_t u = 2 + warp; u < n_ent; u += kWarps) {
-            const double ck = s_coef[u - 1];
-            const double* from = neg_side[t * n_neg + u - 2] == 0 ? U : Wv;
-            for (uint32_t c = lane; c < d; c += 32) Gs[(size_t)u * d + c] = ck * from[c];
+        __syncwarp();
+        double gs[kE], go[kE];
+        products(sB, sA, gs, go);                           // R b, R^T a
+        // the four numbers of every slot, folded into the first slot of its key (lane v: the numbers of slot v)
+        double c1 = 0, c2 = 0, c3 = 0, c4 = 0;
+        for (int z = 0; z < (int)n_ent; ++z) {
+            const int rz = __shfl_sync(full, rep, z);
+            const double cz = __shfl_sync(full, my_coef, z);
+            const uint32_t sz = __shfl_sync(full, side, z);
+            if (rz != lane) continue;
+            if (z == 0) c1 += 1.0;
+            else if (z == 1) c2 += 1.0;
+            else if (sz == 0u) c3 += cz;
+            else c4 += cz;
         }
-        __syncthreads();
-        for (uint32_t c = tid; c < d; c += kRescalThreads) {
-            double acc = Wp[c];
-            for (int w2 = 1; w2 < kWarps; ++w2) acc += Wp[(size_t)w2 * d + c];
-            Gs[d + c] = acc;
-        }
-        __syncthreads();
-        // entity gradient rows: slots with the same key folded into the first, in slot order
         float* out = grad + (uint64_t)t * n_slots * d;
-        for (uint32_t u = warp; u < n_ent; u += kWarps) {
-            if (s_rep[u] != (int)u) continue;
-            for (uint32_t c = lane; c < d; c += 32) {
-                double g = Gs[(size_t)u * d + c];
-                for (uint32_t z = u + 1; z < n_ent; ++z)
-                    if (s_rep[z] == (int)u) g += Gs[(size_t)z * d + c];
-                out[(size_t)u * d + c] = (float)g;
+        for (int v = 0; v < (int)n_ent; ++v) {
+            if (__shfl_sync(full, rep, v) != v) continue;   // a later slot of a key: marked "no key", never read
+            const double f1 = __shfl_sync(full, c1, v), f2 = __shfl_sync(full, c2, v);
+            const double f3 = __shfl_sync(full, c3, v), f4 = __shfl_sync(full, c4, v);
+#pragma unroll
+            for (int k = 0; k < kE; ++k) {
+                const uint32_t e = lane + 32 * k;
+                if (e < d) out[(size_t)v * d + e] = (float)(f1 * gs[k] + f2 * go[k] + f3 * u[k] + f4 * w[k]);
             }
         }
         // matrix rows: a[alpha] x_o + x_s[alpha] b'
         float* outR = out + (uint64_t)n_ent * d;
-        if (col) {
-            const d4r o4 = {xo[4 * lane], xo[4 * lane + 1], xo[4 * lane + 2], xo[4 * lane + 3]};
-            const d4r b4 = {Bp[4 * lane], Bp[4 * lane + 1], Bp[4 * lane + 2], Bp[4 * lane + 3]};
+        for (uint32_t al = 0; al < d; ++al) {
+            const double aa = sA[al], sa = sxs[al];
 #pragma unroll
-            for (int j = 0; j < kRows; ++j) {
-                const uint32_t al = warp + kWarps * j;
-                if (al >= d) break;
-                const double aa = A[al], sa = xs[al];
-                float4 g;
-                g.x = (float)(aa * o4.x + sa * b4.x);
-                g.y = (float)(aa * o4.y + sa * b4.y);
-                g.z = (float)(aa * o4.z + sa * b4.z);
-                g.w = (float)(aa * o4.w + sa * b4.w);
-                *reinterpret_cast<float4*>(outR + (size_t)al * d + 4 * lane) = g;
+            for (int k = 0; k < kE; ++k) {
+                const uint32_t e = lane + 32 * k;
+                if (e < d) outR[(size_t)al * d + e] = (float)(aa * xo[k] + sa * bp[k]);
             }
         }
     }
-    if (tid == 0) loss_partial[blockIdx.x] = loss;
+    if (lane == 0) s_wl[warp] = loss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double tot = 0;
+        for (int i = 0; i < kWarps; ++i) tot += s_wl[i];
+        loss_partial[blockIdx.x] = tot;
+    }
 }
 
 // Keys of the occurrence slots: 2 + n_neg entity slots (a slot that repeats an earlier slot's key gets the "no key"
@@ -261,24 +256,22 @@ void launch_keys_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, 
 uint32_t launch_grad_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d_r, const uint32_t* d_o,
                             const uint32_t* d_neg_ent, const uint8_t* d_neg_side, uint64_t n, uint32_t n_neg,
                             uint64_t rel_key_base, uint32_t dim, cudaStream_t s) {
-    const size_t smem = rescal_smem(dim, n_neg);
-    // two blocks per SM (registers: the warps hold the matrix), at most one block per data point
-    uint64_t g = tmin<uint64_t>(n, (uint64_t)ps->sm_count * 2);
+    const size_t smem = rescal_smem(dim);
+    (void)n_neg;
+    // two blocks per SM, a warp per data point at a time
+    uint64_t g = tmin<uint64_t>((n + 7) / 8, (uint64_t)ps->sm_count * 2);
     if (g > kMaxLossBlocks) g = kMaxLossBlocks;
     const uint32_t grid = (uint32_t)g;
-#define RESCAL_LAUNCH(kRows)                                                                                        \
+#define RESCAL_LAUNCH(kE)                                                                                           \
     do {                                                                                                            \
-        static std::atomic<unsigned long long> smem_set{0};                                                         \
-        opt_in_smem((const void*)rescal_grad_kernel<kRows>, rescal_smem(128, kRescalMaxNeg), &smem_set);            \
-        if (ps->prof) prof_before(ps, "rescal_grad_kernel<" #kRows ">", s);                                         \
-        rescal_grad_kernel<kRows><<<grid, kRescalThreads, smem, s>>>(                                               \
+        if (ps->prof) prof_before(ps, "rescal_grad_kernel<" #kE ">", s);                                            \
+        rescal_grad_kernel<kE><<<grid, kRescalThreads, smem, s>>>(                                                  \
             d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, (const float*)ps->store, ps->table,  \
             ps->cfg.slots_per_part, ps->cfg.num_keys, (float*)ps->upd, ps->loss_partial);                          \
     } while (0)
-    if (dim <= 32) RESCAL_LAUNCH(4);
-    else if (dim <= 64) RESCAL_LAUNCH(8);
-    else if (dim <= 104) RESCAL_LAUNCH(13);
-    else RESCAL_LAUNCH(16);
+    if (dim <= 32) RESCAL_LAUNCH(1);
+    else if (dim <= 64) RESCAL_LAUNCH(2);
+    else RESCAL_LAUNCH(4);
 #undef RESCAL_LAUNCH
     if (ps->prof) prof_after(ps, s);
     ps->launches++;
