@@ -38,8 +38,10 @@ __device__ __forceinline__ double rescal_sigmoid(double z) {
 constexpr int kRescalThreads = 256;
 constexpr int kRescalMaxNeg = 29;
 
-// shared memory of a warp, fp64: x_o, x_s, b, a (read as broadcasts by the lanes)
-__host__ __device__ inline size_t rescal_smem(uint32_t d) { return (size_t)(kRescalThreads / 32) * 4 * d * sizeof(double); }
+// shared memory of a warp, fp64: x_s and a (read as broadcasts by the lanes), and a 32 x 33 tile
+__host__ __device__ inline size_t rescal_smem(uint32_t d) {
+    return (size_t)(kRescalThreads / 32) * (2 * d + 32 * 33) * sizeof(double);
+}
 
 // kE: elements of a vector per lane, d <= 32 kE
 template <int kE>
@@ -53,13 +55,12 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
     __shared__ double s_wl[kRescalThreads / 32];
     constexpr int kWarps = kRescalThreads / 32;
     const unsigned full = 0xffffffffu;
-    const uint32_t L = 2 * d, d4 = d / 4;
+    const uint32_t L = 2 * d;
     const uint32_t n_ent = 2 + n_neg, n_slots = n_ent + d;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    double* sxo = reinterpret_cast<double*>(smem_raw) + (size_t)warp * 4 * d;
-    double* sxs = sxo + d;
-    double* sB = sxs + d;
-    double* sA = sB + d;
+    double* sxs = reinterpret_cast<double*>(smem_raw) + (size_t)warp * (2 * d + 32 * 33);
+    double* sA = sxs + d;
+    double* tile = sA + d;                                  // [32][33]
     const uint64_t n_warps = (uint64_t)gridDim.x * kWarps;
     double loss = 0;                                        // lane 0's
     for (uint64_t t = (uint64_t)blockIdx.x * kWarps + warp; t < n; t += n_warps) {
@@ -96,41 +97,47 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
 #pragma unroll
         for (int k = 0; k < kE; ++k) {
             const uint32_t e = lane + 32 * k;
-            if (e < d) { sxo[e] = xo[k]; sxs[e] = xs[k]; }
+            if (e < d) sxs[e] = xs[k];
         }
         __syncwarp();
-        // v = R y (lane per row) and z = R^T s (lane per column), y and s in shared memory
-        auto products = [&](const double* sy, const double* ss, double (&v)[kE], double (&z)[kE]) {
+        // v = R y and z = R^T s in one pass over the matrix, row by row (coalesced: a lane reads its columns of the
+        // row).  The lane's columns' share of the row's dot product with y goes to a 32 x 32 tile of the warp, and
+        // after 32 rows lane j adds up row j's shares, in lane order.  y: the lanes' elements; s: in shared memory.
+        auto products = [&](const double (&y)[kE], const double* ss, double (&v)[kE], double (&z)[kE]) {
 #pragma unroll
             for (int k = 0; k < kE; ++k) v[k] = z[k] = 0;
-            for (uint32_t b4 = 0; b4 < d4; ++b4) {
-                const double2 y01 = *reinterpret_cast<const double2*>(sy + 4 * b4);
-                const double2 y23 = *reinterpret_cast<const double2*>(sy + 4 * b4 + 2);
 #pragma unroll
-                for (int k = 0; k < kE; ++k) {
-                    if ((uint32_t)(lane + 32 * k) < d) {
-                        const float4 r = *reinterpret_cast<const float4*>(rowp[k] + 4 * b4);
-                        v[k] += (double)r.x * y01.x + (double)r.y * y01.y + (double)r.z * y23.x + (double)r.w * y23.y;
+            for (int kk = 0; kk < kE; ++kk) {
+                const uint32_t a0 = 32u * kk;               // the rows a0 .. a0 + 31 are the lanes' rows number kk
+                if (a0 >= d) break;
+                const uint32_t cnt = d - a0 < 32u ? d - a0 : 32u;
+#pragma unroll 4
+                for (uint32_t j = 0; j < cnt; ++j) {
+                    const float* ra = reinterpret_cast<const float*>(__shfl_sync(full, (unsigned long long)rowp[kk], j));
+                    const double sa = ss[a0 + j];
+                    double p = 0;
+#pragma unroll
+                    for (int k = 0; k < kE; ++k) {
+                        if ((uint32_t)(lane + 32 * k) < d) {
+                            const double r = (double)ra[lane + 32 * k];
+                            z[k] += sa * r;
+                            p += r * y[k];
+                        }
                     }
+                    tile[j * 33 + lane] = p;
                 }
-            }
-            for (uint32_t a0 = 0; a0 < d; a0 += 32) {
-#pragma unroll
-                for (int kk = 0; kk < kE; ++kk) {
-                    if (a0 != 32u * kk) continue;           // the rows a0 .. a0 + 31 are the lanes' rows number kk
-                    const uint32_t cnt = d - a0 < 32u ? d - a0 : 32u;
-                    for (uint32_t j = 0; j < cnt; ++j) {
-                        const float* ra = reinterpret_cast<const float*>(__shfl_sync(full, (unsigned long long)rowp[kk], j));
-                        const double sa = ss[a0 + j];
-#pragma unroll
-                        for (int k = 0; k < kE; ++k)
-                            if ((uint32_t)(lane + 32 * k) < d) z[k] += sa * (double)ra[lane + 32 * k];
-                    }
+                __syncwarp();
+                if ((uint32_t)lane < cnt) {
+                    double acc = 0;
+#pragma unroll 8
+                    for (int l = 0; l < 32; ++l) acc += tile[lane * 33 + l];
+                    v[kk] = acc;
                 }
+                __syncwarp();
             }
         };
         double u[kE], w[kE];
-        products(sxo, sxs, u, w);
+        products(xo, sxs, u, w);
         // scores and their coefficients, one triple after the other; a, b' as they come
         double av[kE], bp[kE];
         double phi = 0;
@@ -164,14 +171,16 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
             }
         }
         if (lane == 0) loss += lsum;
+        double bv[kE];
 #pragma unroll
         for (int k = 0; k < kE; ++k) {
             const uint32_t e = lane + 32 * k;
-            if (e < d) { sB[e] = c_pos * xo[k] + bp[k]; sA[e] = av[k]; }
+            bv[k] = c_pos * xo[k] + bp[k];
+            if (e < d) sA[e] = av[k];
         }
         __syncwarp();
         double gs[kE], go[kE];
-        products(sB, sA, gs, go);                           // R b, R^T a
+        products(bv, sA, gs, go);                           // R b, R^T a
         // the four numbers of every slot, folded into the first slot of its key (lane v: the numbers of slot v)
         double c1 = 0, c2 = 0, c3 = 0, c4 = 0;
         for (int z = 0; z < (int)n_ent; ++z) {
@@ -197,6 +206,7 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
         }
         // matrix rows: a[alpha] x_o + x_s[alpha] b'
         float* outR = out + (uint64_t)n_ent * d;
+#pragma unroll 4
         for (uint32_t al = 0; al < d; ++al) {
             const double aa = sA[al], sa = sxs[al];
 #pragma unroll
@@ -264,6 +274,8 @@ uint32_t launch_grad_rescal(ps_store* ps, const uint32_t* d_s, const uint32_t* d
     const uint32_t grid = (uint32_t)g;
 #define RESCAL_LAUNCH(kE)                                                                                           \
     do {                                                                                                            \
+        static std::atomic<unsigned long long> smem_set{0};                                                         \
+        opt_in_smem((const void*)rescal_grad_kernel<kE>, rescal_smem(128), &smem_set);                              \
         if (ps->prof) prof_before(ps, "rescal_grad_kernel<" #kE ">", s);                                            \
         rescal_grad_kernel<kE><<<grid, kRescalThreads, smem, s>>>(                                                  \
             d_s, d_r, d_o, d_neg_ent, d_neg_side, n, n_neg, rel_key_base, dim, (const float*)ps->store, ps->table,  \
