@@ -37,6 +37,7 @@ __device__ __forceinline__ double rescal_sigmoid(double z) {
 
 constexpr int kRescalThreads = 256;
 constexpr int kRescalMaxNeg = 29;
+constexpr int kBatch = 8;             // matrix rows whose loads a warp has in flight together
 
 // shared memory of a warp, fp64: x_s and a (read as broadcasts by the lanes), and a 32 x 33 tile
 __host__ __device__ inline size_t rescal_smem(uint32_t d) {
@@ -111,20 +112,32 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
                 const uint32_t a0 = 32u * kk;               // the rows a0 .. a0 + 31 are the lanes' rows number kk
                 if (a0 >= d) break;
                 const uint32_t cnt = d - a0 < 32u ? d - a0 : 32u;
-#pragma unroll 4
-                for (uint32_t j = 0; j < cnt; ++j) {
-                    const float* ra = reinterpret_cast<const float*>(__shfl_sync(full, (unsigned long long)rowp[kk], j));
-                    const double sa = ss[a0 + j];
-                    double p = 0;
+                // kBatch rows at a time: all their loads are issued before the first is used
+                for (uint32_t j0 = 0; j0 < cnt; j0 += kBatch) {
+                    const float* ra[kBatch];
+                    float r[kBatch][kE];
 #pragma unroll
-                    for (int k = 0; k < kE; ++k) {
-                        if ((uint32_t)(lane + 32 * k) < d) {
-                            const double r = (double)ra[lane + 32 * k];
-                            z[k] += sa * r;
-                            p += r * y[k];
-                        }
+                    for (int i = 0; i < kBatch; ++i) {
+                        const uint32_t j = j0 + i < cnt ? j0 + i : cnt - 1;
+                        ra[i] = reinterpret_cast<const float*>(__shfl_sync(full, (unsigned long long)rowp[kk], j));
                     }
-                    tile[j * 33 + lane] = p;
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i)
+#pragma unroll
+                        for (int k = 0; k < kE; ++k) r[i][k] = (uint32_t)(lane + 32 * k) < d ? __ldg(ra[i] + lane + 32 * k) : 0.f;
+#pragma unroll
+                    for (int i = 0; i < kBatch; ++i) {
+                        if (j0 + i >= cnt) break;
+                        const double sa = ss[a0 + j0 + i];
+                        double p = 0;
+#pragma unroll
+                        for (int k = 0; k < kE; ++k) {
+                            const double rv = (double)r[i][k];
+                            z[k] += sa * rv;
+                            p += rv * y[k];
+                        }
+                        tile[(j0 + i) * 33 + lane] = p;
+                    }
                 }
                 __syncwarp();
                 if ((uint32_t)lane < cnt) {
@@ -204,15 +217,28 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
                 if (e < d) out[(size_t)v * d + e] = (float)(f1 * gs[k] + f2 * go[k] + f3 * u[k] + f4 * w[k]);
             }
         }
-        // matrix rows: a[alpha] x_o + x_s[alpha] b'
+        // matrix rows: a[alpha] x_o + x_s[alpha] b', written as float4: x_o and b' go through the tile so that a lane
+        // holds four consecutive columns
         float* outR = out + (uint64_t)n_ent * d;
-#pragma unroll 4
-        for (uint32_t al = 0; al < d; ++al) {
-            const double aa = sA[al], sa = sxs[al];
+        __syncwarp();
 #pragma unroll
-            for (int k = 0; k < kE; ++k) {
-                const uint32_t e = lane + 32 * k;
-                if (e < d) outR[(size_t)al * d + e] = (float)(aa * xo[k] + sa * bp[k]);
+        for (int k = 0; k < kE; ++k) {
+            const uint32_t e = lane + 32 * k;
+            if (e < d) { tile[e] = xo[k]; tile[d + e] = bp[k]; }
+        }
+        __syncwarp();
+        if ((uint32_t)lane < d / 4) {
+            const double o0 = tile[4 * lane], o1 = tile[4 * lane + 1], o2 = tile[4 * lane + 2], o3 = tile[4 * lane + 3];
+            const double b0 = tile[d + 4 * lane], b1 = tile[d + 4 * lane + 1], b2 = tile[d + 4 * lane + 2], b3 = tile[d + 4 * lane + 3];
+#pragma unroll 4
+            for (uint32_t al = 0; al < d; ++al) {
+                const double aa = sA[al], sa = sxs[al];
+                float4 g;
+                g.x = (float)(aa * o0 + sa * b0);
+                g.y = (float)(aa * o1 + sa * b1);
+                g.z = (float)(aa * o2 + sa * b2);
+                g.w = (float)(aa * o3 + sa * b3);
+                *reinterpret_cast<float4*>(outR + (size_t)al * d + 4 * lane) = g;
             }
         }
     }
