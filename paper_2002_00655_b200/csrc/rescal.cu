@@ -151,36 +151,49 @@ rescal_grad_kernel(const uint32_t* __restrict__ ts, const uint32_t* __restrict__
         };
         double u[kE], w[kE];
         products(xo, sxs, u, w);
-        // scores and their coefficients, one triple after the other; a, b' as they come
-        double av[kE], bp[kE];
-        double phi = 0;
+        // scores: lane 1 keeps the positive's, lane 2 + q negative q's; then every lane forms its triple's coefficient
+        // and loss term (the exponentials once per data point, not once per triple); then a and b'
+        double phi_mine = 0;
+        {
+            double p = 0;
 #pragma unroll
-        for (int k = 0; k < kE; ++k) phi += xs[k] * u[k];
-        phi = warp_sum_d(phi);
-        const double c_pos = -rescal_sigmoid(-phi);
-        double my_coef = 0;                                 // lane 2 + q: the coefficient of negative q
-        double lsum = rescal_softplus(-phi);
+            for (int k = 0; k < kE; ++k) p += xs[k] * u[k];
+            p = warp_sum_d(p);
+            if (lane == 1) phi_mine = p;
+        }
+        for (uint32_t q = 0; q < n_neg; ++q) {
+            const float* pk = store + __shfl_sync(full, erow, 2 + q) * L;
+            const bool subj = __shfl_sync(full, side, 2 + q) == 0u;
+            double p = 0;
+#pragma unroll
+            for (int k = 0; k < kE; ++k) {
+                const uint32_t e = lane + 32 * k;
+                if (e < d) p += (double)pk[e] * (subj ? u[k] : w[k]);
+            }
+            p = warp_sum_d(p);
+            if (lane == (int)(2 + q)) phi_mine = p;
+        }
+        double my_coef = 0, my_loss = 0;                    // d loss / d phi and the loss term of this lane's triple
+        if (lane >= 1 && lane < (int)n_ent) {
+            const double y = lane == 1 ? 1.0 : -1.0;
+            my_coef = -y * rescal_sigmoid(-y * phi_mine);
+            my_loss = rescal_softplus(-y * phi_mine);
+        }
+        const double lsum = warp_sum_d(my_loss);
+        const double c_pos = __shfl_sync(full, my_coef, 1);
+        double av[kE], bp[kE];
 #pragma unroll
         for (int k = 0; k < kE; ++k) { av[k] = c_pos * xs[k]; bp[k] = 0; }
         for (uint32_t q = 0; q < n_neg; ++q) {
             const float* pk = store + __shfl_sync(full, erow, 2 + q) * L;
             const bool subj = __shfl_sync(full, side, 2 + q) == 0u;
-            double xk[kE];
-            double p = 0;
+            const double cq = __shfl_sync(full, my_coef, 2 + q);
 #pragma unroll
             for (int k = 0; k < kE; ++k) {
                 const uint32_t e = lane + 32 * k;
-                xk[k] = e < d ? (double)pk[e] : 0.0;
-                p += xk[k] * (subj ? u[k] : w[k]);
-            }
-            p = warp_sum_d(p);
-            const double cq = rescal_sigmoid(p);            // y = -1: d softplus(phi) / d phi
-            lsum += rescal_softplus(p);
-            if (lane == (int)(2 + q)) my_coef = cq;
-#pragma unroll
-            for (int k = 0; k < kE; ++k) {
-                if (subj) av[k] += cq * xk[k];
-                else bp[k] += cq * xk[k];
+                const double xk = e < d ? (double)pk[e] : 0.0;
+                if (subj) av[k] += cq * xk;
+                else bp[k] += cq * xk;
             }
         }
         if (lane == 0) loss += lsum;
