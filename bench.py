@@ -118,6 +118,7 @@ def smi_clocks():
 TRAFFIC = {
     ("mf_large", "mf_sub_kernel<4,gather4>"): 46.1e6,                 # profiles/mf_step_kernels_ncu_full.md (same-batch twin)
     ("kge", "kge_reduce_kernel<2>"): 321.6e6,                   # profiles/kge_step_kernels_ncu_full.md
+    ("rescal", "rescal_grad_kernel<4>"): 501.4e6,               # profiles/rescal_step_kernels_ncu_full.md
     ("sgns", "push_reduce_kernel<3,true>"): 1561.1e6,           # profiles/sgns_step_kernels_ncu_full.md
 }
 
