@@ -60,6 +60,18 @@ def test_rescal_single_steps(d, n_neg, batch, ents, rels, G):
     rescal_run(d, n_neg, batch, ents, rels, steps=3, single_step=True, G=G)
 
 
+def test_rescal_seeded_random_shapes():
+    """Single steps on a dozen seeded shapes: every fourth dimension up to 128, zero to 29 negatives, few to many
+    entities (slots of a data point that share a key), one to nine relations."""
+    r = np.random.RandomState(20260104)
+    for _ in range(12):
+        d = 4 * int(r.randint(1, 33))
+        n_neg = int(r.randint(0, 30))
+        batch = int(r.randint(1, 120))
+        ents = int(round(10 ** r.uniform(0.7, 3.3)))
+        rescal_run(d, n_neg, batch, ents, int(r.randint(1, 10)), steps=2, single_step=True, G=float(r.choice([0.0, 0.3])))
+
+
 def test_rescal_free_running_with_relocations():
     """Four steps without re-synchronising the two sides, keys relocated between the steps on a store of 8 partitions
     (location transparency, Section 2.3).  As for ComplEx, a first AdaGrad step on a gradient component near zero
