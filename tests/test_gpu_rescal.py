@@ -107,3 +107,42 @@ def test_rescal_bad_index_and_unsupported_shapes():
     o.step_rescal(s.cpu(), r_ok.cpu(), t.cpu(), neg.cpu(), side.cpu(), ents, d, 0.1, 1e-8)
     g.sync()
     compare_state(g, o, what="rescal step after the refused ones")
+
+
+def test_rescal_pipelined_ordered_and_graph_replay_agree_bit_for_bit():
+    """Eight steps with relocations in between: ordered calls, pipelined calls (the key kernel and the sort of step t+1
+    beside step t's kernels) and pipelined calls captured into one CUDA graph leave identical stores and losses."""
+    d, n_neg, batch, ents, rels, steps = 32, 6, 300, 400, 4, 8
+    cfg = W.scaled(W.KGE_TINY, entities=ents, relations=rels, dim=4, n_neg=n_neg, batch=batch, n_triples=steps * batch)
+    K = ents + rels * d
+    rows = rescal_rows(ents, rels, d, 9, 0.0)
+    data = [tuple(t.cuda() for t in W.kge_triples(cfg, *cfg.batch_range(b), "cpu")) for b in range(steps)]
+    loc_keys = dev(np.random.default_rng(4).integers(0, K, size=300))
+
+    def run(g, b):
+        ps.ps_step_rescal(g.h, *data[b], n_neg, ents, d, 0.1, 1e-8, g.loss)
+        if b % 3 == 1:
+            g.localize(b % 4, loc_keys)
+
+    stores = []
+    for mode in ("ordered", "pipelined", "graph"):
+        g, _ = make_pair(K, 2 * d, 4, K, rows=rows, max_batch_keys=(2 + n_neg + d) * batch)
+        ps.ps_set_pipelining(g.h, mode != "ordered")
+        if mode != "graph":
+            for b in range(steps):
+                run(g, b)
+        else:
+            run(g, 0)
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for b in range(1, steps - 1):
+                    run(g, b)
+            graph.replay()
+            torch.cuda.synchronize()
+            run(g, steps - 1)
+        g.sync()
+        stores.append((g.export(), loss_of(g)))
+    for (e, l), what in zip(stores[1:], ("pipelined", "graph replay")):
+        assert all((x == y).all() for x, y in zip(stores[0][0], e)), f"{what} differs from ordered calls"
+        assert l == stores[0][1]
