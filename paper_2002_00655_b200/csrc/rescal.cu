@@ -16,9 +16,11 @@
 //
 // One WARP works on one data point at a time, with no block-wide synchronisation (a block of eight warps per data
 // point, the matrix in shared memory or in registers, spent its time in a dozen dependent phases: 660-700 us per
-// step of 8,192 data points).  Lane l holds elements l, l + 32, l + 64, l + 96 of every vector, in fp64.  A product
-// with R takes a lane per row (the lane reads its rows front to back, the vector comes from shared memory as
-// broadcasts), a product with R^T a lane per column (row by row, coalesced); neither needs a sum across lanes.
+// step of 8,192 data points).  Lane l holds elements l, l + 32, l + 64, l + 96 of every vector, in fp64.  A pass over
+// the matrix goes row by row, coalesced (a lane reads its columns of the row, the loads of eight rows are issued
+// before the first is used) and gives two products at once: the row's dot product with a vector (the lanes' shares go
+// through a 32 x 33 tile of the warp and one lane adds a row's shares in lane order) and the product of the transpose
+// with another vector (a lane accumulates its columns).  Two passes per data point.
 // The gradient of an entity slot is c1 (R b) + c2 (R^T a) + c3 u + c4 w with four numbers per slot, so slots that
 // hold the same entity are folded by adding their numbers, and no gradient is stored before it is final.  Written per
 // occurrence slot (2 + n_neg entity slots, then d matrix rows): the gradient row of d values; the ComplEx path's
